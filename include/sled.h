@@ -1,0 +1,228 @@
+/*
+ * sled.h -- C boundary of the batched verification step of SLED's edge server.
+ *
+ * The paper (Section 3.2) states the server's job: edge devices send the draft
+ * tokens they generated, one shared target model verifies the drafts of many
+ * devices together (Section 3.4), and each device gets back the position of its
+ * first rejected token and the corrective token.  Acceptance follows Eq. 1 of
+ * Section 3.1 (accept a draft x with probability min(1, p_target(x)/p_draft(x)),
+ * on a rejection draw the replacement from the normalised positive part of
+ * p_target - p_draft); when every draft is accepted one more token is drawn from
+ * the target distribution that follows them.
+ *
+ * All entry points are plain C: fixed-width integers, raw pointers, an opaque
+ * engine handle.  Unless a parameter says otherwise a pointer is a HOST pointer.
+ * Every function returns SLED_OK (0) or a negative sled_status; a failed call
+ * changes no context, page or counter.  An engine is used by one thread at a
+ * time.  All device work is issued on the engine's stream.
+ */
+#ifndef SLED_H_
+#define SLED_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sled_engine sled_engine;
+typedef struct sled_kvm sled_kvm;
+
+enum sled_status {
+  SLED_OK = 0,
+  SLED_ERR_ARG = -1,          /* null pointer, bad size, unsupported shape */
+  SLED_ERR_UNKNOWN_CTX = -2,  /* ctx_id not open */
+  SLED_ERR_DUP_CTX = -3,      /* ctx_id twice in one batch, or opened twice */
+  SLED_ERR_K_RANGE = -4,      /* k < 0 or k > max_k */
+  SLED_ERR_TOKEN_RANGE = -5,  /* token id outside [0, vocab) */
+  SLED_ERR_NO_PAGES = -6,     /* KV pool exhausted */
+  SLED_ERR_BATCH_TOO_LARGE = -7, /* n_reqs > max_batch or sum(k_i + 1) > max_step_tokens */
+  SLED_ERR_NONFINITE = -8,    /* per-request status: a logit that had to be read was NaN or Inf */
+  SLED_ERR_DEVICE = -9,       /* CUDA error, or a bounded device-side wait ran out */
+  SLED_ERR_NO_DEVICE = -10    /* no usable CUDA device: there is no CPU fallback */
+};
+
+enum sled_dtype { SLED_F32 = 0, SLED_BF16 = 1 };
+
+/* Shape of the Llama-style target model and the engine's capacities.
+ * (The paper fixes only "Llama family", Section 4; shapes come from the workload.) */
+typedef struct sled_config {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, ffn_dim, vocab;
+  float rms_eps;          /* RMSNorm epsilon */
+  float rope_theta;       /* rotary base; pairs (2i, 2i+1) rotate by pos * theta^(-2i/head_dim) */
+  int32_t weight_dtype;   /* sled_dtype of every array in sled_weights; SLED_BF16 runs the linear
+                             layers on the tensor cores with bf16 activations and fp32 accumulation,
+                             SLED_F32 keeps everything in fp32 */
+  int32_t kv_dtype;       /* sled_dtype of the cached keys and values */
+  int32_t page_size;      /* tokens per KV page (16) */
+  int32_t n_pages;        /* pages in the pool; one page holds page_size tokens of every layer */
+  int32_t max_batch;      /* most requests per sled_verify_batch */
+  int32_t max_k;          /* most draft tokens per request */
+  int32_t max_step_tokens;/* most sum(k_i + 1) per step; also the prefill chunk */
+  float temperature;      /* divides the target logits before the softmax (> 0) */
+  int32_t greedy;         /* 1: accept iff the draft equals the argmax, emit the argmax */
+  int32_t probs_on_device;/* 1: sled_request.draft_probs are DEVICE pointers */
+  int32_t device_index;   /* CUDA device ordinal */
+  void* stream;           /* cudaStream_t to launch on; NULL: the engine creates one */
+} sled_config;
+
+/* Target weights, row-major [out][in], all of type weight_dtype.  HOST or DEVICE
+ * pointers (found out per pointer).  Copied during sled_init: the caller may free
+ * them when it returns.  Per-layer members point to arrays of n_layers pointers. */
+typedef struct sled_weights {
+  const void* tok_emb;            /* [vocab][d_model] */
+  const void* final_norm;         /* [d_model] */
+  const void* lm_head;            /* [vocab][d_model] */
+  const void* const* attn_norm;   /* [d_model] */
+  const void* const* wq;          /* [n_q_heads*head_dim][d_model] */
+  const void* const* wk;          /* [n_kv_heads*head_dim][d_model] */
+  const void* const* wv;          /* [n_kv_heads*head_dim][d_model] */
+  const void* const* wo;          /* [d_model][n_q_heads*head_dim] */
+  const void* const* ffn_norm;    /* [d_model] */
+  const void* const* w_gate;      /* [ffn_dim][d_model] */
+  const void* const* w_up;        /* [ffn_dim][d_model] */
+  const void* const* w_down;      /* [d_model][ffn_dim] */
+} sled_weights;
+
+/* One device's verification request (Section 3.2: the draft tokens it sends;
+ * Eq. 1 needs the draft model's distribution at each of them as well).  All
+ * devices share the target's tokenizer (Section 3.4), so a row of draft_probs
+ * has exactly `vocab` entries.  Borrowed for the duration of the call. */
+typedef struct sled_request {
+  uint64_t ctx_id;             /* context opened by sled_prefill */
+  const int32_t* draft_tokens; /* [k], host */
+  const float* draft_probs;    /* [k][vocab] fp32, rows sum to 1; host, or device if probs_on_device;
+                                  may be NULL when k == 0 or in greedy mode */
+  int32_t k;                   /* 0 <= k <= max_k; k = 0 is an ordinary decoding step */
+} sled_request;
+
+/* The feedback of Section 3.2: how many drafts were accepted (the first rejected
+ * one is draft n_accepted + 1) and the corrective token, or the bonus token when
+ * n_accepted == k. */
+typedef struct sled_result {
+  int32_t n_accepted;
+  int32_t next_token;
+  int32_t status;   /* SLED_OK or SLED_ERR_NONFINITE (then nothing of this request is committed) */
+} sled_result;
+
+typedef struct sled_stats {
+  int64_t steps, requests, tokens_scored, drafts_accepted, tokens_committed;
+  int32_t pages_total, pages_free, contexts_open;
+  int64_t kernels_launched;    /* device kernels launched by this engine so far */
+  int64_t kernels_last_step;   /* ... by the last sled_verify_batch */
+  /* device time of the last step by kind, filled when sled_debug_set_timing(1) */
+  float ms_linear, ms_attention, ms_accept, ms_other, ms_step;
+  int32_t linear_launches_last_step, attention_launches_last_step;
+} sled_stats;
+
+/* ---- the three calls of the verification service ---------------------------------- */
+
+/* Creates an engine: checks cfg, allocates weights, KV pool and workspaces on
+ * cfg->device_index, copies the weights.  Errors: SLED_ERR_ARG, SLED_ERR_NO_DEVICE,
+ * SLED_ERR_DEVICE (allocation failed: nothing is left allocated). */
+int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out);
+
+/* One batched verification step (Sections 3.1, 3.4).  For request i the target is
+ * evaluated at the k_i + 1 tokens [pending_i, d_1..d_k] in one ragged pass over all
+ * requests (no padding to a common length); draft j of context i is decided with the
+ * Philox4x32-10 uniforms of (seed, ctx_id, absolute position of that token), so a
+ * request's outcome does not depend on its batch slot or on the other requests.
+ * Afterwards the KV entries of pending_i and of the accepted drafts are kept, those
+ * of the rejected drafts are dropped, pages left empty return to the pool, and
+ * next_token becomes the context's pending token.  results: caller-allocated [n_reqs].
+ * All requests are validated and all pages reserved before anything changes. */
+int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, uint64_t seed,
+                      sled_result* results);
+
+/* Closes a context: its pages return to the pool. */
+int sled_release(sled_engine* e, uint64_t ctx_id);
+
+/* ---- what makes the three usable --------------------------------------------------- */
+
+/* Opens a context from a device's prompt (Section 3.2: prompts are tokenised on the
+ * device): caches the keys/values of tokens[0..n-2]; tokens[n-1] becomes the pending
+ * token, fed first by the next verification.  n >= 1. */
+int sled_prefill(sled_engine* e, uint64_t ctx_id, const int32_t* tokens, int32_t n);
+
+int sled_set_sampling(sled_engine* e, float temperature, int32_t greedy);
+int sled_get_stats(sled_engine* e, sled_stats* out);
+/* cudaStream_t all work of this engine is issued on (for timing with events). */
+void* sled_get_stream(sled_engine* e);
+void sled_shutdown(sled_engine* e);
+const char* sled_strerror(int status);
+
+/* ---- stand-alone pieces of the step (device-resident operands) ---------------------- */
+
+/* Acceptance only (Eq. 1 + residual / bonus draw) on logits already in device memory.
+ *   logits   DEVICE [n_rows][vocab] fp32, request i owns rows cu_rows[i] .. cu_rows[i+1]-1
+ *            (k_i + 1 rows: row j scores draft j+1, the last one the bonus token)
+ *   cu_rows  HOST [n_reqs+1];  drafts HOST [n_rows - n_reqs] packed request after request
+ *   q_rows   DEVICE [sum k_i][vocab] fp32 packed the same way (NULL if greedy)
+ *   ctx_ids, pos0 HOST [n_reqs]: Philox counter words; pos0 = index of the pending token
+ *   results  HOST [n_reqs]
+ * stream: cudaStream_t or NULL for the default stream.  device_ms (may be NULL) receives the
+ * kernel's duration measured with events on that stream.  Synchronises before returning. */
+int sled_accept_rows(const float* logits, const int32_t* cu_rows, const int32_t* drafts, const float* q_rows,
+                     const uint64_t* ctx_ids, const int64_t* pos0, int32_t n_reqs, int32_t vocab,
+                     float temperature, int32_t greedy, uint64_t seed, sled_result* results, void* stream,
+                     float* device_ms);
+
+/* Ragged verification attention only, over the engine's paged cache: request i's last
+ * q_len[i] cached tokens are taken as the new ones; query j of request i attends to the
+ * keys 0 .. n_kv_i - q_len_i + j of ctx_ids[i] in layer `layer`.
+ *   q    DEVICE [sum q_len][n_q_heads][head_dim] in the activation type (bf16 with bf16 weights)
+ *   out  DEVICE same shape and type.
+ * device_ms (may be NULL) receives the duration of the attention kernels (events on the
+ * engine's stream).  Synchronises before returning. */
+int sled_attention_ragged(sled_engine* e, int32_t layer, const uint64_t* ctx_ids, const int32_t* q_len,
+                          int32_t n_reqs, const void* q, void* out, float* device_ms);
+
+/* ---- test and benchmark hooks ------------------------------------------------------- */
+
+/* Opens a context with given cache content instead of a prefill.  K, V: HOST or DEVICE,
+ * [n_layers][n_tokens][n_kv_heads][head_dim] of kv_dtype. */
+int sled_debug_load_kv(sled_engine* e, uint64_t ctx_id, const void* K, const void* V, int32_t n_tokens,
+                       int32_t pending);
+/* Reads one layer's cache of a context back: K, V HOST [n_tokens][n_kv_heads][head_dim] of kv_dtype. */
+int sled_debug_read_kv(sled_engine* e, uint64_t ctx_id, int32_t layer, void* K, void* V, int32_t n_tokens);
+/* Copies the logits of the last step, rows [0, n_rows), to dst (HOST or DEVICE) [n_rows][vocab] fp32. */
+int sled_debug_copy_logits(sled_engine* e, float* dst, int32_t n_rows);
+/* Sets a context back to n_kv cached tokens (<= its current count) and a pending token. */
+int sled_debug_truncate(sled_engine* e, uint64_t ctx_id, int64_t n_kv, int32_t pending);
+/* commit = 0: verification steps leave every context as it was (repeatable timing). */
+int sled_debug_set_commit(sled_engine* e, int32_t commit);
+/* on = 1: record device time per kernel kind into sled_stats (adds events between kernels). */
+int sled_debug_set_timing(sled_engine* e, int32_t on);
+/* Context state: cached tokens, pending token, owned pages (ids into pages_out, up to cap). */
+int sled_debug_query_ctx(sled_engine* e, uint64_t ctx_id, int64_t* n_kv, int32_t* pending, int32_t* n_pages,
+                         int32_t* pages_out, int32_t cap);
+
+/* Permutes the free-page list (seeded), so contexts opened afterwards get physically scattered pages. */
+int sled_debug_shuffle_pages(sled_engine* e, uint64_t seed);
+
+/* ---- host-side KV page manager (no device needed) ----------------------------------- */
+/* The bookkeeping the engine uses for commit / rollback, exported so it can be
+ * exercised alone.  A context owns ceil(tokens / page_size) pages; pages are handed out
+ * and returned whole; a batch reservation either fits entirely or changes nothing. */
+sled_kvm* sled_kvm_create(int32_t n_pages, int32_t page_size);
+void sled_kvm_destroy(sled_kvm* m);
+int sled_kvm_open(sled_kvm* m, uint64_t ctx_id, int64_t n_kv, int32_t pending);
+/* Reserves room for extra[i] more tokens behind the cached ones of each context. */
+int sled_kvm_reserve_batch(sled_kvm* m, const uint64_t* ctx_ids, const int32_t* extra, int32_t n);
+/* Keeps n_keep of the reserved tokens, returns pages that no longer hold any, sets pending. */
+int sled_kvm_commit(sled_kvm* m, uint64_t ctx_id, int32_t n_keep, int32_t pending);
+int sled_kvm_release(sled_kvm* m, uint64_t ctx_id);
+int sled_kvm_query(sled_kvm* m, uint64_t ctx_id, int64_t* n_kv, int32_t* pending, int32_t* n_pages,
+                   int32_t* pages_out, int32_t cap);
+int32_t sled_kvm_free_pages(sled_kvm* m);
+/* Ragged packing of one step: for request i with k[i] drafts, writes token rows
+ * cu_q[i] .. cu_q[i+1]-1 (row 0 = pending token, then the drafts): ids, owning request,
+ * absolute position and physical cache slot (page * page_size + offset).  Pages must have
+ * been reserved.  Output arrays: cu_q [n+1], others [sum(k_i+1)]. */
+int sled_kvm_pack(sled_kvm* m, const uint64_t* ctx_ids, const int32_t* k, const int32_t* const* drafts, int32_t n,
+                  int32_t* cu_q, int32_t* ids, int32_t* tok_req, int32_t* tok_pos, int32_t* tok_slot);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLED_H_ */

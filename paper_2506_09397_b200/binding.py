@@ -1,0 +1,340 @@
+"""Thin ctypes binding of libsled.so: same names as include/sled.h, argument marshalling only.
+
+Every step of the verification path runs inside the CUDA library; this module only turns
+Python objects into the plain pointers and sizes the C boundary takes.  There is no CPU
+fallback: loading fails loudly when the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsled.so")
+
+SLED_OK = 0
+SLED_ERR_ARG, SLED_ERR_UNKNOWN_CTX, SLED_ERR_DUP_CTX, SLED_ERR_K_RANGE, SLED_ERR_TOKEN_RANGE = -1, -2, -3, -4, -5
+SLED_ERR_NO_PAGES, SLED_ERR_BATCH_TOO_LARGE, SLED_ERR_NONFINITE, SLED_ERR_DEVICE, SLED_ERR_NO_DEVICE = -6, -7, -8, -9, -10
+SLED_F32, SLED_BF16 = 0, 1
+
+EXPORTS = (
+    "sled_init", "sled_verify_batch", "sled_release", "sled_prefill", "sled_set_sampling", "sled_get_stats",
+    "sled_get_stream", "sled_shutdown", "sled_strerror", "sled_accept_rows", "sled_attention_ragged",
+    "sled_debug_load_kv", "sled_debug_read_kv", "sled_debug_copy_logits", "sled_debug_truncate",
+    "sled_debug_set_commit", "sled_debug_set_timing", "sled_debug_query_ctx", "sled_debug_shuffle_pages",
+    "sled_kvm_create", "sled_kvm_destroy", "sled_kvm_open", "sled_kvm_reserve_batch", "sled_kvm_commit",
+    "sled_kvm_release", "sled_kvm_query", "sled_kvm_free_pages", "sled_kvm_pack",
+)
+
+
+class SledConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "ffn_dim", "vocab")] + [
+        ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("weight_dtype", C.c_int32), ("kv_dtype", C.c_int32),
+        ("page_size", C.c_int32), ("n_pages", C.c_int32), ("max_batch", C.c_int32), ("max_k", C.c_int32),
+        ("max_step_tokens", C.c_int32), ("temperature", C.c_float), ("greedy", C.c_int32),
+        ("probs_on_device", C.c_int32), ("device_index", C.c_int32), ("stream", C.c_void_p)]
+
+
+class SledWeights(C.Structure):
+    _fields_ = [("tok_emb", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p)] + [
+        (n, C.POINTER(C.c_void_p)) for n in
+        ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")]
+
+
+class SledRequest(C.Structure):
+    _fields_ = [("ctx_id", C.c_uint64), ("draft_tokens", C.c_void_p), ("draft_probs", C.c_void_p), ("k", C.c_int32)]
+
+
+class SledResult(C.Structure):
+    _fields_ = [("n_accepted", C.c_int32), ("next_token", C.c_int32), ("status", C.c_int32)]
+
+
+class SledStats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("steps", "requests", "tokens_scored", "drafts_accepted", "tokens_committed")] + [
+        (n, C.c_int32) for n in ("pages_total", "pages_free", "contexts_open")] + [
+        ("kernels_launched", C.c_int64), ("kernels_last_step", C.c_int64)] + [
+        (n, C.c_float) for n in ("ms_linear", "ms_attention", "ms_accept", "ms_other", "ms_step")] + [
+        ("linear_launches_last_step", C.c_int32), ("attention_launches_last_step", C.c_int32)]
+
+
+class SledError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def lib():
+    """Loads libsled.so (raises if it has not been built: nothing else can run the path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with paper_2506_09397_b200.build.build(); "
+                               "there is no fallback implementation")
+        L = C.CDLL(LIB_PATH)
+        P, I32, I64, U64, F = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64, C.c_float
+        sig = {
+            "sled_init": (C.c_int, [C.POINTER(SledWeights), C.POINTER(SledConfig), C.POINTER(P)]),
+            "sled_verify_batch": (C.c_int, [P, C.POINTER(SledRequest), I32, U64, C.POINTER(SledResult)]),
+            "sled_release": (C.c_int, [P, U64]),
+            "sled_prefill": (C.c_int, [P, U64, P, I32]),
+            "sled_set_sampling": (C.c_int, [P, F, I32]),
+            "sled_get_stats": (C.c_int, [P, C.POINTER(SledStats)]),
+            "sled_get_stream": (P, [P]),
+            "sled_shutdown": (None, [P]),
+            "sled_strerror": (C.c_char_p, [C.c_int]),
+            "sled_accept_rows": (C.c_int, [P, P, P, P, P, P, I32, I32, F, I32, U64, C.POINTER(SledResult), P,
+                                           C.POINTER(F)]),
+            "sled_attention_ragged": (C.c_int, [P, I32, P, P, I32, P, P, C.POINTER(F)]),
+            "sled_debug_load_kv": (C.c_int, [P, U64, P, P, I32, I32]),
+            "sled_debug_read_kv": (C.c_int, [P, U64, I32, P, P, I32]),
+            "sled_debug_copy_logits": (C.c_int, [P, P, I32]),
+            "sled_debug_truncate": (C.c_int, [P, U64, I64, I32]),
+            "sled_debug_set_commit": (C.c_int, [P, I32]),
+            "sled_debug_set_timing": (C.c_int, [P, I32]),
+            "sled_debug_query_ctx": (C.c_int, [P, U64, C.POINTER(I64), C.POINTER(I32), C.POINTER(I32), P, I32]),
+            "sled_debug_shuffle_pages": (C.c_int, [P, U64]),
+            "sled_kvm_create": (P, [I32, I32]),
+            "sled_kvm_destroy": (None, [P]),
+            "sled_kvm_open": (C.c_int, [P, U64, I64, I32]),
+            "sled_kvm_reserve_batch": (C.c_int, [P, P, P, I32]),
+            "sled_kvm_commit": (C.c_int, [P, U64, I32, I32]),
+            "sled_kvm_release": (C.c_int, [P, U64]),
+            "sled_kvm_query": (C.c_int, [P, U64, C.POINTER(I64), C.POINTER(I32), C.POINTER(I32), P, I32]),
+            "sled_kvm_free_pages": (I32, [P]),
+            "sled_kvm_pack": (C.c_int, [P, P, P, P, I32, P, P, P, P, P]),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().sled_strerror(code).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != SLED_OK:
+        raise SledError(code, what)
+
+
+def _addr(t) -> int:
+    if t is None:
+        return 0
+    if isinstance(t, np.ndarray):
+        assert t.flags["C_CONTIGUOUS"]
+        return t.ctypes.data
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+_PER_LAYER = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
+_DT = {"fp32": SLED_F32, "bf16": SLED_BF16}
+
+
+class Engine:
+    """Owner of one sled_engine handle.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, shape, weights: dict, *, n_pages: int, max_batch: int, max_k: int, max_step_tokens: int,
+                 temperature: float = 1.0, greedy: bool = False, probs_on_device: bool = False, device_index: int = 0,
+                 page_size: int = 16, stream: int | None = None):
+        self.shape = shape
+        cfg = SledConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                         shape.ffn_dim, shape.vocab, shape.rms_eps, shape.rope_theta, _DT[shape.weight_dtype],
+                         _DT[shape.kv_dtype], page_size, n_pages, max_batch, max_k, max_step_tokens, temperature,
+                         int(greedy), int(probs_on_device), device_index, stream)
+        w = SledWeights()
+        w.tok_emb, w.final_norm, w.lm_head = _addr(weights["tok_emb"]), _addr(weights["final_norm"]), _addr(weights["lm_head"])
+        keep = []
+        for name in _PER_LAYER:
+            arr = (C.c_void_p * shape.n_layers)(*[_addr(t) for t in weights[name]])
+            keep.append(arr)
+            setattr(w, name, C.cast(arr, C.POINTER(C.c_void_p)))
+        h = C.c_void_p()
+        _check(lib().sled_init(C.byref(w), C.byref(cfg), C.byref(h)), "sled_init")
+        self.h = h
+        self.cfg = cfg
+        self.probs_on_device = probs_on_device
+
+    # -- the three calls
+    def verify_batch(self, requests, seed: int):
+        """requests: list of (ctx_id, draft_tokens int32 host array [k], draft_probs [k, V] fp32 or None).
+        Returns list of (n_accepted, next_token, status)."""
+        n = len(requests)
+        reqs = (SledRequest * max(n, 1))()
+        keep = []
+        for i, (ctx, toks, probs) in enumerate(requests):
+            toks = np.ascontiguousarray(np.asarray(toks, dtype=np.int32).reshape(-1))
+            keep.append(toks)
+            if probs is not None and not isinstance(probs, torch.Tensor):
+                probs = np.ascontiguousarray(probs, dtype=np.float32)
+                keep.append(probs)
+            reqs[i].ctx_id = ctx
+            reqs[i].draft_tokens = toks.ctypes.data if toks.size else None
+            reqs[i].draft_probs = _addr(probs) if probs is not None and toks.size else None
+            reqs[i].k = toks.size
+        res = (SledResult * max(n, 1))()
+        _check(lib().sled_verify_batch(self.h, reqs, n, seed, res), "sled_verify_batch")
+        return [(res[i].n_accepted, res[i].next_token, res[i].status) for i in range(n)]
+
+    def verify_batch_raw(self, reqs, n: int, seed: int, res) -> int:
+        """Pre-marshalled arrays (SledRequest * n, SledResult * n): the bare call, for timing."""
+        return lib().sled_verify_batch(self.h, reqs, n, seed, res)
+
+    def release(self, ctx_id: int) -> None:
+        _check(lib().sled_release(self.h, ctx_id), "sled_release")
+
+    def prefill(self, ctx_id: int, tokens) -> None:
+        t = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
+        _check(lib().sled_prefill(self.h, ctx_id, t.ctypes.data, t.size), "sled_prefill")
+
+    # -- the rest
+    def set_sampling(self, temperature: float, greedy: bool) -> None:
+        _check(lib().sled_set_sampling(self.h, temperature, int(greedy)), "sled_set_sampling")
+
+    def stats(self) -> SledStats:
+        s = SledStats()
+        _check(lib().sled_get_stats(self.h, C.byref(s)), "sled_get_stats")
+        return s
+
+    def stream(self) -> int:
+        return lib().sled_get_stream(self.h) or 0
+
+    def load_kv(self, ctx_id: int, K, V, pending: int) -> None:
+        n = K.shape[1]
+        _check(lib().sled_debug_load_kv(self.h, ctx_id, _addr(K), _addr(V), n, pending), "sled_debug_load_kv")
+
+    def read_kv(self, ctx_id: int, layer: int, n_tokens: int):
+        s = self.shape
+        dt = torch.bfloat16 if s.kv_dtype == "bf16" else torch.float32
+        K = torch.empty(n_tokens, s.n_kv_heads, s.head_dim, dtype=dt)
+        V = torch.empty_like(K)
+        _check(lib().sled_debug_read_kv(self.h, ctx_id, layer, K.data_ptr(), V.data_ptr(), n_tokens), "sled_debug_read_kv")
+        return K, V
+
+    def logits(self, n_rows: int) -> np.ndarray:
+        out = np.empty((n_rows, self.shape.vocab), dtype=np.float32)
+        _check(lib().sled_debug_copy_logits(self.h, out.ctypes.data, n_rows), "sled_debug_copy_logits")
+        return out
+
+    def truncate(self, ctx_id: int, n_kv: int, pending: int) -> None:
+        _check(lib().sled_debug_truncate(self.h, ctx_id, n_kv, pending), "sled_debug_truncate")
+
+    def set_commit(self, on: bool) -> None:
+        _check(lib().sled_debug_set_commit(self.h, int(on)), "sled_debug_set_commit")
+
+    def set_timing(self, on: bool) -> None:
+        _check(lib().sled_debug_set_timing(self.h, int(on)), "sled_debug_set_timing")
+
+    def shuffle_pages(self, seed: int) -> None:
+        _check(lib().sled_debug_shuffle_pages(self.h, seed), "sled_debug_shuffle_pages")
+
+    def query_ctx(self, ctx_id: int):
+        n_kv, pend, npg = C.c_int64(), C.c_int32(), C.c_int32()
+        _check(lib().sled_debug_query_ctx(self.h, ctx_id, C.byref(n_kv), C.byref(pend), C.byref(npg), None, 0),
+               "sled_debug_query_ctx")
+        pages = np.zeros(max(npg.value, 1), dtype=np.int32)
+        _check(lib().sled_debug_query_ctx(self.h, ctx_id, None, None, None, pages.ctypes.data, npg.value),
+               "sled_debug_query_ctx")
+        return n_kv.value, pend.value, pages[:npg.value].copy()
+
+    def attention_ragged(self, layer: int, ctx_ids, q_len, q: torch.Tensor, out: torch.Tensor) -> float:
+        ids = np.ascontiguousarray(np.asarray(ctx_ids, dtype=np.uint64))
+        ql = np.ascontiguousarray(np.asarray(q_len, dtype=np.int32))
+        ms = C.c_float()
+        _check(lib().sled_attention_ragged(self.h, layer, ids.ctypes.data, ql.ctypes.data, ids.size, q.data_ptr(),
+                                           out.data_ptr(), C.byref(ms)), "sled_attention_ragged")
+        return ms.value
+
+    def shutdown(self) -> None:
+        if self.h:
+            lib().sled_shutdown(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.shutdown()
+        except Exception:
+            pass
+
+
+def accept_rows(logits: torch.Tensor, cu_rows, drafts, q_rows, ctx_ids, pos0, temperature: float, greedy: bool,
+                seed: int, stream: int = 0):
+    """sled_accept_rows: logits [rows, V] and q_rows [sum k, V] are CUDA tensors, the rest host arrays.
+    Returns (list of (n_accepted, next_token, status), kernel milliseconds)."""
+    cu = np.ascontiguousarray(np.asarray(cu_rows, dtype=np.int32))
+    n = cu.size - 1
+    d = np.ascontiguousarray(np.asarray(drafts, dtype=np.int32).reshape(-1))
+    ids = np.ascontiguousarray(np.asarray(ctx_ids, dtype=np.uint64))
+    p0 = np.ascontiguousarray(np.asarray(pos0, dtype=np.int64))
+    res = (SledResult * n)()
+    ms = C.c_float()
+    _check(lib().sled_accept_rows(logits.data_ptr(), cu.ctypes.data, d.ctypes.data if d.size else None,
+                                  _addr(q_rows) if q_rows is not None else None, ids.ctypes.data, p0.ctypes.data, n,
+                                  logits.shape[1], temperature, int(greedy), seed, res, stream, C.byref(ms)),
+           "sled_accept_rows")
+    return [(res[i].n_accepted, res[i].next_token, res[i].status) for i in range(n)], ms.value
+
+
+class KvManager:
+    """The host-side page manager alone (sled_kvm_*): needs no device."""
+
+    def __init__(self, n_pages: int, page_size: int):
+        self.h = lib().sled_kvm_create(n_pages, page_size)
+        if not self.h:
+            raise SledError(SLED_ERR_ARG, "sled_kvm_create")
+
+    def open(self, ctx: int, n_kv: int, pending: int) -> int:
+        return lib().sled_kvm_open(self.h, ctx, n_kv, pending)
+
+    def reserve_batch(self, ctxs, extra) -> int:
+        c = np.ascontiguousarray(np.asarray(ctxs, dtype=np.uint64))
+        x = np.ascontiguousarray(np.asarray(extra, dtype=np.int32))
+        return lib().sled_kvm_reserve_batch(self.h, c.ctypes.data, x.ctypes.data, c.size)
+
+    def commit(self, ctx: int, n_keep: int, pending: int) -> int:
+        return lib().sled_kvm_commit(self.h, ctx, n_keep, pending)
+
+    def release(self, ctx: int) -> int:
+        return lib().sled_kvm_release(self.h, ctx)
+
+    def query(self, ctx: int):
+        n_kv, pend, npg = C.c_int64(), C.c_int32(), C.c_int32()
+        rc = lib().sled_kvm_query(self.h, ctx, C.byref(n_kv), C.byref(pend), C.byref(npg), None, 0)
+        if rc:
+            return rc, None
+        pages = np.zeros(max(npg.value, 1), dtype=np.int32)
+        lib().sled_kvm_query(self.h, ctx, None, None, None, pages.ctypes.data, npg.value)
+        return 0, (n_kv.value, pend.value, pages[:npg.value].copy())
+
+    def free_pages(self) -> int:
+        return lib().sled_kvm_free_pages(self.h)
+
+    def pack(self, ctxs, ks, drafts):
+        c = np.ascontiguousarray(np.asarray(ctxs, dtype=np.uint64))
+        k = np.ascontiguousarray(np.asarray(ks, dtype=np.int32))
+        n = c.size
+        T = int(k.sum()) + n
+        arrs = [np.ascontiguousarray(np.asarray(d, dtype=np.int32).reshape(-1)) for d in drafts]
+        ptrs = (C.c_void_p * max(n, 1))(*[a.ctypes.data if a.size else None for a in arrs])
+        cu = np.zeros(n + 1, np.int32)
+        out = [np.zeros(max(T, 1), np.int32) for _ in range(4)]
+        rc = lib().sled_kvm_pack(self.h, c.ctypes.data, k.ctypes.data, ptrs, n, cu.ctypes.data,
+                                 *[o.ctypes.data for o in out])
+        return rc, cu, [o[:T] for o in out]
+
+    def __del__(self):
+        try:
+            if self.h:
+                lib().sled_kvm_destroy(self.h)
+                self.h = None
+        except Exception:
+            pass

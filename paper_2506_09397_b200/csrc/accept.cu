@@ -1,0 +1,265 @@
+// Fused vocabulary softmax + speculative acceptance + corrective / bonus draw.
+//
+// One block per request walks its rows in order and stops at the deciding row: rows
+// behind the first rejection are never read.  All quantities that decide anything are
+// order-independent: the row maximum, integer softmax numerators E_v (a fixed sequence
+// of correctly rounded fp32 operations followed by an exact scaling to 2^40), their
+// exact 64-bit sum Z, and integer prefix sums for the inverse-CDF draw.  The accept test
+// u < p/q is evaluated as U * q_d * Z < E_d * 2^24 in fp64 with U the 24-bit uniform.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace sled {
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kVec = 4;                       // consecutive vocabulary entries per thread per tile
+constexpr int kTile = kThreads * kVec;        // 4096 entries per tile
+constexpr int kMaxTiles = 1024;               // vocabularies up to 4M entries
+
+enum { ST_OK = 0, ST_NONFINITE = -8 };
+
+__device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1, uint32_t c2,
+                                              uint32_t c3, uint32_t out[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// trunc(exp(x) * 2^40), x <= 0, by explicit round-to-nearest operations only
+__device__ __forceinline__ unsigned long long fixed_exp(float x) {
+  if (!(x >= -30.0f)) return 0ull;
+  const float shift = 12582912.0f;
+  const float t = __fmaf_rn(x, 0x1.715476p+0f, shift);   // log2(e)
+  const float nf = __fsub_rn(t, shift);
+  float r = __fmaf_rn(nf, -0x1.62e4p-1f, x);              // ln 2, high part
+  r = __fmaf_rn(nf, -0x1.7f7d1cp-20f, r);                 // ln 2, low part
+  float p = 0x1.6c16c2p-10f;                              // 1/720
+  p = __fmaf_rn(p, r, 0x1.111112p-7f);                    // 1/120
+  p = __fmaf_rn(p, r, 0x1.555556p-5f);                    // 1/24
+  p = __fmaf_rn(p, r, 0x1.555556p-3f);                    // 1/6
+  p = __fmaf_rn(p, r, 0.5f);
+  p = __fmaf_rn(p, r, 1.0f);
+  p = __fmaf_rn(p, r, 1.0f);
+  const int n = static_cast<int>(nf);
+  // p * 2^(n+40): p is in [0.7, 1.42], n + 40 >= -3, so the exponent add cannot leave the normal range
+  const float scaled = __uint_as_float(__float_as_uint(p) + (static_cast<uint32_t>(n + 40) << 23));
+  return __float2ull_rz(scaled);
+}
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// block-wide sum, result to every thread; scratch holds 32 values
+__device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v, unsigned long long* scratch) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_sum_u64(v);
+  __syncthreads();
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  unsigned long long t = lane < (kThreads / 32) ? scratch[lane] : 0ull;
+  return warp_sum_u64(t);
+}
+
+struct Shared {
+  unsigned long long sum_scratch[32];
+  unsigned long long tile_sum[kMaxTiles];
+  unsigned long long warp_pref[32];
+  float max_scratch[32];
+  int idx_scratch[32];
+  int flag;
+  int decision;      // 1 accepted, 0 decide here
+  int pick;
+};
+
+__global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
+  __shared__ Shared sh;
+  const int req = blockIdx.x;
+  const int row0 = a.cu_q[req];
+  const int k = a.cu_q[req + 1] - row0 - 1;
+  const int V = a.V;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float* qbase = a.q_rows ? a.q_rows[req] : nullptr;
+  int32_t* res = a.results + 3 * req;
+
+  for (int j = 0; j <= k; ++j) {
+    const float* z = a.logits + static_cast<int64_t>(row0 + j) * V;
+    // ---- pass 1: maximum of the scaled logits (argmax of the raw ones when greedy), finiteness
+    float best = -INFINITY;
+    int best_i = 0x7fffffff;
+    int bad = 0;
+    for (int v = threadIdx.x; v < V; v += kThreads) {
+      const float x = z[v];
+      bad |= !(fabsf(x) < INFINITY);
+      const float sv = a.greedy ? x : __fmul_rn(x, a.inv_tau);
+      if (sv > best) { best = sv; best_i = v; }   // ascending v per thread: first maximum kept
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+      if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
+    }
+    bad = __syncthreads_or(bad);
+    if (lane == 0) { sh.max_scratch[warp] = best; sh.idx_scratch[warp] = best_i; }
+    __syncthreads();
+    if (bad) {
+      if (threadIdx.x == 0) { res[0] = 0; res[1] = -1; res[2] = ST_NONFINITE; }
+      return;
+    }
+    best = sh.max_scratch[0];
+    best_i = sh.idx_scratch[0];
+    for (int w = 1; w < kThreads / 32; ++w) {
+      const float ob = sh.max_scratch[w];
+      const int oi = sh.idx_scratch[w];
+      if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
+    }
+    if (a.greedy) {
+      if (j < k && a.ids[row0 + 1 + j] == best_i) continue;
+      if (threadIdx.x == 0) { res[0] = j; res[1] = best_i; res[2] = ST_OK; }
+      return;
+    }
+    const float m = best;
+    // ---- pass 2: Z = sum of the integer numerators
+    unsigned long long zsum = 0;
+    for (int v = threadIdx.x; v < V; v += kThreads) zsum += fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
+    const unsigned long long Z = block_sum_u64(zsum, sh.sum_scratch);
+    // ---- the accept test of draft j+1, or fall through on the bonus row
+    const float* qrow = nullptr;
+    uint32_t u_smp = 0;
+    if (threadIdx.x == 0) {
+      uint32_t w[4];
+      philox4x32_10(static_cast<uint32_t>(a.seed), static_cast<uint32_t>(a.seed >> 32), a.ctx_lo[req], a.ctx_hi[req],
+                    static_cast<uint32_t>(a.pos0[req] + j + 1), 0u, w);
+      int accepted = 0;
+      if (j < k) {
+        const int d = a.ids[row0 + 1 + j];
+        const unsigned long long Ed = fixed_exp(__fsub_rn(__fmul_rn(z[d], a.inv_tau), m));
+        const float qd = qbase[static_cast<int64_t>(j) * V + d];
+        const double lhs = __dmul_rn(__dmul_rn(static_cast<double>(w[0] >> 8), static_cast<double>(qd)),
+                                     __ull2double_rn(Z));
+        const double rhs = __dmul_rn(__ull2double_rn(Ed), 16777216.0);
+        accepted = lhs < rhs;
+      }
+      sh.decision = accepted;
+      sh.flag = static_cast<int>(w[1]);
+    }
+    __syncthreads();
+    if (sh.decision) continue;
+    u_smp = static_cast<uint32_t>(sh.flag);
+    if (j < k) qrow = qbase + static_cast<int64_t>(j) * V;
+
+    // ---- deciding row: weights R_v = max(E_v - trunc(q_v * Z), 0) (or E_v), tile sums in vocabulary order
+    const int n_tiles = (V + kTile - 1) / kTile;
+    const double Zd = __ull2double_rn(Z);
+    bool use_q = qrow != nullptr;
+    unsigned long long W = 0;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+      for (int tl = threadIdx.x; tl < n_tiles; tl += kThreads) sh.tile_sum[tl] = 0ull;
+      __syncthreads();
+      for (int tl = 0; tl < n_tiles; ++tl) {
+        unsigned long long mine = 0;
+        const int v0 = tl * kTile + threadIdx.x * kVec;
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) {
+          const int v = v0 + e;
+          if (v < V) {
+            unsigned long long E = fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
+            if (use_q) {
+              const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(qrow[v]), Zd));
+              E = E > Q ? E - Q : 0ull;
+            }
+            mine += E;
+          }
+        }
+        mine = warp_sum_u64(mine);
+        if (lane == 0 && mine) atomicAdd(&sh.tile_sum[tl], mine);  // integer adds: any order, same sum
+      }
+      __syncthreads();
+      W = 0;
+      for (int tl = 0; tl < n_tiles; ++tl) W += sh.tile_sum[tl];
+      if (W != 0 || !use_q) break;
+      use_q = false;   // residual mass zero (p <= q everywhere after rounding): draw from p itself
+      __syncthreads();
+    }
+    // ---- inverse CDF: tgt = (U' * W) >> 32, first v whose running sum exceeds tgt
+    const unsigned long long tgt = __umul64hi(W, static_cast<unsigned long long>(u_smp) << 32);
+    int tl_hit = 0;
+    unsigned long long before = 0;
+    for (int tl = 0; tl < n_tiles; ++tl) {
+      const unsigned long long nx = before + sh.tile_sum[tl];
+      if (nx > tgt) { tl_hit = tl; break; }
+      before = nx;
+      tl_hit = tl;  // only left at the last tile if nothing exceeded (cannot happen for W > 0)
+    }
+    unsigned long long r[kVec];
+    unsigned long long mine = 0;
+    {
+      const int v0 = tl_hit * kTile + threadIdx.x * kVec;
+#pragma unroll
+      for (int e = 0; e < kVec; ++e) {
+        const int v = v0 + e;
+        unsigned long long E = 0;
+        if (v < V) {
+          E = fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
+          if (use_q) {
+            const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(qrow[v]), Zd));
+            E = E > Q ? E - Q : 0ull;
+          }
+        }
+        r[e] = E;
+        mine += E;
+      }
+    }
+    // exclusive prefix of `mine` over the block in thread order
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    __syncthreads();
+    if (lane == 31) sh.warp_pref[warp] = incl;
+    if (threadIdx.x == 0) sh.pick = V - 1;
+    __syncthreads();
+    unsigned long long run = before + incl - mine;
+    for (int w = 0; w < warp; ++w) run += sh.warp_pref[w];
+    // exactly one thread sees the crossing
+    if (run <= tgt && run + mine > tgt) {
+      int pick = tl_hit * kTile + threadIdx.x * kVec;
+#pragma unroll
+      for (int e = 0; e < kVec; ++e) {
+        run += r[e];
+        if (run > tgt) { pick += e; break; }
+      }
+      sh.pick = pick;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) { res[0] = j; res[1] = sh.pick; res[2] = ST_OK; }
+    return;
+  }
+}
+
+}  // namespace
+
+int launch_accept(const AcceptArgs& a, cudaStream_t s) {
+  if (a.B <= 0) return 0;
+  if (a.V > kTile * kMaxTiles) return -1;
+  accept_kernel<<<a.B, kThreads, 0, s>>>(a);
+  return 1;
+}
+
+}  // namespace sled

@@ -1,0 +1,324 @@
+// bf16 linear layers on the 5th-generation tensor cores (sm_100a).
+//
+// One CTA computes a 128 (weight rows) x TN (tokens) tile over one K slice:
+//   warp 0   : TMA producer  - streams 64-wide K slabs of W and of the activations into a
+//              ring of shared-memory stages (128-byte swizzle), weights with an evict-first
+//              L2 policy (read once per step), activations evict-last (re-read by every tile)
+//   warp 1   : allocates tensor memory, issues tcgen05.mma (M=128, N=TN, K=16) x 4 per slab,
+//              commits each stage back to the producer and the finished tile to the epilogue
+//   warps 2-5: epilogue - tcgen05.ld the fp32 accumulators (lane = weight row, column = token)
+//              and store them transposed, 32 consecutive outputs of one token per warp store
+// The token extent of the MMA is a run-time field of the instruction descriptor, so a step
+// with T tokens pays for round_up(T, 16) columns, not for a fixed tile.
+// Every mbarrier wait is bounded: when it runs out the CTA records a code in *error, lets
+// copies in flight land, frees its tensor memory and returns.
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstdio>
+
+#include "gemm_tc.h"
+
+namespace sled {
+
+namespace {
+
+constexpr int kBlockM = 128;          // weight rows per tile (UMMA M)
+constexpr int kBlockK = 64;           // bf16 elements per K slab = one 128-byte swizzle row
+constexpr int kWStageBytes = kBlockM * kBlockK * 2;
+constexpr long long kWaitCycles = 200000000LL;  // ~0.1 s at 2 GHz
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait: false (and *error = code) when the phase did not complete in time
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* error, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (clock64() - t0 > kWaitCycles) {
+      atomicCAS(error, 0, code);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+
+// shared-memory operand descriptor: K-major tile of 128-byte rows, 128-byte swizzle,
+// 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffff) >> 4);   // start address / 16
+  d |= static_cast<uint64_t>(1) << 16;                      // leading byte offset (unused with swizzle)
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;              // stride byte offset between 8-row groups
+  d |= static_cast<uint64_t>(1) << 46;                      // descriptor version of this architecture
+  d |= static_cast<uint64_t>(2) << 61;                      // 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <int TN_MAX, int STAGES>
+struct SmemLayout {
+  static constexpr int kAStageBytes = TN_MAX * kBlockK * 2;
+  static constexpr int kStageBytes = kWStageBytes + kAStageBytes;
+  static constexpr int kTiles = STAGES * kStageBytes;
+  static constexpr int kTotal = kTiles + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+template <int TN_MAX, int STAGES>
+__global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CUtensorMap map_w,
+                                                       const __grid_constant__ CUtensorMap map_a, int T, int N,
+                                                       int kb_total, int kb_per_split, float* __restrict__ out,
+                                                       long long split_stride, int32_t* error) {
+  using L = SmemLayout<TN_MAX, STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t bars = base + L::kTiles;                 // full[STAGES], empty[STAGES], tmem_full, then the tmem address
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kTiles + 8 * (2 * STAGES + 1));
+  volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * (2 * STAGES + 1) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tile = blockIdx.x, t_tile = blockIdx.y, split = blockIdx.z;
+  const int kb0 = split * kb_per_split;
+  const int nkb = min(kb_per_split, kb_total - kb0);
+  const int t0 = t_tile * TN_MAX;
+  const int tn = min(TN_MAX, ((T - t0) + 15) & ~15);     // token columns of this tile, multiple of 16
+
+  if (threadIdx.x == 0) *abort_slot = *reinterpret_cast<volatile int32_t*>(error);
+  __syncthreads();
+  if (*abort_slot != 0) return;                           // an earlier CTA gave up: do not start
+
+  if (warp == 0 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    for (int s = 0; s < 2 * STAGES + 1; ++s) mbar_init(bars + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // tensor memory for the accumulator tile: TN_MAX fp32 columns x 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))),
+                 "r"(static_cast<uint32_t>(TN_MAX < 32 ? 32 : TN_MAX)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  bool ok = true;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint64_t pol_first, pol_last;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_last));
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(bars + 8 * (STAGES + s), ph ^ 1, error, 1)) { ok = false; break; }
+        const uint32_t full = bars + 8 * s;
+        mbar_expect_tx(full, L::kStageBytes);
+        const uint32_t wdst = base + s * L::kStageBytes;
+        tma_load_2d(wdst, &map_w, (kb0 + kb) * kBlockK, m_tile * kBlockM, full, pol_first);
+        tma_load_2d(wdst + kWStageBytes, &map_a, (kb0 + kb) * kBlockK, t0, full, pol_last);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = tn, M = 128
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(tn >> 3) << 17) |
+                             (static_cast<uint32_t>(kBlockM >> 4) << 24);
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(bars + 8 * s, ph, error, 2)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t wsrc = base + s * L::kStageBytes;
+        const uint64_t adesc = umma_desc(wsrc), bdesc = umma_desc(wsrc + kWStageBytes);
+#pragma unroll
+        for (int kk = 0; kk < kBlockK / 16; ++kk)   // 16 bf16 = 32 bytes further along K inside the swizzled row
+          umma_bf16(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+        umma_commit(bars + 8 * (STAGES + s));       // stage free once these MMAs have read it
+      }
+      if (ok) umma_commit(bars + 8 * (2 * STAGES)); // accumulator complete
+    }
+  } else {
+    const int quad = warp & 3;                      // a warp may only touch tensor-memory lanes 32*(warp%4)..+31
+    if (nkb > 0) ok = mbar_wait(bars + 8 * (2 * STAGES), 0, error, 3);
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    if (ok) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int n = m_tile * kBlockM + quad * 32 + lane;
+      float* dst = out + static_cast<long long>(split) * split_stride + n;
+      for (int c0 = 0; c0 < tn; c0 += 16) {
+        uint32_t v[16];
+        if (nkb > 0) {
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+              : "r"(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(c0)));
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = 0u;
+        }
+        if (n < N) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int t = t0 + c0 + i;
+            if (t < T) dst[static_cast<long long>(t) * N] = __uint_as_float(v[i]);
+          }
+        }
+      }
+    }
+  }
+
+  // teardown
+  if (!ok) *abort_slot = 1;
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    if (*abort_slot != 0) {
+      // something timed out: give copies and MMAs still in flight time to land before the memory goes away
+      const long long t1 = clock64();
+      while (clock64() - t1 < 2000000LL) __nanosleep(1000);
+    }
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(static_cast<uint32_t>(TN_MAX < 32 ? 32 : TN_MAX)) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+int make_map(CUtensorMap* map, const void* ptr, int rows, int K, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return -1;
+  if (K % 8 || (reinterpret_cast<uintptr_t>(ptr) & 15)) return -1;   // rows must stay 16-byte aligned; a K tail is zero-filled by TMA
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
+  cuuint32_t box[2] = {kBlockK, static_cast<cuuint32_t>(box_rows)};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    std::fprintf(stderr, "sled: cuTensorMapEncodeTiled failed (%d) rows=%d K=%d box=%d\n", static_cast<int>(r), rows, K, box_rows);
+    return -1;
+  }
+  return 0;
+}
+
+template <int TN_MAX, int STAGES>
+int launch_one(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K, int n_split, float* out,
+               int64_t split_stride, int32_t* error, cudaStream_t s) {
+  using L = SmemLayout<TN_MAX, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(tc_gemm_kernel<TN_MAX, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess)
+      return -1;
+    configured = true;
+  }
+  const int kb_total = (K + kBlockK - 1) / kBlockK;
+  const int kb_per = (kb_total + n_split - 1) / n_split;
+  dim3 grid((N + kBlockM - 1) / kBlockM, (T + TN_MAX - 1) / TN_MAX, n_split);
+  tc_gemm_kernel<TN_MAX, STAGES><<<grid, 192, L::kTotal, s>>>(mw, ma, T, N, kb_total, kb_per, out, split_stride, error);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int tile_tokens(int T) { return T <= 64 ? 64 : (T <= 128 ? 128 : 256); }
+
+}  // namespace
+
+int tc_weight_init(TcWeight* w, const void* dev_ptr, int N, int K) {
+  if (make_map(&w->map, dev_ptr, N, K, kBlockM)) return -1;
+  w->N = N;
+  w->K = K;
+  w->ready = true;
+  return 0;
+}
+
+void tc_weight_free(TcWeight* w) { w->ready = false; }
+
+int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K) {
+  if (rows % 256) return -1;
+  const int boxes[3] = {64, 128, 256};
+  for (int i = 0; i < 3; ++i)
+    if (make_map(&a->map[i], dev_ptr, rows, K, boxes[i])) return -1;
+  a->rows = rows;
+  a->K = K;
+  return 0;
+}
+
+int tc_gemm_split(int T, int N, int K, int n_sm) {
+  const int tn = tile_tokens(T);
+  const int tiles = ((N + kBlockM - 1) / kBlockM) * ((T + tn - 1) / tn);
+  const int kb_total = (K + kBlockK - 1) / kBlockK;
+  const int target = 2 * n_sm;                 // two CTAs fit on an SM
+  int s = 1;
+  if (tiles * 5 < target * 3) s = (target + tiles - 1) / tiles;
+  s = std::min(s, std::max(1, kb_total / 4));  // at least 4 slabs per slice
+  s = std::max(1, std::min(s, 16));
+  const int kb_per = (kb_total + s - 1) / s;
+  return (kb_total + kb_per - 1) / kb_per;     // slices that actually get work
+}
+
+int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
+                   int32_t* error, int n_sm, cudaStream_t s) {
+  (void)n_sm;
+  if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
+  const int tn = tile_tokens(T);
+  if (tn == 64) return launch_one<64, 4>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, s);
+  if (tn == 128) return launch_one<128, 3>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, s);
+  return launch_one<256, 2>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, s);
+}
+
+}  // namespace sled

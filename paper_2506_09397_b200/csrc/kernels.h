@@ -1,0 +1,73 @@
+// Host-callable launchers of the device kernels.  Every launcher only enqueues work on
+// the given stream and returns the number of kernels it launched (negative: bad argument).
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace sled {
+
+enum DType { F32 = 0, BF16 = 1 };
+
+// ---- elementwise / small kernels (kernels_small.cu)
+int launch_embed(const void* table, int wdtype, const int32_t* ids, int T, int d, float* x, cudaStream_t s);
+// x += sum_s partial[s] (if partial), then out = RMSNorm(x) * gain in the activation type
+int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t split_stride, const void* gain, int wdtype,
+                       float eps, int T, int d, void* out, int adtype, cudaStream_t s);
+int launch_rope_table(const int32_t* tok_pos, int T, int h, float theta, float2* cs, cudaStream_t s);
+// sums the QKV partials, rotates Q and K, writes Q to q_out and K, V into their cache slots
+int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, const float2* cs, const int32_t* tok_slot,
+                   int T, int Hq, int Hkv, int h, int page_size, void* q_out, int adtype, void* kpool, void* vpool,
+                   int kvdtype, cudaStream_t s);
+int launch_swiglu(const float* partial, int n_split, int64_t split_stride, int T, int F, void* out, int adtype,
+                  cudaStream_t s);
+// contiguous [n][Hkv][h] <-> paged cache of one layer
+int launch_kv_scatter(const void* src, const int32_t* slots, int n, int Hkv, int h, int page_size, void* pool,
+                      int kvdtype, cudaStream_t s);
+int launch_kv_gather(const void* pool, const int32_t* slots, int n, int Hkv, int h, int page_size, void* dst,
+                     int kvdtype, cudaStream_t s);
+
+// ---- fp32 / generic CUDA-core GEMM (kernels_small.cu): out[s][T][N] = A[T][Kslice_s] . W[N][Kslice_s]^T
+int launch_gemm_simt(const void* A, int adtype, const void* W, int wdtype, int T, int N, int K, int n_split,
+                     float* out, int64_t split_stride, cudaStream_t s);
+
+// ---- ragged verification attention over the paged cache (attention.cu)
+struct AttnArgs {
+  const int4* items;  // {request, kv head, first key, key count}
+  int n_items;
+  const void* q;      // [T][Hq][h] activation type
+  void* out;          // [T][Hq][h] activation type
+  const void* kpool;  // one layer: [page][Hkv][page_size][h]
+  const void* vpool;
+  const int32_t* cu_q;       // [B+1]
+  const int32_t* kv_base;    // [B] cached tokens before the step: query j sees keys 0 .. kv_base + j
+  const int32_t* page_table; // flat
+  const int32_t* pt_off;     // [B+1]
+  const int32_t* tok_req;    // [T]
+  const int32_t* tok_part;   // [T] first partial-result row of a token (tokens of split requests only)
+  const int32_t* req_chunks; // [B] number of key chunks of a request
+  float* part_acc;           // [rows][Hq][h]
+  float* part_ml;            // [rows][Hq][2]
+  int T, Hq, Hkv, h, page_size, chunk_keys;
+  int adtype, kvdtype;
+};
+int launch_attention(const AttnArgs& a, cudaStream_t s);
+
+// ---- fused vocabulary softmax + acceptance + corrective / bonus draw (accept.cu)
+struct AcceptArgs {
+  const float* logits;        // [rows][V]
+  const int32_t* cu_q;        // [B+1] first row of each request
+  const int32_t* ids;         // [rows] fed tokens: drafts of request i are ids[cu_q[i]+1 ..]
+  const float* const* q_rows; // [B] device pointer to the request's [k][V] draft distributions (may hold null)
+  const uint32_t* ctx_lo;     // [B]
+  const uint32_t* ctx_hi;     // [B]
+  const int32_t* pos0;        // [B] absolute index of the pending token
+  int32_t* results;           // [B][3] n_accepted, next_token, status
+  int B, V;
+  float inv_tau;
+  int greedy;
+  uint64_t seed;
+};
+int launch_accept(const AcceptArgs& a, cudaStream_t s);
+
+}  // namespace sled

@@ -1,0 +1,279 @@
+// Small kernels of the verification step: token embedding, residual-add + RMSNorm,
+// rotary embedding with the write of new keys/values into their cache pages, SwiGLU,
+// cache scatter/gather, and the CUDA-core GEMM used by the fp32 configuration.
+// The linear layers leave split-K partial sums behind; the kernel that consumes a
+// linear layer's output adds them up, in a fixed order, while it does its own work.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace sled {
+
+// ------------------------------------------------------------------ embedding --
+template <typename WT>
+__global__ void embed_kernel(const WT* __restrict__ table, const int32_t* __restrict__ ids, int d, float* __restrict__ x) {
+  const int t = blockIdx.x;
+  const WT* row = table + static_cast<int64_t>(ids[t]) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) x[static_cast<int64_t>(t) * d + i] = to_f32(row[i]);
+}
+
+int launch_embed(const void* table, int wdtype, const int32_t* ids, int T, int d, float* x, cudaStream_t s) {
+  if (T <= 0) return 0;
+  if (wdtype == BF16)
+    embed_kernel<<<T, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(table), ids, d, x);
+  else
+    embed_kernel<<<T, 256, 0, s>>>(static_cast<const float*>(table), ids, d, x);
+  return 1;
+}
+
+// ------------------------------------------------------- residual add + RMSNorm --
+// One block per token.  x (fp32 residual stream) is updated in place with the split-K
+// partial sums of the preceding linear layer, then normalised:
+//   y_i = x_i * rsqrt(mean(x^2) + eps) * g_i
+template <typename WT, typename AT>
+__global__ void add_rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ partial, int n_split,
+                                   int64_t split_stride, const WT* __restrict__ gain, float eps, int d,
+                                   AT* __restrict__ out) {
+  __shared__ float scratch[32];
+  const int64_t base = static_cast<int64_t>(blockIdx.x) * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    float v = x[base + i];
+    for (int sp = 0; sp < n_split; ++sp) v += partial[sp * split_stride + base + i];
+    if (n_split > 0) x[base + i] = v;
+    ss += v * v;
+  }
+  ss = block_sum(ss, scratch);
+  const float scale = rsqrtf(ss / static_cast<float>(d) + eps);
+  for (int i = threadIdx.x; i < d; i += blockDim.x)  // each thread re-reads what it wrote itself
+    out[base + i] = from_f32<AT>(x[base + i] * scale * to_f32(gain[i]));
+}
+
+int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t split_stride, const void* gain, int wdtype,
+                       float eps, int T, int d, void* out, int adtype, cudaStream_t s) {
+  if (T <= 0) return 0;
+  if (!partial) n_split = 0;
+  const int nt = d >= 2048 ? 512 : 256;
+  if (wdtype == BF16 && adtype == BF16)
+    add_rmsnorm_kernel<<<T, nt, 0, s>>>(x, partial, n_split, split_stride, static_cast<const __nv_bfloat16*>(gain), eps,
+                                        d, static_cast<__nv_bfloat16*>(out));
+  else if (wdtype == F32 && adtype == F32)
+    add_rmsnorm_kernel<<<T, nt, 0, s>>>(x, partial, n_split, split_stride, static_cast<const float*>(gain), eps, d,
+                                        static_cast<float*>(out));
+  else
+    return -1;
+  return 1;
+}
+
+// --------------------------------------------------------------- rotary table --
+// cs[t][i] = (cos, sin)(pos_t * theta^(-2i/h)), angle and functions in fp64, stored fp32;
+// computed once per step and shared by all layers and heads.
+__global__ void rope_table_kernel(const int32_t* __restrict__ tok_pos, int h, double log2_theta, float2* __restrict__ cs) {
+  const int t = blockIdx.x, i = threadIdx.x;
+  if (i >= h / 2) return;
+  const double inv_freq = exp2(-2.0 * static_cast<double>(i) / static_cast<double>(h) * log2_theta);
+  double sn, c;
+  sincos(static_cast<double>(tok_pos[t]) * inv_freq, &sn, &c);
+  cs[static_cast<int64_t>(t) * (h / 2) + i] = make_float2(static_cast<float>(c), static_cast<float>(sn));
+}
+
+int launch_rope_table(const int32_t* tok_pos, int T, int h, float theta, float2* cs, cudaStream_t s) {
+  if (T <= 0) return 0;
+  rope_table_kernel<<<T, h / 2, 0, s>>>(tok_pos, h, log2(static_cast<double>(theta)), cs);
+  return 1;
+}
+
+// ------------------------------------------------------ RoPE + cache write --
+// grid (T, Hq + 2 Hkv), h/2 threads: thread i owns the pair (2i, 2i+1) of one head.
+// Cache layout of one layer: [page][Hkv][page_size][h]; slot = page * page_size + offset.
+template <typename AT, typename KT>
+__global__ void rope_kv_kernel(const float* __restrict__ partial, int n_split, int64_t split_stride,
+                               const float2* __restrict__ cs, const int32_t* __restrict__ tok_slot, int Hq, int Hkv,
+                               int h, int page_size, AT* __restrict__ q_out, KT* __restrict__ kpool,
+                               KT* __restrict__ vpool) {
+  const int t = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
+  const int n_cols = (Hq + 2 * Hkv) * h;
+  const int64_t src = static_cast<int64_t>(t) * n_cols + head * h + 2 * i;
+  float a = 0.f, b = 0.f;
+  for (int sp = 0; sp < n_split; ++sp) {
+    const float2 v = *reinterpret_cast<const float2*>(partial + sp * split_stride + src);
+    a += v.x;
+    b += v.y;
+  }
+  if (head < Hq + Hkv) {
+    const float2 c = cs[static_cast<int64_t>(t) * (h / 2) + i];
+    const float ra = a * c.x - b * c.y, rb = a * c.y + b * c.x;
+    a = ra;
+    b = rb;
+  }
+  if (head < Hq) {
+    AT* dst = q_out + (static_cast<int64_t>(t) * Hq + head) * h + 2 * i;
+    dst[0] = from_f32<AT>(a);
+    dst[1] = from_f32<AT>(b);
+  } else {
+    const bool is_k = head < Hq + Hkv;
+    const int kvh = is_k ? head - Hq : head - Hq - Hkv;
+    const int slot = tok_slot[t];
+    const int64_t off = ((static_cast<int64_t>(slot / page_size) * Hkv + kvh) * page_size + slot % page_size) * h + 2 * i;
+    KT* dst = (is_k ? kpool : vpool) + off;
+    dst[0] = from_f32<KT>(a);
+    dst[1] = from_f32<KT>(b);
+  }
+}
+
+int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, const float2* cs, const int32_t* tok_slot,
+                   int T, int Hq, int Hkv, int h, int page_size, void* q_out, int adtype, void* kpool, void* vpool,
+                   int kvdtype, cudaStream_t s) {
+  if (T <= 0) return 0;
+  dim3 grid(T, Hq + 2 * Hkv);
+  if (adtype == BF16 && kvdtype == BF16)
+    rope_kv_kernel<<<grid, h / 2, 0, s>>>(partial, n_split, split_stride, cs, tok_slot, Hq, Hkv, h, page_size,
+                                          static_cast<__nv_bfloat16*>(q_out), static_cast<__nv_bfloat16*>(kpool),
+                                          static_cast<__nv_bfloat16*>(vpool));
+  else if (adtype == F32 && kvdtype == F32)
+    rope_kv_kernel<<<grid, h / 2, 0, s>>>(partial, n_split, split_stride, cs, tok_slot, Hq, Hkv, h, page_size,
+                                          static_cast<float*>(q_out), static_cast<float*>(kpool),
+                                          static_cast<float*>(vpool));
+  else if (adtype == F32 && kvdtype == BF16)
+    rope_kv_kernel<<<grid, h / 2, 0, s>>>(partial, n_split, split_stride, cs, tok_slot, Hq, Hkv, h, page_size,
+                                          static_cast<float*>(q_out), static_cast<__nv_bfloat16*>(kpool),
+                                          static_cast<__nv_bfloat16*>(vpool));
+  else
+    return -1;
+  return 1;
+}
+
+// --------------------------------------------------------------------- SwiGLU --
+// partial: [split][T][2F], gate in columns [0, F), up in [F, 2F):  out = silu(gate) * up
+template <typename AT>
+__global__ void swiglu_kernel(const float* __restrict__ partial, int n_split, int64_t split_stride, int F,
+                              AT* __restrict__ out) {
+  const int t = blockIdx.y;
+  const int f = blockIdx.x * blockDim.x + threadIdx.x;
+  if (f >= F) return;
+  const int64_t row = static_cast<int64_t>(t) * 2 * F;
+  float g = 0.f, u = 0.f;
+  for (int sp = 0; sp < n_split; ++sp) {
+    g += partial[sp * split_stride + row + f];
+    u += partial[sp * split_stride + row + F + f];
+  }
+  out[static_cast<int64_t>(t) * F + f] = from_f32<AT>(g / (1.f + __expf(-g)) * u);
+}
+
+int launch_swiglu(const float* partial, int n_split, int64_t split_stride, int T, int F, void* out, int adtype,
+                  cudaStream_t s) {
+  if (T <= 0) return 0;
+  dim3 grid((F + 255) / 256, T);
+  if (adtype == BF16)
+    swiglu_kernel<<<grid, 256, 0, s>>>(partial, n_split, split_stride, F, static_cast<__nv_bfloat16*>(out));
+  else
+    swiglu_kernel<<<grid, 256, 0, s>>>(partial, n_split, split_stride, F, static_cast<float*>(out));
+  return 1;
+}
+
+// -------------------------------------------------- cache scatter / gather --
+template <typename KT, bool TO_POOL>
+__global__ void kv_move_kernel(KT* __restrict__ pool, KT* __restrict__ flat, const int32_t* __restrict__ slots, int Hkv,
+                               int h, int page_size) {
+  const int n = blockIdx.x, kvh = blockIdx.y;
+  const int slot = slots[n];
+  const int64_t po = ((static_cast<int64_t>(slot / page_size) * Hkv + kvh) * page_size + slot % page_size) * h;
+  const int64_t fo = (static_cast<int64_t>(n) * Hkv + kvh) * h;
+  for (int i = threadIdx.x; i < h; i += blockDim.x) {
+    if (TO_POOL) pool[po + i] = flat[fo + i];
+    else flat[fo + i] = pool[po + i];
+  }
+}
+
+int launch_kv_scatter(const void* src, const int32_t* slots, int n, int Hkv, int h, int page_size, void* pool,
+                      int kvdtype, cudaStream_t s) {
+  if (n <= 0) return 0;
+  dim3 grid(n, Hkv);
+  if (kvdtype == BF16)
+    kv_move_kernel<__nv_bfloat16, true><<<grid, 64, 0, s>>>(static_cast<__nv_bfloat16*>(pool),
+        const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(src)), slots, Hkv, h, page_size);
+  else
+    kv_move_kernel<float, true><<<grid, 64, 0, s>>>(static_cast<float*>(pool),
+        const_cast<float*>(static_cast<const float*>(src)), slots, Hkv, h, page_size);
+  return 1;
+}
+
+int launch_kv_gather(const void* pool, const int32_t* slots, int n, int Hkv, int h, int page_size, void* dst,
+                     int kvdtype, cudaStream_t s) {
+  if (n <= 0) return 0;
+  dim3 grid(n, Hkv);
+  if (kvdtype == BF16)
+    kv_move_kernel<__nv_bfloat16, false><<<grid, 64, 0, s>>>(
+        const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(pool)), static_cast<__nv_bfloat16*>(dst), slots,
+        Hkv, h, page_size);
+  else
+    kv_move_kernel<float, false><<<grid, 64, 0, s>>>(const_cast<float*>(static_cast<const float*>(pool)),
+                                                     static_cast<float*>(dst), slots, Hkv, h, page_size);
+  return 1;
+}
+
+// ------------------------------------------------------------ CUDA-core GEMM --
+// out[z][t][n] = sum over the z-th K slice of A[t][k] * W[n][k], fp32 accumulation.
+// 32 x 64 output tile per block of 256 threads (2 x 4 outputs per thread), K step 32.
+template <typename AT, typename WT>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const AT* __restrict__ A, const WT* __restrict__ W, int T, int N,
+                                                        int K, int k_per_split, float* __restrict__ out,
+                                                        int64_t split_stride) {
+  constexpr int BM = 32, BN = 64, BK = 32;
+  __shared__ float As[BK][BM + 1];
+  __shared__ float Ws[BK][BN + 1];
+  const int t0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int k_begin = blockIdx.z * k_per_split, k_end = min(K, k_begin + k_per_split);
+  const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;  // tx -> 4 columns, ty -> 2 rows
+  float acc[2][4] = {};
+  for (int k0 = k_begin; k0 < k_end; k0 += BK) {
+    for (int e = threadIdx.x; e < BM * BK; e += 256) {
+      const int m = e / BK, kk = e % BK;
+      const int t = t0 + m, k = k0 + kk;
+      As[kk][m] = (t < T && k < k_end) ? to_f32(A[static_cast<int64_t>(t) * K + k]) : 0.f;
+    }
+    for (int e = threadIdx.x; e < BN * BK; e += 256) {
+      const int n = e / BK, kk = e % BK;
+      const int nn = n0 + n, k = k0 + kk;
+      Ws[kk][n] = (nn < N && k < k_end) ? to_f32(W[static_cast<int64_t>(nn) * K + k]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a[2], w[4];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) a[i] = As[kk][ty * 2 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) w[j] = Ws[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], w[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  float* o = out + blockIdx.z * split_stride;
+  for (int i = 0; i < 2; ++i)
+    for (int j = 0; j < 4; ++j) {
+      const int t = t0 + ty * 2 + i, n = n0 + tx * 4 + j;
+      if (t < T && n < N) o[static_cast<int64_t>(t) * N + n] = acc[i][j];
+    }
+}
+
+int launch_gemm_simt(const void* A, int adtype, const void* W, int wdtype, int T, int N, int K, int n_split,
+                     float* out, int64_t split_stride, cudaStream_t s) {
+  if (T <= 0) return 0;
+  if (n_split < 1) n_split = 1;
+  int k_per_split = ((K + n_split - 1) / n_split + 31) / 32 * 32;
+  dim3 grid((N + 63) / 64, (T + 31) / 32, n_split);
+  if (adtype == F32 && wdtype == F32)
+    gemm_simt_kernel<<<grid, 256, 0, s>>>(static_cast<const float*>(A), static_cast<const float*>(W), T, N, K,
+                                          k_per_split, out, split_stride);
+  else if (adtype == BF16 && wdtype == BF16)
+    gemm_simt_kernel<<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(A), static_cast<const __nv_bfloat16*>(W), T,
+                                          N, K, k_per_split, out, split_stride);
+  else
+    return -1;
+  return 1;
+}
+
+}  // namespace sled

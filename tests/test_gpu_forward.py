@@ -1,0 +1,193 @@
+"""Whole verification step on the GPU vs the oracle: logits within tolerance, decisions equal
+(or explained by a deciding margin below the tolerance), cache commit / rollback."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2506_09397_b200 import binding as B
+from paper_2506_09397_b200 import inputs as I
+from util import oracle_weights, rel_margin_ok
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"fp32": 1e-4, "bf16": 2e-2}   # max |logit difference| allowed per weight type
+
+
+def _engine(shape, w, **kw):
+    args = dict(n_pages=256, max_batch=16, max_k=8, max_step_tokens=160)
+    args.update(kw)
+    return B.Engine(shape, w, **args)
+
+
+def _verify_both(eng, orc, reqs, seed, tau, greedy, tol, explain):
+    """reqs: list of (ctx, drafts tensor, q tensor).  Runs one step on both sides and compares."""
+    got = eng.verify_batch([(c, d.numpy(), None if greedy else q.numpy()) for c, d, q in reqs], seed)
+    T = sum(len(d) + 1 for _, d, _ in reqs)
+    glog = eng.logits(T)
+    row = 0
+    for (c, d, q), g in zip(reqs, got):
+        k = len(d)
+        pos0 = orc.ctx[c].n_kv
+        st, n_acc, nxt, ologits, mg = orc.verify(c, d.numpy(), None if greedy else q.numpy(), seed, tau, greedy, commit=False)
+        mine = glog[row:row + k + 1]
+        row += k + 1
+        assert np.max(np.abs(mine - ologits)) <= tol, (c, float(np.max(np.abs(mine - ologits))))
+        # bit-exact given identical logits: the oracle's rule on the GPU's logits
+        st2, n2, x2, _ = O.accept(mine, None if greedy or k == 0 else q.numpy(), d.numpy(), tau, greedy, seed, c, pos0)
+        assert (n2, x2) == g[:2] and g[2] == 0
+        if (n_acc, nxt) != g[:2]:
+            assert rel_margin_ok(mg, tol), (c, (n_acc, nxt), g, mg.accept_rel, mg.sample_rel, mg.greedy_gap)
+            explain.append(c)
+        # the oracle follows the GPU's decision so that both sides keep the same history
+        oc = orc.ctx[c]
+        oc.n_kv += g[0] + 1
+        oc.tokens += [int(x) for x in d[:g[0]]] + [g[1]]
+        oc.pending = g[1]
+    return got
+
+
+@pytest.mark.parametrize("shape_name", ["tiny", "tiny_bf16", "small_gqa"])
+def test_prefilled_contexts_multi_step(shape_name):
+    shape = I.SHAPES[shape_name]
+    tol = TOL[shape.weight_dtype]
+    w = I.make_weights(shape, seed=0)
+    eng = _engine(shape, w)
+    orc = O.OracleModel(shape, oracle_weights(w))
+    ctxs = [11, 12, 13, 14]
+    lens = [64, 64, 64, 64] if shape_name == "tiny" else [33, 5, 64, 18]
+    for c, n in zip(ctxs, lens):
+        p = I.make_prompt(shape.vocab, n, 0, c)
+        eng.prefill(c, p)
+        orc.prefill(c, p)
+    # cache written by the prefill: on the format's grid and close to the oracle's
+    K, V = eng.read_kv(ctxs[0], shape.n_layers - 1, lens[0] - 1)
+    ok = orc.ctx[ctxs[0]].K[shape.n_layers - 1, :lens[0] - 1]
+    assert np.max(np.abs(K.float().numpy() - ok)) <= (2e-2 if shape.kv_dtype == "bf16" else 1e-5)
+    explain = []
+    for step in range(4):
+        ks = [4, 4, 4, 4] if (shape_name == "tiny" and step == 0) else I.draw_k(4, [0, 1, 3, 5, 8], seed=step)
+        reqs = []
+        for c, k in zip(ctxs, ks):
+            d, q = I.make_drafts(shape.vocab, k, 0, c, step)
+            reqs.append((c, d, q))
+        greedy = step == 3
+        eng.set_sampling(1.0 if step < 2 else 0.8, greedy)
+        _verify_both(eng, orc, reqs, seed=step, tau=1.0 if step < 2 else 0.8, greedy=greedy, tol=tol, explain=explain)
+        for c in ctxs:   # commit / rollback bookkeeping agrees
+            n_kv, pending, pages = eng.query_ctx(c)
+            assert (n_kv, pending) == (orc.ctx[c].n_kv, orc.ctx[c].pending)
+            assert len(pages) == (n_kv + 15) // 16
+    assert len(explain) <= 1
+    st = eng.stats()
+    assert st.steps == 4 and st.kernels_last_step > 0 and st.tokens_committed > 0
+    for c in ctxs:
+        eng.release(c)
+    assert eng.stats().pages_free == 256
+    eng.shutdown()
+
+
+def test_greedy_accepts_its_own_continuation():
+    # generate with k = 0 steps, then verify that continuation as drafts: all accepted + bonus
+    shape = I.TINY
+    w = I.make_weights(shape, seed=0)
+    eng = _engine(shape, w, greedy=True)
+    p = I.make_prompt(shape.vocab, 20, 0, 1)
+    eng.prefill(1, p)
+    gen = []
+    for _ in range(7):
+        (n_acc, nxt, st), = eng.verify_batch([(1, [], None)], 0)
+        assert (n_acc, st) == (0, 0)
+        gen.append(nxt)
+    eng.prefill(2, p)
+    (n_acc, nxt, st), = eng.verify_batch([(2, gen[:6], None)], 0)
+    assert (n_acc, nxt) == (6, gen[6])
+    eng.prefill(3, p)
+    bad = list(gen[:6])
+    bad[2] = (bad[2] + 1) % shape.vocab
+    (n_acc, nxt, st), = eng.verify_batch([(3, bad, None)], 0)
+    assert (n_acc, nxt) == (2, gen[2])
+    assert eng.query_ctx(3)[0] == 19 + 3
+    eng.shutdown()
+
+
+def test_batch_composition_does_not_change_a_request():
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=1)
+    eng = _engine(shape, w)
+    eng.set_commit(False)
+    for c, n in [(1, 40), (2, 9), (3, 70)]:
+        eng.prefill(c, I.make_prompt(shape.vocab, n, 1, c))
+    reqs = {c: I.make_drafts(shape.vocab, k, 1, c) for c, k in [(1, 5), (2, 8), (3, 2)]}
+    alone = {}
+    for c, (d, q) in reqs.items():
+        alone[c] = (eng.verify_batch([(c, d.numpy(), q.numpy())], 7)[0], eng.logits(len(d) + 1))
+    order = [3, 1, 2]
+    got = eng.verify_batch([(c, reqs[c][0].numpy(), reqs[c][1].numpy()) for c in order], 7)
+    lg = eng.logits(sum(len(reqs[c][0]) + 1 for c in order))
+    row = 0
+    for c, g in zip(order, got):
+        k = len(reqs[c][0])
+        assert np.max(np.abs(lg[row:row + k + 1] - alone[c][1])) <= 2e-3   # same math, different tile shapes
+        row += k + 1
+        assert g == alone[c][0]
+    eng.shutdown()
+
+
+def test_synthetic_cache_and_long_context_split():
+    # cache content loaded directly; one context long enough that its keys are split over several blocks
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=2)
+    eng = _engine(shape, w, n_pages=400)
+    eng.shuffle_pages(5)
+    orc = O.OracleModel(shape, oracle_weights(w))
+    lens = {21: 1500, 22: 300, 23: 17}
+    for c, n in lens.items():
+        K, V = I.make_kv(shape, n, 2, c)
+        K, V = K * 0.3, V * 0.3
+        eng.load_kv(c, K.contiguous(), V.contiguous(), pending=5)
+        orc.load_kv(c, K.float().numpy(), V.float().numpy(), pending=5)
+        Kb, Vb = eng.read_kv(c, 1, n)
+        assert torch.equal(Kb, K[1]) and torch.equal(Vb, V[1])   # paged gather == the contiguous cache
+    reqs = []
+    for c, k in zip(lens, [8, 3, 6]):
+        d, q = I.make_drafts(shape.vocab, k, 2, c)
+        reqs.append((c, d, q))
+    explain = []
+    _verify_both(eng, orc, reqs, seed=3, tau=1.0, greedy=False, tol=2e-2, explain=explain)
+    assert not explain
+    eng.shutdown()
+
+
+def test_errors_leave_everything_unchanged():
+    shape = I.TINY
+    w = I.make_weights(shape, seed=0)
+    eng = _engine(shape, w, n_pages=8, max_batch=2, max_k=4, max_step_tokens=10)
+    eng.prefill(1, I.make_prompt(shape.vocab, 30, 0, 1))
+    eng.prefill(2, I.make_prompt(shape.vocab, 30, 0, 2))
+    before = (eng.query_ctx(1), eng.query_ctx(2), eng.stats().pages_free)
+    d, q = I.make_drafts(shape.vocab, 4, 0, 1)
+
+    def code(reqs):
+        with pytest.raises(B.SledError) as ei:
+            eng.verify_batch(reqs, 0)
+        return ei.value.code
+
+    assert code([(9, d.numpy(), q.numpy())]) == B.SLED_ERR_UNKNOWN_CTX
+    assert code([(1, d.numpy(), q.numpy()), (1, d.numpy(), q.numpy())]) == B.SLED_ERR_DUP_CTX
+    assert code([(1, np.arange(5), np.zeros((5, shape.vocab), np.float32))]) == B.SLED_ERR_K_RANGE
+    assert code([(1, np.array([shape.vocab]), q.numpy()[:1])]) == B.SLED_ERR_TOKEN_RANGE
+    assert code([(1, d.numpy(), None)]) == B.SLED_ERR_ARG
+    assert code([(1, d.numpy(), q.numpy())] * 3) == B.SLED_ERR_BATCH_TOO_LARGE
+    with pytest.raises(B.SledError) as ei:
+        eng.prefill(3, I.make_prompt(shape.vocab, 16 * 8, 0, 3))
+    assert ei.value.code == B.SLED_ERR_NO_PAGES
+    with pytest.raises(B.SledError) as ei:
+        eng.prefill(1, [1, 2])
+    assert ei.value.code == B.SLED_ERR_DUP_CTX
+    after = (eng.query_ctx(1), eng.query_ctx(2), eng.stats().pages_free)
+    assert str(before) == str(after)
+    eng.release(1)
+    with pytest.raises(B.SledError):
+        eng.verify_batch([(1, d.numpy(), q.numpy())], 0)
+    eng.shutdown()

@@ -1,0 +1,127 @@
+"""Host-side logic of the CUDA library that needs no device: exported symbols, the page manager's
+invariants under random verify / release sequences, ragged packing, and error returns."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2506_09397_b200 import binding as B
+from paper_2506_09397_b200 import build as builder
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    builder.build()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "sled.h")).read()
+    declared = set(re.findall(r"^(?:int|void|void\*|const char\*|int32_t|sled_kvm\*)\s+(sled_[a-z_0-9]+)\(", header, re.M))
+    assert len(declared) > 20
+    assert declared == set(B.EXPORTS)
+    raw = C.CDLL(B.LIB_PATH)
+    for name in declared:
+        assert hasattr(raw, name), name
+
+
+def test_strerror_and_null_arguments():
+    L = B.lib()
+    assert B.strerror(0) == "ok"
+    assert "fallback" in B.strerror(B.SLED_ERR_NO_DEVICE)
+    assert L.sled_init(None, None, None) == B.SLED_ERR_ARG
+    assert L.sled_verify_batch(None, None, 0, 0, None) == B.SLED_ERR_ARG
+    assert L.sled_release(None, 0) == B.SLED_ERR_ARG
+
+
+def test_init_without_a_device_fails_loudly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    from paper_2506_09397_b200 import inputs as I
+    w = I.make_weights(I.TINY, 0)
+    with pytest.raises(B.SledError) as ei:
+        B.Engine(I.TINY, w, n_pages=64, max_batch=4, max_k=4, max_step_tokens=32)
+    assert ei.value.code == B.SLED_ERR_NO_DEVICE
+
+
+def _check_invariants(m, live, n_pages, ps):
+    owned = []
+    for ctx, (n_kv, pending) in live.items():
+        rc, q = m.query(ctx)
+        assert rc == 0
+        assert q[0] == n_kv and q[1] == pending
+        assert len(q[2]) == (n_kv + ps - 1) // ps          # exactly the pages its tokens need
+        owned += list(q[2])
+    assert len(owned) == len(set(owned))                     # no page owned twice
+    assert all(0 <= p < n_pages for p in owned)
+    assert len(owned) + m.free_pages() == n_pages            # free + owned = pool
+
+
+def test_page_manager_random_walk():
+    rng = np.random.default_rng(0)
+    n_pages, ps = 40, 16
+    m = B.KvManager(n_pages, ps)
+    live = {}
+    nxt = 1
+    for step in range(3000):
+        op = rng.integers(0, 10)
+        if op < 2 and len(live) < 8:
+            n_kv = int(rng.integers(0, 70))
+            rc = m.open(nxt, n_kv, 7)
+            need = (n_kv + ps - 1) // ps
+            if rc == 0:
+                live[nxt] = (n_kv, 7)
+            else:
+                assert rc == B.SLED_ERR_NO_PAGES and need > m.free_pages()
+            nxt += 1
+        elif op < 8 and live:
+            ids = list(rng.choice(list(live), size=min(len(live), int(rng.integers(1, 5))), replace=False))
+            ks = [int(rng.integers(0, 9)) for _ in ids]
+            free_before = m.free_pages()
+            rc = m.reserve_batch(ids, [k + 1 for k in ks])
+            if rc != 0:
+                assert rc == B.SLED_ERR_NO_PAGES and m.free_pages() == free_before
+                _check_invariants(m, live, n_pages, ps)       # a failed reservation changed nothing
+                continue
+            rc, cu, (tok, req, pos, slot) = m.pack(ids, ks, [np.arange(k) + 100 for k in ks])
+            assert rc == 0 and cu[-1] == sum(k + 1 for k in ks)
+            for i, ctx in enumerate(ids):
+                n_kv, pending = live[ctx]
+                rows = slice(cu[i], cu[i + 1])
+                assert tok[rows][0] == pending and list(tok[rows][1:]) == list(np.arange(ks[i]) + 100)
+                assert list(pos[rows]) == list(range(n_kv, n_kv + ks[i] + 1))
+                assert all(req[rows] == i)
+                pages = m.query(ctx)[1][2]
+                assert list(slot[rows]) == [pages[p // ps] * ps + p % ps for p in range(n_kv, n_kv + ks[i] + 1)]
+            for ctx, k in zip(ids, ks):
+                n_acc = int(rng.integers(0, k + 1))
+                assert m.commit(ctx, n_acc + 1, 50 + n_acc) == 0
+                live[ctx] = (live[ctx][0] + n_acc + 1, 50 + n_acc)
+        elif live:
+            ctx = int(rng.choice(list(live)))
+            assert m.release(ctx) == 0
+            del live[ctx]
+        _check_invariants(m, live, n_pages, ps)
+    for ctx in list(live):
+        m.release(ctx)
+    assert m.free_pages() == n_pages
+
+
+def test_page_manager_errors():
+    m = B.KvManager(4, 16)
+    assert m.open(1, 10, 0) == 0
+    assert m.open(1, 10, 0) == B.SLED_ERR_DUP_CTX
+    assert m.reserve_batch([1, 1], [1, 1]) == B.SLED_ERR_DUP_CTX
+    assert m.reserve_batch([2], [1]) == B.SLED_ERR_UNKNOWN_CTX
+    assert m.reserve_batch([1], [16 * 4]) == B.SLED_ERR_NO_PAGES
+    assert m.commit(1, 1, 0) == B.SLED_ERR_ARG            # nothing reserved
+    assert m.release(9) == B.SLED_ERR_UNKNOWN_CTX
+    assert m.reserve_batch([1], [7]) == 0
+    assert m.commit(1, 8, 0) == B.SLED_ERR_ARG            # more than reserved
+    assert m.commit(1, 6, 3) == 0
+    assert m.query(1)[1][:2] == (16, 3)
+    assert m.free_pages() == 3                              # 16 tokens fit one page: the second went back
