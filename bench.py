@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the batched verification step (one step = one sled_verify_batch over a batch of
+synthetic device requests, commit / rollback included).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+                    [--shape llama8b] [--batch 16] [--layers L] [--greedy]
+
+Prints ONE JSON line.  Metric: verified (committed) tokens per second at the Llama-3-8B shape.
+`value` is measured with the draft distributions already in device memory, `e2e` with them in
+pinned host memory (copied in and results copied out inside the timed region).  `roofline` is for
+the tensor-core linear-layer kernel, the dominant one.  `--impl reference` times the CPU oracle.
+Under torchrun every rank runs its own replica on its own requests (no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from dataclasses import replace
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2506_09397_b200 import inputs as I
+
+METRIC = "verified_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def parse_args(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="sled", choices=["sled", "reference"])
+    ap.add_argument("--shape", default="llama8b", choices=sorted(I.SHAPES))
+    ap.add_argument("--batch", type=int, default=16)
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (small captures for ncu)")
+    ap.add_argument("--greedy", action="store_true")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args(argv)
+
+
+def workload(args, rank: int):
+    """Per-rank batch description: draft lengths and context lengths (seeded by rank)."""
+    shape = I.SHAPES[args.shape]
+    if args.layers:
+        shape = replace(shape, n_layers=args.layers)
+    seed = args.seed + 1000 * rank
+    if shape.name == "llama1b":
+        ks = I.draw_k(args.batch, [2, 3, 4, 5, 6, 7, 8], seed)
+        ctx = I.draw_context_lengths(args.batch, 256, 2048, seed)
+    elif shape.name == "llama8b":
+        ks = I.draw_k(args.batch, [3, 5, 8], seed)
+        ctx = I.draw_context_lengths(args.batch, 512, 4096, seed)
+    else:
+        ks = I.draw_k(args.batch, [2, 4, 8], seed)
+        ctx = I.draw_context_lengths(args.batch, 32, 256, seed)
+    return shape, ks, ctx, seed
+
+
+def workload_name(args, shape, ks, ctx):
+    return (f"{shape.name} ({shape.n_layers} layers) full verify step, B={args.batch}, k_i in {sorted(set(ks))}, "
+            f"contexts {min(ctx)}..{max(ctx)}, {'greedy' if args.greedy else 'sampling tau=1.0'}")
+
+
+# ------------------------------------------------------------------ clocks --
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        sm, mx, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[1]))
+                mx = max(mx, float(r[2]))
+                for name, val in zip(names, r[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                pass
+        busy = [x for x in sm if x > 0]
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------ algorithmic work --
+def linear_shapes(shape):
+    s = shape
+    qd, kd = s.n_q_heads * s.head_dim, s.n_kv_heads * s.head_dim
+    per_layer = [(qd + 2 * kd, s.d_model), (s.d_model, qd), (2 * s.ffn_dim, s.d_model), (s.d_model, s.ffn_dim)]
+    return per_layer * s.n_layers + [(s.vocab, s.d_model)]
+
+
+def linear_bytes(shape, T: int) -> float:
+    """Bytes the linear layers must move in one step: every weight once (bf16), their bf16 inputs,
+    their fp32 outputs."""
+    es = 2 if shape.weight_dtype == "bf16" else 4
+    return float(sum(n * k * es + T * k * es + T * n * 4 for n, k in linear_shapes(shape)))
+
+
+def linear_flops(shape, T: int) -> float:
+    return 2.0 * T * shape.streamed_params()
+
+
+def step_bytes(shape, ks, ctx, n_reject: int) -> float:
+    """All bytes one step must move: weights, KV read and written, logits written and read,
+    one draft-distribution row per rejecting request."""
+    T = sum(k + 1 for k in ks)
+    kvb = shape.kv_bytes_per_token()
+    return (linear_bytes(shape, T) + sum(c + k + 1 for c, k in zip(ctx, ks)) * kvb + T * kvb
+            + T * shape.vocab * 4 + n_reject * shape.vocab * 4)
+
+
+# ------------------------------------------------------------------ oracle arm --
+def oracle_sample_time(shape, weights_host, ks, ctx, seed, which: int, greedy: bool):
+    """Times the CPU oracle on request `which` of the batch.  Returns (seconds, committed tokens, threads)."""
+    from oracle import oracle as O
+    conv = lambda t: t.numpy() if t.dtype == torch.float32 else t
+    w = {k: [conv(t) for t in v] if isinstance(v, list) else conv(v) for k, v in weights_host.items()}
+    orc = O.OracleModel(shape, w)
+    K, V = I.make_kv(shape, ctx[which], seed, which)
+    orc.load_kv(which, K.float().numpy(), V.float().numpy(), pending=1)
+    del K, V
+    d, q = I.make_drafts(shape.vocab, ks[which], seed, which)
+    t0 = time.perf_counter()
+    st, n_acc, nxt, _, _ = orc.verify(which, d.numpy(), None if greedy else q.numpy(), seed, 1.0, greedy)
+    return time.perf_counter() - t0, n_acc + 1, O.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shape, ks, ctx, seed = workload(args, 0)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    w = I.weights_to(I.make_weights(shape, seed, device=dev), "cpu")
+    which = int(np.argmin(ks))
+    times, toks, threads = [], 0, 1
+    for i in range(args.warmup + args.steps):
+        dt, n_tok, threads = oracle_sample_time(shape, w, ks, ctx, seed, which, args.greedy)
+        if i >= args.warmup:
+            times.append(dt)
+            toks += n_tok
+    total = sum(times)
+    value = toks / total
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+            "config": {"workload": workload_name(args, shape, ks, ctx)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": f"each step = request {which} of the batch alone (k={ks[which]}, "
+                                       f"context {ctx[which]}), 1 of {args.batch} requests"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# -------------------------------------------------------------------- sled arm --
+def aggregate(local_tokens: float, local_ms: float, world: int):
+    """Whole-job numbers from per-rank ones: tokens add up, the time is the slowest rank's."""
+    if world == 1:
+        return local_tokens, local_ms
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([local_tokens], dtype=torch.float64, device=dev)
+    m = torch.tensor([local_ms], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    dist.all_reduce(m, op=dist.ReduceOp.MAX)
+    return float(t.item()), float(m.item())
+
+
+def run_sled(args):
+    from paper_2506_09397_b200 import binding as B
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the verification path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    shape, ks, ctx, seed = workload(args, rank)
+    Bn = args.batch
+    T = sum(k + 1 for k in ks)
+    dev = f"cuda:{local_rank}"
+
+    w = I.make_weights(shape, seed, device=dev)
+    n_pages = sum((c + k + 1 + 15) // 16 for c, k in zip(ctx, ks)) + 64
+    stream = torch.cuda.Stream(device=dev)
+    eng = B.Engine(shape, w, n_pages=n_pages, max_batch=Bn, max_k=max(ks), max_step_tokens=max(T, 16),
+                   temperature=1.0, greedy=args.greedy, device_index=local_rank, stream=stream.cuda_stream)
+    need_host_w = (rank == 0 and world == 1 and not args.no_cpu_baseline)
+    w_host = I.weights_to(w, "cpu") if need_host_w else None
+    del w
+    torch.cuda.empty_cache()
+    eng.shuffle_pages(seed)
+    for i in range(Bn):
+        K, V = I.make_kv(shape, ctx[i], seed, i, device=dev)
+        eng.load_kv(i, K, V, pending=1)
+        del K, V
+    drafts_host, q_dev, q_host = [], [], []
+    for i in range(Bn):
+        d, q = I.make_drafts(shape.vocab, ks[i], seed, i, device=dev)
+        drafts_host.append(np.ascontiguousarray(d.cpu().numpy()))
+        q_dev.append(q)
+        if not args.no_e2e:
+            q_host.append(q.cpu().pin_memory())
+    torch.cuda.synchronize()
+
+    def marshal(qs):
+        reqs = (B.SledRequest * Bn)()
+        for i in range(Bn):
+            reqs[i].ctx_id = i
+            reqs[i].draft_tokens = drafts_host[i].ctypes.data
+            reqs[i].draft_probs = None if args.greedy else qs[i].data_ptr()
+            reqs[i].k = ks[i]
+        return reqs
+
+    res = (B.SledResult * Bn)()
+    L = B.lib()
+
+    def one_step(reqs, step_seed):
+        rc = eng.verify_batch_raw(reqs, Bn, step_seed, res)
+        if rc != 0:
+            raise SystemExit(f"sled_verify_batch failed: {B.strerror(rc)}")
+        committed = 0
+        for i in range(Bn):
+            committed += res[i].n_accepted + 1
+            L.sled_debug_truncate(eng.h, i, ctx[i], 1)   # same state for every step (host bookkeeping only)
+        return committed
+
+    def timed(reqs, steps, warmup):
+        for s in range(warmup):
+            one_step(reqs, 100 + s)
+        launches0 = eng.stats().kernels_launched
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        committed = 0
+        e0.record(stream)
+        for s in range(steps):
+            committed += one_step(reqs, 1000 + s)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        return committed, e0.elapsed_time(e1), eng.stats().kernels_launched - launches0
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    reqs_dev = marshal(q_dev)
+    committed, ms, launches = timed(reqs_dev, args.steps, args.warmup)
+    clocks = sampler.stop()
+    tok_all, ms_all = aggregate(float(committed), ms, world)
+    value = tok_all / (ms_all / 1e3)
+
+    e2e = None
+    if not args.no_e2e:
+        reqs_host = marshal(q_host)
+        c2, ms2, _ = timed(reqs_host, args.steps, args.warmup)
+        t2, m2 = aggregate(float(c2), ms2, world)
+        h2d = 0 if args.greedy else sum(k * shape.vocab * 4 for k in ks)
+        e2e = {"value": t2 / (m2 / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d + 64 * T,
+               "d2h_bytes_per_step": 12 * Bn, "ms_per_step": m2 / args.steps}
+
+    # device time per kernel kind (events between kernels; extra steps, not the ones behind `value`)
+    eng.set_timing(True)
+    lin_ms, attn_ms, acc_ms, oth_ms, step_ms = [], [], [], [], []
+    n_rej = 0
+    for s in range(5):
+        one_step(reqs_dev, 2000 + s)
+        st = eng.stats()
+        lin_ms.append(st.ms_linear); attn_ms.append(st.ms_attention); acc_ms.append(st.ms_accept)
+        oth_ms.append(st.ms_other); step_ms.append(st.ms_step)
+        n_rej = sum(1 for i in range(Bn) if res[i].n_accepted < ks[i])
+    eng.set_timing(False)
+    st = eng.stats()
+    n_lin = st.linear_launches_last_step
+    lin = statistics.median(lin_ms)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    hbm_peak = peaks.get("hbm_gbs", 6650.0)
+    tc_peak = peaks.get("bf16_tflops_sustained", 1400.0)
+    peak_src = "measured" if peaks else "fallback"
+    lb, lf = linear_bytes(shape, T), linear_flops(shape, T)
+    if lb / (hbm_peak * 1e9) >= lf / (tc_peak * 1e12):
+        ach = lb / (lin / 1e3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak}
+    else:
+        ach = lf / (lin / 1e3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": tc_peak, "unit": "TFLOP/s", "frac": ach / tc_peak}
+    roof.update({"traffic": None, "kernel": "linear-layer kernel (all linear layers of a step)", "peak_source": peak_src,
+                 "launches_per_step": n_lin, "avg_launch_ms": lin / max(n_lin, 1),
+                 "algorithmic_bytes_per_step": lb, "algorithmic_flops_per_step": lf})
+    sb = step_bytes(shape, ks, ctx, n_rej)
+    step_s = ms_all / args.steps / 1e3
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_all / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if shape.weight_dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": workload_name(args, shape, ks, ctx), "tokens_scored_per_step": T,
+                       "l2": "inputs larger than L2 (a step streams %.2f GB of weights)" % (2e-9 * shape.streamed_params()),
+                       "draft_distributions": "independent of the target (softmax of N(0,1) logits)",
+                       "kv": "synthetic N(0,1) cache content in permuted 16-token pages"},
+            "clocks": clocks, "gpu_launches": int(launches),
+            "scored_positions_per_s": T * world / step_s,
+            "acceptance_rate": (committed / args.steps - Bn) / max(sum(ks), 1),
+            "step_hbm": {"algorithmic_bytes": sb, "achieved_GBps": sb / step_s / 1e9,
+                         "frac_of_hbm_peak": sb / step_s / 1e9 / hbm_peak, "peak_source": peak_src},
+            "kernel_ms": {"linear": lin, "attention": statistics.median(attn_ms), "accept": statistics.median(acc_ms),
+                          "other": statistics.median(oth_ms), "step_with_events": statistics.median(step_ms)},
+            "roofline": roof}
+    if e2e:
+        line["e2e"] = e2e
+    if need_host_w:
+        which = int(np.argmin(ks))
+        dt, n_tok, threads = oracle_sample_time(shape, w_host, ks, ctx, seed, which, args.greedy)
+        line["cpu_baseline"] = {"value": n_tok / dt, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
+                                "sample": f"request {which} of the batch alone (k={ks[which]}, context {ctx[which]}), "
+                                          f"1 of {Bn} requests, one pass"}
+    eng.shutdown()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main(argv=None):
+    args = parse_args(argv)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_sled(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -61,7 +61,8 @@ typedef struct sled_config {
   int32_t max_step_tokens;/* most sum(k_i + 1) per step; also the prefill chunk */
   float temperature;      /* divides the target logits before the softmax (> 0) */
   int32_t greedy;         /* 1: accept iff the draft equals the argmax, emit the argmax */
-  int32_t probs_on_device;/* 1: sled_request.draft_probs are DEVICE pointers */
+  int32_t probs_on_device;/* 1: every sled_request.draft_probs will be a DEVICE pointer (no staging buffer is
+                             allocated, host rows are then refused); 0: host or device, found out per request */
   int32_t device_index;   /* CUDA device ordinal */
   void* stream;           /* cudaStream_t to launch on; NULL: the engine creates one */
 } sled_config;
@@ -91,8 +92,8 @@ typedef struct sled_weights {
 typedef struct sled_request {
   uint64_t ctx_id;             /* context opened by sled_prefill */
   const int32_t* draft_tokens; /* [k], host */
-  const float* draft_probs;    /* [k][vocab] fp32, rows sum to 1; host, or device if probs_on_device;
-                                  may be NULL when k == 0 or in greedy mode */
+  const float* draft_probs;    /* [k][vocab] fp32, rows sum to 1; host (copied in during the forward pass) or
+                                  device (read in place); may be NULL when k == 0 or in greedy mode */
   int32_t k;                   /* 0 <= k <= max_k; k = 0 is an ordinary decoding step */
 } sled_request;
 

@@ -742,7 +742,12 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
       h_hi[i] = static_cast<uint32_t>(ctxs[i] >> 32);
       h_qptr[i] = nullptr;
       if (reqs[i].k > 0 && !c.greedy) {
-        if (c.probs_on_device) h_qptr[i] = reqs[i].draft_probs;
+        cudaPointerAttributes attr{};
+        const bool on_device = cudaPointerGetAttributes(&attr, reqs[i].draft_probs) == cudaSuccess &&
+                               attr.type == cudaMemoryTypeDevice;
+        cudaGetLastError();
+        if (on_device) h_qptr[i] = reqs[i].draft_probs;   // read in place by the acceptance kernel
+        else if (!e->q_stage) return rollback(SLED_ERR_ARG);  // engine was created for device-resident rows only
         else {
           // draft distributions travel on the copy stream while the forward pass runs
           float* dst = e->q_stage + row * c.vocab;

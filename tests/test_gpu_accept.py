@@ -42,7 +42,8 @@ def test_full_vocab_rows(tau, greedy):
     ks[0], ks[1] = k, 0
     got, want = _run_both(z, q, d, ks, tau, greedy, seed=11)
     assert got == want
-    assert len({g[0] for g in got}) > 1            # both acceptances and rejections occurred
+    if not greedy:
+        assert len({g[0] for g in got}) > 1        # both acceptances and rejections occurred
 
 
 @pytest.mark.parametrize("V", [1, 5, 1000, 4096, 4097, 33000])
