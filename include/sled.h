@@ -168,6 +168,26 @@ int sled_accept_rows(const float* logits, const int32_t* cu_rows, const int32_t*
                      float temperature, int32_t greedy, uint64_t seed, sled_result* results, void* stream,
                      float* device_ms);
 
+/* The same acceptance as sled_accept_rows for callers that must not allocate device memory
+ * (the paper has no counterpart: this is a property of the library, not of the method).
+ * A process whose GPU memory is wholly owned by another allocator, a latency path on which an
+ * allocation would stall the device, or a caller between two points of a fixed schedule cannot
+ * afford the cudaMalloc / cudaFree pair that sled_accept_rows performs for its small device-side
+ * description of the batch.  Here that description lives in a fixed array inside the library
+ * image: SLED_STATIC_MAX_REQS requests and SLED_STATIC_MAX_ROWS rows at most (about 90 KB, held
+ * by every GPU that loads the library until the process ends).  Larger batches are refused with
+ * SLED_ERR_BATCH_TOO_LARGE.  The call allocates nothing on the device and nothing on the host
+ * heap; it does not measure time.  Arguments and results are those of sled_accept_rows.
+ * The first call on a device looks up the array's device address (with that device current);
+ * make that first call before starting any stream capture.  All calls on a device share the one
+ * array and every call rewrites it completely, so two calls must not overlap on the GPU: issue
+ * them from one thread, one after the other (the call synchronises `stream` before returning). */
+#define SLED_STATIC_MAX_REQS 1024
+#define SLED_STATIC_MAX_ROWS 8192
+int sled_accept_rows_static(const float* logits, const int32_t* cu_rows, const int32_t* drafts, const float* q_rows,
+                            const uint64_t* ctx_ids, const int64_t* pos0, int32_t n_reqs, int32_t vocab,
+                            float temperature, int32_t greedy, uint64_t seed, sled_result* results, void* stream);
+
 /* Ragged verification attention only, over the engine's paged cache: request i's last
  * q_len[i] cached tokens are taken as the new ones; query j of request i attends to the
  * keys 0 .. n_kv_i - q_len_i + j of ctx_ids[i] in layer `layer`.

@@ -22,7 +22,7 @@ SLED_F32, SLED_BF16 = 0, 1
 
 EXPORTS = (
     "sled_init", "sled_verify_batch", "sled_release", "sled_prefill", "sled_set_sampling", "sled_get_stats",
-    "sled_get_stream", "sled_shutdown", "sled_strerror", "sled_accept_rows", "sled_attention_ragged",
+    "sled_get_stream", "sled_shutdown", "sled_strerror", "sled_accept_rows", "sled_accept_rows_static", "sled_attention_ragged",
     "sled_debug_load_kv", "sled_debug_read_kv", "sled_debug_copy_logits", "sled_debug_truncate",
     "sled_debug_set_commit", "sled_debug_set_timing", "sled_debug_query_ctx", "sled_debug_shuffle_pages",
     "sled_kvm_create", "sled_kvm_destroy", "sled_kvm_open", "sled_kvm_reserve_batch", "sled_kvm_commit",
@@ -91,6 +91,7 @@ def lib():
             "sled_strerror": (C.c_char_p, [C.c_int]),
             "sled_accept_rows": (C.c_int, [P, P, P, P, P, P, I32, I32, F, I32, U64, C.POINTER(SledResult), P,
                                            C.POINTER(F)]),
+            "sled_accept_rows_static": (C.c_int, [P, P, P, P, P, P, I32, I32, F, I32, U64, C.POINTER(SledResult), P]),
             "sled_attention_ragged": (C.c_int, [P, I32, P, P, I32, P, P, C.POINTER(F)]),
             "sled_debug_load_kv": (C.c_int, [P, U64, P, P, I32, I32]),
             "sled_debug_read_kv": (C.c_int, [P, U64, I32, P, P, I32]),
@@ -282,6 +283,24 @@ def accept_rows(logits: torch.Tensor, cu_rows, drafts, q_rows, ctx_ids, pos0, te
                                   logits.shape[1], temperature, int(greedy), seed, res, stream, C.byref(ms)),
            "sled_accept_rows")
     return [(res[i].n_accepted, res[i].next_token, res[i].status) for i in range(n)], ms.value
+
+
+def accept_rows_static(logits: torch.Tensor, cu_rows, drafts, q_rows, ctx_ids, pos0, temperature: float,
+                       greedy: bool, seed: int, stream: int = 0):
+    """sled_accept_rows_static: same arguments and results as accept_rows, for callers that must not
+    allocate device memory (the batch description goes into a fixed array inside the library, at most
+    1024 requests / 8192 rows; calls on one device must not overlap).  Returns the result list."""
+    cu = np.ascontiguousarray(np.asarray(cu_rows, dtype=np.int32))
+    n = cu.size - 1
+    d = np.ascontiguousarray(np.asarray(drafts, dtype=np.int32).reshape(-1))
+    ids = np.ascontiguousarray(np.asarray(ctx_ids, dtype=np.uint64))
+    p0 = np.ascontiguousarray(np.asarray(pos0, dtype=np.int64))
+    res = (SledResult * max(n, 1))()
+    _check(lib().sled_accept_rows_static(logits.data_ptr(), cu.ctypes.data, d.ctypes.data if d.size else None,
+                                         _addr(q_rows) if q_rows is not None else None, ids.ctypes.data,
+                                         p0.ctypes.data, n, logits.shape[1], temperature, int(greedy), seed, res,
+                                         stream), "sled_accept_rows_static")
+    return [(res[i].n_accepted, res[i].next_token, res[i].status) for i in range(n)]
 
 
 class KvManager:
