@@ -69,6 +69,7 @@ struct sled_engine {
   char* kpool = nullptr;
   char* vpool = nullptr;
   size_t kv_layer_bytes = 0;
+  std::vector<CUtensorMap> kv_maps;  // [2 * layer + {0: K, 1: V}] for the tensor-core attention kernel
   float* x = nullptr;
   void* act_norm = nullptr;
   void* q_buf = nullptr;
@@ -311,6 +312,11 @@ AttnArgs attn_args(sled_engine* e, const Packed& pk, int layer, const void* q, v
   a.chunk_keys = pk.chunk_keys;
   a.adtype = e->adtype();
   a.kvdtype = e->cfg.kv_dtype;
+  if (!e->kv_maps.empty()) {
+    a.map_k = &e->kv_maps[2 * layer];
+    a.map_v = &e->kv_maps[2 * layer + 1];
+    a.error = e->tc_error;
+  }
   return a;
 }
 
@@ -566,6 +572,9 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->kpool), e->kv_layer_bytes * c.n_layers))) return fail(rc);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->vpool), e->kv_layer_bytes * c.n_layers))) return fail(rc);
 
+  CU_TRY(cudaMemset(e->kpool, 0, e->kv_layer_bytes * c.n_layers));  // never-written slots are read (and masked): keep them finite
+  CU_TRY(cudaMemset(e->vpool, 0, e->kv_layer_bytes * c.n_layers));
+
   // step workspaces
   const size_t maxT = c.max_step_tokens, as = dtype_size(e->adtype());
   const size_t padT = align_up(maxT, 256);  // activation buffers are read in row tiles by the tensor-core path
@@ -596,6 +605,14 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if (c.weight_dtype == SLED_BF16) {
     if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->tc_error), 16))) return fail(rc);
     CU_TRY(cudaMemset(e->tc_error, 0, 16));
+    if (c.page_size == 16 && (c.head_dim == 64 || c.head_dim == 128)) {
+      e->kv_maps.resize(2 * c.n_layers);
+      const long long rows = static_cast<long long>(c.n_pages) * c.n_kv_heads * c.page_size;
+      for (int l = 0; l < c.n_layers; ++l)
+        if (tma_map_bf16_rows(&e->kv_maps[2 * l], e->kpool + e->kv_layer_bytes * l, rows, c.head_dim, 16) ||
+            tma_map_bf16_rows(&e->kv_maps[2 * l + 1], e->vpool + e->kv_layer_bytes * l, rows, c.head_dim, 16))
+          return fail(SLED_ERR_DEVICE);
+    }
     if (tc_activation_init(&e->tc_norm, e->act_norm, static_cast<int>(padT), d) ||
         tc_activation_init(&e->tc_attn, e->attn_out, static_cast<int>(padT), qd) ||
         tc_activation_init(&e->tc_ffn, e->act_ffn, static_cast<int>(padT), F))

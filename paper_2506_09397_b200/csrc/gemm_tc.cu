@@ -239,7 +239,7 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-int make_map(CUtensorMap* map, const void* ptr, int rows, int K, int box_rows) {
+int make_map(CUtensorMap* map, const void* ptr, long long rows, int K, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return -1;
   if (K % 8 || (reinterpret_cast<uintptr_t>(ptr) & 15)) return -1;   // rows must stay 16-byte aligned; a K tail is zero-filled by TMA
@@ -251,7 +251,7 @@ int make_map(CUtensorMap* map, const void* ptr, int rows, int K, int box_rows) {
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
-    std::fprintf(stderr, "sled: cuTensorMapEncodeTiled failed (%d) rows=%d K=%d box=%d\n", static_cast<int>(r), rows, K, box_rows);
+    std::fprintf(stderr, "sled: cuTensorMapEncodeTiled failed (%d) rows=%lld K=%d box=%d\n", static_cast<int>(r), rows, K, box_rows);
     return -1;
   }
   return 0;
@@ -277,6 +277,10 @@ int launch_one(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K
 int tile_tokens(int T) { return T <= 64 ? 64 : (T <= 128 ? 128 : 256); }
 
 }  // namespace
+
+int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int cols, int box_rows) {
+  return make_map(map, dev_ptr, rows, cols, box_rows);
+}
 
 int tc_weight_init(TcWeight* w, const void* dev_ptr, int N, int K) {
   if (make_map(&w->map, dev_ptr, N, K, kBlockM)) return -1;

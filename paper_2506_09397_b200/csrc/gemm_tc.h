@@ -20,6 +20,8 @@ struct TcActivation {   // [rows][K] bf16, row-major, device memory; rows is a m
   int rows = 0, K = 0;
 };
 
+// 2D bf16 tensor map over a row-major [rows][cols] array: boxes of 64 columns x box_rows rows, 128-byte swizzle
+int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int cols, int box_rows);
 int tc_weight_init(TcWeight* w, const void* dev_ptr, int N, int K);
 void tc_weight_free(TcWeight* w);
 int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K);

@@ -1,6 +1,7 @@
 // Host-callable launchers of the device kernels.  Every launcher only enqueues work on
 // the given stream and returns the number of kernels it launched (negative: bad argument).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -50,8 +51,15 @@ struct AttnArgs {
   float* part_ml;            // [rows][Hq][2]
   int T, Hq, Hkv, h, page_size, chunk_keys;
   int adtype, kvdtype;
+  // tensor-core path (bf16 cache, 16-token pages): tensor maps over this layer's K and V pool
+  // viewed as [page*Hkv*16 + slot][h], and a device word that records a bounded wait running out
+  const CUtensorMap* map_k = nullptr;
+  const CUtensorMap* map_v = nullptr;
+  int32_t* error = nullptr;
 };
 int launch_attention(const AttnArgs& a, cudaStream_t s);
+// tensor-core kernel alone (attention_mma.cu); returns 1 or a negative value
+int launch_attention_mma(const AttnArgs& a, cudaStream_t s);
 
 // ---- fused vocabulary softmax + acceptance + corrective / bonus draw (accept.cu)
 struct AcceptArgs {
