@@ -87,6 +87,7 @@ struct Shared {
 
 __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
   __shared__ Shared sh;
+  pdl_enter();
   const int req = blockIdx.x;
   const int row0 = a.cu_q[req];
   const int k = a.cu_q[req + 1] - row0 - 1;
@@ -258,7 +259,7 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
 int launch_accept(const AcceptArgs& a, cudaStream_t s) {
   if (a.B <= 0) return 0;
   if (a.V > kTile * kMaxTiles) return -1;
-  accept_kernel<<<a.B, kThreads, 0, s>>>(a);
+  SLED_LAUNCH_PDL(accept_kernel, dim3(a.B), dim3(kThreads), 0, s, a);
   return 1;
 }
 

@@ -42,6 +42,7 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(AttnArgs a) {
   constexpr int EPV = 16 / sizeof(KT);  // storage elements per 16-byte load
   __shared__ __align__(16) float Ks[kTileKeys][H];
   __shared__ __align__(16) float Vs[kTileKeys][H];
+  pdl_enter();
 
   const int4 item = a.items[blockIdx.x];
   const int req = item.x, kvh = item.y, key_start = item.z, key_count = item.w;
@@ -161,6 +162,7 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(AttnArgs a) {
 // Merge of the per-chunk partial results of split requests: grid (T, Hq), h threads.
 template <typename AT>
 __global__ void attn_merge_kernel(AttnArgs a) {
+  pdl_enter();
   const int t = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
   const int n = a.req_chunks[a.tok_req[t]];
   if (n <= 1) return;
@@ -182,11 +184,11 @@ __global__ void attn_merge_kernel(AttnArgs a) {
 template <typename KT, typename AT>
 int launch_typed(const AttnArgs& a, cudaStream_t s) {
   if (a.h == 64)
-    attn_simt_kernel<KT, AT, 64><<<a.n_items, 256, 0, s>>>(a);
+    SLED_LAUNCH_PDL((attn_simt_kernel<KT, AT, 64>), dim3(a.n_items), dim3(256), 0, s, a);
   else if (a.h == 128)
-    attn_simt_kernel<KT, AT, 128><<<a.n_items, 256, 0, s>>>(a);
+    SLED_LAUNCH_PDL((attn_simt_kernel<KT, AT, 128>), dim3(a.n_items), dim3(256), 0, s, a);
   else if (a.h == 32)
-    attn_simt_kernel<KT, AT, 32><<<a.n_items, 256, 0, s>>>(a);
+    SLED_LAUNCH_PDL((attn_simt_kernel<KT, AT, 32>), dim3(a.n_items), dim3(256), 0, s, a);
   else
     return -1;
   return 1;
@@ -205,8 +207,8 @@ int launch_attention(const AttnArgs& a, cudaStream_t s) {
   if (n < 0) return n;
   if (a.part_acc) {  // some request was split
     dim3 grid(a.T, a.Hq);
-    if (a.adtype == BF16) attn_merge_kernel<__nv_bfloat16><<<grid, a.h, 0, s>>>(a);
-    else attn_merge_kernel<float><<<grid, a.h, 0, s>>>(a);
+    if (a.adtype == BF16) SLED_LAUNCH_PDL(attn_merge_kernel<__nv_bfloat16>, grid, dim3(a.h), 0, s, a);
+    else SLED_LAUNCH_PDL(attn_merge_kernel<float>, grid, dim3(a.h), 0, s, a);
     ++n;
   }
   return n;

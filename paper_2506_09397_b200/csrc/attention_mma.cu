@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(AttnArgs a, const __grid_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, tq = lane & 3;
+  pdl_enter();
   if (threadIdx.x == 0) s_abort = *reinterpret_cast<volatile int32_t*>(a.error);
   __syncthreads();
   if (s_abort != 0) return;
@@ -308,7 +309,7 @@ int launch_h(const AttnArgs& a, cudaStream_t s) {
       return -1;
     configured = true;
   }
-  attn_mma_kernel<H><<<a.n_items, 128, L::kTotal, s>>>(a, *a.map_k, *a.map_v);
+  SLED_LAUNCH_PDL(attn_mma_kernel<H>, dim3(a.n_items), dim3(128), L::kTotal, s, a, *a.map_k, *a.map_v);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -37,4 +37,32 @@ __device__ __forceinline__ float block_sum(float v, float* scratch) {
   return warp_sum(t);
 }
 
+// Programmatic dependent launch.  Every kernel of a verification step is launched so that it may
+// begin while its predecessor in the stream drains; it lets its own successor do the same at once
+// and must call pdl_wait() before it touches anything an earlier kernel wrote (and before it exits,
+// so that "this grid is complete" always implies "everything before it is complete").
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() {
+  pdl_launch_dependents();
+  pdl_wait();
+}
+
 }  // namespace sled
+
+// Launch with the programmatic-serialization attribute (host side).  `kern` must be a concrete
+// __global__ function (template arguments spelled out).
+#define SLED_LAUNCH_PDL(kern, grid_, block_, smem_, stream_, ...)                                  \
+  do {                                                                                         \
+    cudaLaunchConfig_t cfg__{};                                                                \
+    cfg__.gridDim = (grid_);                                                                    \
+    cfg__.blockDim = (block_);                                                                  \
+    cfg__.dynamicSmemBytes = (smem_);                                                           \
+    cfg__.stream = (stream_);                                                                   \
+    cudaLaunchAttribute attr__[1];                                                             \
+    attr__[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                         \
+    attr__[0].val.programmaticStreamSerializationAllowed = 1;                                  \
+    cfg__.attrs = attr__;                                                                      \
+    cfg__.numAttrs = 1;                                                                        \
+    cudaLaunchKernelEx(&cfg__, kern, __VA_ARGS__);                                             \
+  } while (0)

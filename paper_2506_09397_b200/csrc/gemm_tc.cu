@@ -87,6 +87,8 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
       : "memory");
 }
 
+__device__ __forceinline__ void pdl_wait_here() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -103,7 +105,7 @@ template <int TN_MAX, int STAGES>
 __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CUtensorMap map_w,
                                                        const __grid_constant__ CUtensorMap map_a, int T, int N,
                                                        int kb_total, int kb_per_split, float* __restrict__ out,
-                                                       long long split_stride, int32_t* error) {
+                                                       long long split_stride, int32_t* error, int cluster) {
   using L = SmemLayout<TN_MAX, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -114,7 +116,13 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
   volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * (2 * STAGES + 1) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m_tile = blockIdx.x, t_tile = blockIdx.y, split = blockIdx.z;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its own prologue
+  // cluster == 1: K slices (if any) are separate CTAs along grid z, each leaving its own partial sum.
+  // cluster  > 1: the CTAs of a cluster share one output tile, each takes one K slice, and the partial
+  //               sums are added up through distributed shared memory before one result is stored.
+  const int rank = cluster > 1 ? static_cast<int>(blockIdx.x % cluster) : 0;
+  const int m_tile = cluster > 1 ? blockIdx.x / cluster : blockIdx.x, t_tile = blockIdx.y;
+  const int split = cluster > 1 ? rank : blockIdx.z;
   const int kb0 = split * kb_per_split;
   const int nkb = min(kb_per_split, kb_total - kb0);
   const int t0 = t_tile * TN_MAX;
@@ -122,7 +130,11 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
 
   if (threadIdx.x == 0) *abort_slot = *reinterpret_cast<volatile int32_t*>(error);
   __syncthreads();
-  if (*abort_slot != 0) return;                           // an earlier CTA gave up: do not start
+  const int seen_abort = *abort_slot;
+  __syncthreads();
+  if (seen_abort != 0 && cluster == 1) return;            // an earlier CTA gave up: do not start (a cluster's
+                                                          // CTAs must all reach its barriers, so they never leave early)
+  if (threadIdx.x == 0) *abort_slot = 0;
 
   if (warp == 0 && lane == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
@@ -146,7 +158,18 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
       uint64_t pol_first, pol_last;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_last));
-      for (int kb = 0; kb < nkb; ++kb) {
+      // The weights do not depend on the previous kernel: fill the ring with weight slabs first, then wait
+      // for the predecessor (its output is this kernel's activation operand), then add the activation slabs.
+      const int pre = min(STAGES, nkb);
+      for (int kb = 0; kb < pre; ++kb) {
+        const uint32_t full = bars + 8 * kb;
+        mbar_expect_tx(full, L::kStageBytes);
+        tma_load_2d(base + kb * L::kStageBytes, &map_w, (kb0 + kb) * kBlockK, m_tile * kBlockM, full, pol_first);
+      }
+      pdl_wait_here();
+      for (int kb = 0; kb < pre; ++kb)
+        tma_load_2d(base + kb * L::kStageBytes + kWStageBytes, &map_a, (kb0 + kb) * kBlockK, t0, bars + 8 * kb, pol_last);
+      for (int kb = pre; kb < nkb; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
         if (!mbar_wait(bars + 8 * (STAGES + s), ph ^ 1, error, 1)) { ok = false; break; }
@@ -180,7 +203,7 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
     const int quad = warp & 3;                      // a warp may only touch tensor-memory lanes 32*(warp%4)..+31
     if (nkb > 0) ok = mbar_wait(bars + 8 * (2 * STAGES), 0, error, 3);
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-    if (ok) {
+    if (ok && cluster == 1) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int n = m_tile * kBlockM + quad * 32 + lane;
       float* dst = out + static_cast<long long>(split) * split_stride + n;
@@ -203,6 +226,59 @@ __global__ void __launch_bounds__(192) tc_gemm_kernel(const __grid_constant__ CU
             const int t = t0 + c0 + i;
             if (t < T) dst[static_cast<long long>(t) * N] = __uint_as_float(v[i]);
           }
+        }
+      }
+    }
+  }
+
+  if (cluster > 1) {
+    // Reduction over the cluster.  The accumulator tile is cut into chunks of 16 token columns; chunk c
+    // belongs to rank c % cluster.  Every CTA sends each chunk of its partial sum to the owner's shared
+    // memory (slot [c / cluster][sender], laid out [column][128 rows]); the pipeline stages are reused as
+    // receive space, hence the first barrier: nobody may still be streaming operands.  Owners then add the
+    // senders' slots in rank order, so the result does not depend on timing.
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    const int n_chunks = tn >> 4;
+    const int quad = warp & 3, row = quad * 32 + lane;
+    if (warp >= 2) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      for (int c = 0; c < n_chunks; ++c) {
+        const int owner = c % cluster, slot = c / cluster;
+        uint32_t v[16];
+        if (ok && nkb > 0) {
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+              : "r"(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(c * 16)));
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = 0u;
+        }
+        const uint32_t local = base + static_cast<uint32_t>(((slot * cluster + rank) * 2048 + row) * 4);
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(owner));
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(remote + i * 512), "r"(v[i]) : "memory");
+      }
+    }
+    __syncwarp();
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (warp >= 2) {
+      const float* recv = reinterpret_cast<const float*>(base_ptr);
+      const int n = m_tile * kBlockM + row;
+      for (int c = rank; c < n_chunks; c += cluster) {
+        const int slot = c / cluster;
+#pragma unroll 4
+        for (int i = 0; i < 16; ++i) {
+          float sum = 0.f;
+          for (int src = 0; src < cluster; ++src) sum += recv[(slot * cluster + src) * 2048 + i * 128 + row];
+          const int t = t0 + c * 16 + i;
+          if (t < T && n < N) out[static_cast<long long>(t) * N + n] = sum;
         }
       }
     }
@@ -258,7 +334,7 @@ int make_map(CUtensorMap* map, const void* ptr, long long rows, int K, int box_r
 }
 
 template <int TN_MAX, int STAGES>
-int launch_one(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K, int n_split, float* out,
+int launch_one(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K, int n_split, int cluster, float* out,
                int64_t split_stride, int32_t* error, cudaStream_t s) {
   using L = SmemLayout<TN_MAX, STAGES>;
   static bool configured = false;
@@ -268,10 +344,27 @@ int launch_one(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K
     configured = true;
   }
   const int kb_total = (K + kBlockK - 1) / kBlockK;
-  const int kb_per = (kb_total + n_split - 1) / n_split;
-  dim3 grid((N + kBlockM - 1) / kBlockM, (T + TN_MAX - 1) / TN_MAX, n_split);
-  tc_gemm_kernel<TN_MAX, STAGES><<<grid, 192, L::kTotal, s>>>(mw, ma, T, N, kb_total, kb_per, out, split_stride, error);
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  const int slices = cluster > 1 ? cluster : n_split;
+  const int kb_per = (kb_total + slices - 1) / slices;
+  const int m_tiles = (N + kBlockM - 1) / kBlockM, t_tiles = (T + TN_MAX - 1) / TN_MAX;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = cluster > 1 ? dim3(m_tiles * cluster, t_tiles, 1) : dim3(m_tiles, t_tiles, n_split);
+  cfg.blockDim = dim3(192, 1, 1);
+  cfg.dynamicSmemBytes = L::kTotal;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster > 1 ? cluster : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while the previous kernel drains
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  const long long stride = split_stride;
+  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<TN_MAX, STAGES>, mw, ma, T, N, kb_total, kb_per, out, stride, error,
+                                       cluster);
+  return err == cudaSuccess ? 1 : -1;
 }
 
 int tile_tokens(int T) { return T <= 64 ? 64 : (T <= 128 ? 128 : 256); }
@@ -302,27 +395,34 @@ int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K) {
   return 0;
 }
 
-int tc_gemm_split(int T, int N, int K, int n_sm) {
+// Cluster size (= number of K slices reduced on chip) for a shape: as many slices as keep all CTAs resident
+// at once (two per SM), power of two, every slice non-empty.  Token tiles wider than 128 columns would not
+// fit the receive space, they run unsplit.
+static int choose_cluster(int T, int N, int K, int n_sm) {
   const int tn = tile_tokens(T);
+  if (tn > 128) return 1;
   const int tiles = ((N + kBlockM - 1) / kBlockM) * ((T + tn - 1) / tn);
   const int kb_total = (K + kBlockK - 1) / kBlockK;
-  const int target = 2 * n_sm;                 // two CTAs fit on an SM
-  int s = 1;
-  if (tiles * 5 < target * 3) s = (target + tiles - 1) / tiles;
-  s = std::min(s, std::max(1, kb_total / 4));  // at least 4 slabs per slice
-  s = std::max(1, std::min(s, 16));
-  const int kb_per = (kb_total + s - 1) / s;
-  return (kb_total + kb_per - 1) / kb_per;     // slices that actually get work
+  for (int c = 8; c >= 2; c >>= 1) {
+    const int kb_per = (kb_total + c - 1) / c;
+    if (tiles * c <= 2 * n_sm && kb_total >= 2 * c && (c - 1) * kb_per < kb_total) return c;
+  }
+  return 1;
+}
+
+int tc_gemm_split(int T, int N, int K, int n_sm) {
+  (void)T; (void)N; (void)K; (void)n_sm;
+  return 1;   // K slices are reduced inside the kernel: one output slice
 }
 
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
                    int32_t* error, int n_sm, cudaStream_t s) {
-  (void)n_sm;
-  if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
+  if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split != 1) return -1;
   const int tn = tile_tokens(T);
-  if (tn == 64) return launch_one<64, 4>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, s);
-  if (tn == 128) return launch_one<128, 3>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, s);
-  return launch_one<256, 2>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, s);
+  const int cluster = choose_cluster(T, w.N, w.K, n_sm);
+  if (tn == 64) return launch_one<64, 4>(w.map, a.map[0], T, w.N, w.K, 1, cluster, out, split_stride, error, s);
+  if (tn == 128) return launch_one<128, 3>(w.map, a.map[1], T, w.N, w.K, 1, cluster, out, split_stride, error, s);
+  return launch_one<256, 2>(w.map, a.map[2], T, w.N, w.K, 1, cluster, out, split_stride, error, s);
 }
 
 }  // namespace sled

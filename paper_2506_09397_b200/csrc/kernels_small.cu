@@ -11,6 +11,7 @@ namespace sled {
 // ------------------------------------------------------------------ embedding --
 template <typename WT>
 __global__ void embed_kernel(const WT* __restrict__ table, const int32_t* __restrict__ ids, int d, float* __restrict__ x) {
+  pdl_enter();
   const int t = blockIdx.x;
   const WT* row = table + static_cast<int64_t>(ids[t]) * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) x[static_cast<int64_t>(t) * d + i] = to_f32(row[i]);
@@ -19,9 +20,9 @@ __global__ void embed_kernel(const WT* __restrict__ table, const int32_t* __rest
 int launch_embed(const void* table, int wdtype, const int32_t* ids, int T, int d, float* x, cudaStream_t s) {
   if (T <= 0) return 0;
   if (wdtype == BF16)
-    embed_kernel<<<T, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(table), ids, d, x);
+    SLED_LAUNCH_PDL(embed_kernel<__nv_bfloat16>, dim3(T), dim3(256), 0, s, static_cast<const __nv_bfloat16*>(table), ids, d, x);
   else
-    embed_kernel<<<T, 256, 0, s>>>(static_cast<const float*>(table), ids, d, x);
+    SLED_LAUNCH_PDL(embed_kernel<float>, dim3(T), dim3(256), 0, s, static_cast<const float*>(table), ids, d, x);
   return 1;
 }
 
@@ -33,6 +34,7 @@ template <typename WT, typename AT>
 __global__ void add_rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ partial, int n_split,
                                    int64_t split_stride, const WT* __restrict__ gain, float eps, int d,
                                    AT* __restrict__ out) {
+  pdl_enter();
   __shared__ float scratch[32];
   const int64_t base = static_cast<int64_t>(blockIdx.x) * d;
   float ss = 0.f;
@@ -54,11 +56,11 @@ int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t spli
   if (!partial) n_split = 0;
   const int nt = d >= 2048 ? 512 : 256;
   if (wdtype == BF16 && adtype == BF16)
-    add_rmsnorm_kernel<<<T, nt, 0, s>>>(x, partial, n_split, split_stride, static_cast<const __nv_bfloat16*>(gain), eps,
-                                        d, static_cast<__nv_bfloat16*>(out));
+    SLED_LAUNCH_PDL((add_rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16>), dim3(T), dim3(nt), 0, s, x, partial, n_split,
+                    split_stride, static_cast<const __nv_bfloat16*>(gain), eps, d, static_cast<__nv_bfloat16*>(out));
   else if (wdtype == F32 && adtype == F32)
-    add_rmsnorm_kernel<<<T, nt, 0, s>>>(x, partial, n_split, split_stride, static_cast<const float*>(gain), eps, d,
-                                        static_cast<float*>(out));
+    SLED_LAUNCH_PDL((add_rmsnorm_kernel<float, float>), dim3(T), dim3(nt), 0, s, x, partial, n_split, split_stride,
+                    static_cast<const float*>(gain), eps, d, static_cast<float*>(out));
   else
     return -1;
   return 1;
@@ -68,6 +70,7 @@ int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t spli
 // cs[t][i] = (cos, sin)(pos_t * theta^(-2i/h)), angle and functions in fp64, stored fp32;
 // computed once per step and shared by all layers and heads.
 __global__ void rope_table_kernel(const int32_t* __restrict__ tok_pos, int h, double log2_theta, float2* __restrict__ cs) {
+  pdl_enter();
   const int t = blockIdx.x, i = threadIdx.x;
   if (i >= h / 2) return;
   const double inv_freq = exp2(-2.0 * static_cast<double>(i) / static_cast<double>(h) * log2_theta);
@@ -78,7 +81,7 @@ __global__ void rope_table_kernel(const int32_t* __restrict__ tok_pos, int h, do
 
 int launch_rope_table(const int32_t* tok_pos, int T, int h, float theta, float2* cs, cudaStream_t s) {
   if (T <= 0) return 0;
-  rope_table_kernel<<<T, h / 2, 0, s>>>(tok_pos, h, log2(static_cast<double>(theta)), cs);
+  SLED_LAUNCH_PDL(rope_table_kernel, dim3(T), dim3(h / 2), 0, s, tok_pos, h, log2(static_cast<double>(theta)), cs);
   return 1;
 }
 
@@ -90,6 +93,7 @@ __global__ void rope_kv_kernel(const float* __restrict__ partial, int n_split, i
                                const float2* __restrict__ cs, const int32_t* __restrict__ tok_slot, int Hq, int Hkv,
                                int h, int page_size, AT* __restrict__ q_out, KT* __restrict__ kpool,
                                KT* __restrict__ vpool) {
+  pdl_enter();
   const int t = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
   const int n_cols = (Hq + 2 * Hkv) * h;
   const int64_t src = static_cast<int64_t>(t) * n_cols + head * h + 2 * i;
@@ -126,17 +130,14 @@ int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, cons
   if (T <= 0) return 0;
   dim3 grid(T, Hq + 2 * Hkv);
   if (adtype == BF16 && kvdtype == BF16)
-    rope_kv_kernel<<<grid, h / 2, 0, s>>>(partial, n_split, split_stride, cs, tok_slot, Hq, Hkv, h, page_size,
-                                          static_cast<__nv_bfloat16*>(q_out), static_cast<__nv_bfloat16*>(kpool),
-                                          static_cast<__nv_bfloat16*>(vpool));
+    SLED_LAUNCH_PDL((rope_kv_kernel<__nv_bfloat16, __nv_bfloat16>), grid, dim3(h / 2), 0, s, partial, n_split, split_stride, cs, tok_slot,
+                    Hq, Hkv, h, page_size, static_cast<__nv_bfloat16*>(q_out), static_cast<__nv_bfloat16*>(kpool), static_cast<__nv_bfloat16*>(vpool));
   else if (adtype == F32 && kvdtype == F32)
-    rope_kv_kernel<<<grid, h / 2, 0, s>>>(partial, n_split, split_stride, cs, tok_slot, Hq, Hkv, h, page_size,
-                                          static_cast<float*>(q_out), static_cast<float*>(kpool),
-                                          static_cast<float*>(vpool));
+    SLED_LAUNCH_PDL((rope_kv_kernel<float, float>), grid, dim3(h / 2), 0, s, partial, n_split, split_stride, cs, tok_slot,
+                    Hq, Hkv, h, page_size, static_cast<float*>(q_out), static_cast<float*>(kpool), static_cast<float*>(vpool));
   else if (adtype == F32 && kvdtype == BF16)
-    rope_kv_kernel<<<grid, h / 2, 0, s>>>(partial, n_split, split_stride, cs, tok_slot, Hq, Hkv, h, page_size,
-                                          static_cast<float*>(q_out), static_cast<__nv_bfloat16*>(kpool),
-                                          static_cast<__nv_bfloat16*>(vpool));
+    SLED_LAUNCH_PDL((rope_kv_kernel<float, __nv_bfloat16>), grid, dim3(h / 2), 0, s, partial, n_split, split_stride, cs, tok_slot,
+                    Hq, Hkv, h, page_size, static_cast<float*>(q_out), static_cast<__nv_bfloat16*>(kpool), static_cast<__nv_bfloat16*>(vpool));
   else
     return -1;
   return 1;
@@ -147,6 +148,7 @@ int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, cons
 template <typename AT>
 __global__ void swiglu_kernel(const float* __restrict__ partial, int n_split, int64_t split_stride, int F,
                               AT* __restrict__ out) {
+  pdl_enter();
   const int t = blockIdx.y;
   const int f = blockIdx.x * blockDim.x + threadIdx.x;
   if (f >= F) return;
@@ -164,9 +166,9 @@ int launch_swiglu(const float* partial, int n_split, int64_t split_stride, int T
   if (T <= 0) return 0;
   dim3 grid((F + 255) / 256, T);
   if (adtype == BF16)
-    swiglu_kernel<<<grid, 256, 0, s>>>(partial, n_split, split_stride, F, static_cast<__nv_bfloat16*>(out));
+    SLED_LAUNCH_PDL(swiglu_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, partial, n_split, split_stride, F, static_cast<__nv_bfloat16*>(out));
   else
-    swiglu_kernel<<<grid, 256, 0, s>>>(partial, n_split, split_stride, F, static_cast<float*>(out));
+    SLED_LAUNCH_PDL(swiglu_kernel<float>, grid, dim3(256), 0, s, partial, n_split, split_stride, F, static_cast<float*>(out));
   return 1;
 }
 
@@ -218,6 +220,7 @@ template <typename AT, typename WT>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const AT* __restrict__ A, const WT* __restrict__ W, int T, int N,
                                                         int K, int k_per_split, float* __restrict__ out,
                                                         int64_t split_stride) {
+  pdl_enter();
   constexpr int BM = 32, BN = 64, BK = 32;
   __shared__ float As[BK][BM + 1];
   __shared__ float Ws[BK][BN + 1];
@@ -266,11 +269,12 @@ int launch_gemm_simt(const void* A, int adtype, const void* W, int wdtype, int T
   int k_per_split = ((K + n_split - 1) / n_split + 31) / 32 * 32;
   dim3 grid((N + 63) / 64, (T + 31) / 32, n_split);
   if (adtype == F32 && wdtype == F32)
-    gemm_simt_kernel<<<grid, 256, 0, s>>>(static_cast<const float*>(A), static_cast<const float*>(W), T, N, K,
-                                          k_per_split, out, split_stride);
+    SLED_LAUNCH_PDL((gemm_simt_kernel<float, float>), grid, dim3(256), 0, s, static_cast<const float*>(A),
+                    static_cast<const float*>(W), T, N, K, k_per_split, out, split_stride);
   else if (adtype == BF16 && wdtype == BF16)
-    gemm_simt_kernel<<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(A), static_cast<const __nv_bfloat16*>(W), T,
-                                          N, K, k_per_split, out, split_stride);
+    SLED_LAUNCH_PDL((gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16>), grid, dim3(256), 0, s,
+                    static_cast<const __nv_bfloat16*>(A), static_cast<const __nv_bfloat16*>(W), T, N, K, k_per_split, out,
+                    split_stride);
   else
     return -1;
   return 1;
