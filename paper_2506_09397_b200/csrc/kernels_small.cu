@@ -34,27 +34,37 @@ template <typename WT, typename AT>
 __global__ void add_rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ partial, int n_split,
                                    int64_t split_stride, const WT* __restrict__ gain, float eps, int d,
                                    AT* __restrict__ out) {
-  pdl_enter();
   __shared__ float scratch[32];
+  pdl_enter();
   const int64_t base = static_cast<int64_t>(blockIdx.x) * d;
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = x[base + i];
-    for (int sp = 0; sp < n_split; ++sp) v += partial[sp * split_stride + base + i];
-    if (n_split > 0) x[base + i] = v;
-    ss += v * v;
+  // four consecutive features per thread and pass; the slices of a feature are summed in slice order
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    float4 v = *reinterpret_cast<const float4*>(x + base + i);
+#pragma unroll 8
+    for (int sp = 0; sp < n_split; ++sp) {
+      const float4 p = __ldcg(reinterpret_cast<const float4*>(partial + sp * split_stride + base + i));
+      v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+    }
+    if (n_split > 0) *reinterpret_cast<float4*>(x + base + i) = v;
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = block_sum(ss, scratch);
   const float scale = rsqrtf(ss / static_cast<float>(d) + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x)  // each thread re-reads what it wrote itself
-    out[base + i] = from_f32<AT>(x[base + i] * scale * to_f32(gain[i]));
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {  // each thread re-reads what it wrote itself
+    const float4 v = *reinterpret_cast<const float4*>(x + base + i);
+    out[base + i] = from_f32<AT>(v.x * scale * to_f32(gain[i]));
+    out[base + i + 1] = from_f32<AT>(v.y * scale * to_f32(gain[i + 1]));
+    out[base + i + 2] = from_f32<AT>(v.z * scale * to_f32(gain[i + 2]));
+    out[base + i + 3] = from_f32<AT>(v.w * scale * to_f32(gain[i + 3]));
+  }
 }
 
 int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t split_stride, const void* gain, int wdtype,
                        float eps, int T, int d, void* out, int adtype, cudaStream_t s) {
   if (T <= 0) return 0;
   if (!partial) n_split = 0;
-  const int nt = d >= 2048 ? 512 : 256;
+  const int nt = d >= 4096 ? 1024 : (d >= 2048 ? 512 : 256);   // d is a multiple of 8 (checked at init)
   if (wdtype == BF16 && adtype == BF16)
     SLED_LAUNCH_PDL((add_rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16>), dim3(T), dim3(nt), 0, s, x, partial, n_split,
                     split_stride, static_cast<const __nv_bfloat16*>(gain), eps, d, static_cast<__nv_bfloat16*>(out));
@@ -98,8 +108,9 @@ __global__ void rope_kv_kernel(const float* __restrict__ partial, int n_split, i
   const int n_cols = (Hq + 2 * Hkv) * h;
   const int64_t src = static_cast<int64_t>(t) * n_cols + head * h + 2 * i;
   float a = 0.f, b = 0.f;
+#pragma unroll 8
   for (int sp = 0; sp < n_split; ++sp) {
-    const float2 v = *reinterpret_cast<const float2*>(partial + sp * split_stride + src);
+    const float2 v = __ldcg(reinterpret_cast<const float2*>(partial + sp * split_stride + src));
     a += v.x;
     b += v.y;
   }
