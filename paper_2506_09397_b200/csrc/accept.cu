@@ -1,7 +1,7 @@
 // Fused vocabulary softmax + speculative acceptance + corrective / bonus draw.
 //
-// One block per request walks its rows in order and stops at the deciding row: rows
-// behind the first rejection are never read.  All quantities that decide anything are
+// One block (or, for small batches, one thread-block cluster) per request walks its rows in
+// order and stops at the deciding row: rows behind the first rejection are never read.  All quantities that decide anything are
 // order-independent: the row maximum, integer softmax numerators E_v (a fixed sequence
 // of correctly rounded fp32 operations followed by an exact scaling to 2^40), their
 // exact 64-bit sum Z, and integer prefix sums for the inverse-CDF draw.  The accept test
@@ -74,10 +74,17 @@ __device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v
   return warp_sum_u64(t);
 }
 
+constexpr int kMaxCluster = 8;
+
 struct Shared {
   unsigned long long sum_scratch[32];
   unsigned long long tile_sum[kMaxTiles];
   unsigned long long warp_pref[32];
+  // exchange slots, one per CTA of the cluster (written by every CTA into every CTA's copy)
+  unsigned long long x_sum[2][kMaxCluster];   // Z, then W of the deciding row (double-buffered)
+  float x_max[2][kMaxCluster];                // row maximum (double-buffered over rows)
+  int x_idx[2][kMaxCluster];
+  int x_bad[2][kMaxCluster];
   float max_scratch[32];
   int idx_scratch[32];
   int flag;
@@ -85,16 +92,34 @@ struct Shared {
   int pick;
 };
 
-__global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, int rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// One cluster of C blocks per request; block `rank` owns a contiguous run of 4096-entry vocabulary tiles.
+// Per examined row the blocks exchange (maximum, argmax, finiteness), then the integer sums, through
+// each other's shared memory; every block then takes the same decision from the same numbers.
+__global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a, int C) {
   __shared__ Shared sh;
   pdl_enter();
-  const int req = blockIdx.x;
+  const int req = blockIdx.x / C, rank = blockIdx.x % C;
   const int row0 = a.cu_q[req];
   const int k = a.cu_q[req + 1] - row0 - 1;
   const int V = a.V;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float* qbase = a.q_rows ? a.q_rows[req] : nullptr;
   int32_t* res = a.results + 3 * req;
+  const int n_tiles = (V + kTile - 1) / kTile;
+  const int tiles_per_rank = (n_tiles + C - 1) / C;
+  const int tl_lo = min(n_tiles, rank * tiles_per_rank), tl_hi = min(n_tiles, tl_lo + tiles_per_rank);
+  const int v_lo = tl_lo * kTile, v_hi = min(V, tl_hi * kTile);   // this block's vocabulary range
+  int xphase = 0;   // parity of the sum exchange slots
 
   for (int j = 0; j <= k; ++j) {
     const float* z = a.logits + static_cast<int64_t>(row0 + j) * V;
@@ -102,7 +127,7 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
     float best = -INFINITY;
     int best_i = 0x7fffffff;
     int bad = 0;
-    for (int v = threadIdx.x; v < V; v += kThreads) {
+    for (int v = v_lo + threadIdx.x; v < v_hi; v += kThreads) {
       const float x = z[v];
       bad |= !(fabsf(x) < INFINITY);
       const float sv = a.greedy ? x : __fmul_rn(x, a.inv_tau);
@@ -117,10 +142,6 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
     bad = __syncthreads_or(bad);
     if (lane == 0) { sh.max_scratch[warp] = best; sh.idx_scratch[warp] = best_i; }
     __syncthreads();
-    if (bad) {
-      if (threadIdx.x == 0) { res[0] = 0; res[1] = -1; res[2] = ST_NONFINITE; }
-      return;
-    }
     best = sh.max_scratch[0];
     best_i = sh.idx_scratch[0];
     for (int w = 1; w < kThreads / 32; ++w) {
@@ -128,17 +149,48 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
       const int oi = sh.idx_scratch[w];
       if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
     }
+    if (C > 1) {
+      const int pb = j & 1;
+      if (threadIdx.x < C) {   // thread r delivers this block's triple to block r
+        const int r = threadIdx.x;
+        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(map_to_rank(smem_addr(&sh.x_max[pb][rank]), r)), "f"(best) : "memory");
+        asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(map_to_rank(smem_addr(&sh.x_idx[pb][rank]), r)), "r"(best_i) : "memory");
+        asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(map_to_rank(smem_addr(&sh.x_bad[pb][rank]), r)), "r"(bad) : "memory");
+      }
+      cluster_barrier();
+      best = sh.x_max[pb][0];
+      best_i = sh.x_idx[pb][0];
+      bad = sh.x_bad[pb][0];
+      for (int r = 1; r < C; ++r) {
+        const float ob = sh.x_max[pb][r];
+        const int oi = sh.x_idx[pb][r];
+        bad |= sh.x_bad[pb][r];
+        if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
+      }
+    }
+    if (bad) {
+      if (threadIdx.x == 0 && rank == 0) { res[0] = 0; res[1] = -1; res[2] = ST_NONFINITE; }
+      return;
+    }
     if (a.greedy) {
       if (j < k && a.ids[row0 + 1 + j] == best_i) continue;
-      if (threadIdx.x == 0) { res[0] = j; res[1] = best_i; res[2] = ST_OK; }
+      if (threadIdx.x == 0 && rank == 0) { res[0] = j; res[1] = best_i; res[2] = ST_OK; }
       return;
     }
     const float m = best;
     // ---- pass 2: Z = sum of the integer numerators
     unsigned long long zsum = 0;
-    for (int v = threadIdx.x; v < V; v += kThreads) zsum += fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
-    const unsigned long long Z = block_sum_u64(zsum, sh.sum_scratch);
-    // ---- the accept test of draft j+1, or fall through on the bonus row
+    for (int v = v_lo + threadIdx.x; v < v_hi; v += kThreads) zsum += fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
+    unsigned long long Z = block_sum_u64(zsum, sh.sum_scratch);
+    if (C > 1) {
+      if (threadIdx.x < C)
+        asm volatile("st.shared::cluster.b64 [%0], %1;" ::"r"(map_to_rank(smem_addr(&sh.x_sum[xphase][rank]), threadIdx.x)), "l"(Z) : "memory");
+      cluster_barrier();
+      Z = 0;
+      for (int r = 0; r < C; ++r) Z += sh.x_sum[xphase][r];
+      xphase ^= 1;
+    }
+    // ---- the accept test of draft j+1, or fall through on the bonus row (same numbers in every block)
     const float* qrow = nullptr;
     uint32_t u_smp = 0;
     if (threadIdx.x == 0) {
@@ -164,14 +216,13 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
     if (j < k) qrow = qbase + static_cast<int64_t>(j) * V;
 
     // ---- deciding row: weights R_v = max(E_v - trunc(q_v * Z), 0) (or E_v), tile sums in vocabulary order
-    const int n_tiles = (V + kTile - 1) / kTile;
     const double Zd = __ull2double_rn(Z);
     bool use_q = qrow != nullptr;
-    unsigned long long W = 0;
+    unsigned long long W = 0, before_me = 0;
     for (int attempt = 0; attempt < 2; ++attempt) {
       for (int tl = threadIdx.x; tl < n_tiles; tl += kThreads) sh.tile_sum[tl] = 0ull;
       __syncthreads();
-      for (int tl = 0; tl < n_tiles; ++tl) {
+      for (int tl = tl_lo; tl < tl_hi; ++tl) {
         unsigned long long mine = 0;
         const int v0 = tl * kTile + threadIdx.x * kVec;
 #pragma unroll
@@ -190,21 +241,37 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
         if (lane == 0 && mine) atomicAdd(&sh.tile_sum[tl], mine);  // integer adds: any order, same sum
       }
       __syncthreads();
-      W = 0;
-      for (int tl = 0; tl < n_tiles; ++tl) W += sh.tile_sum[tl];
+      unsigned long long mine_w = 0;
+      for (int tl = tl_lo; tl < tl_hi; ++tl) mine_w += sh.tile_sum[tl];
+      W = mine_w;
+      before_me = 0;
+      if (C > 1) {
+        if (threadIdx.x < C)
+          asm volatile("st.shared::cluster.b64 [%0], %1;" ::"r"(map_to_rank(smem_addr(&sh.x_sum[xphase][rank]), threadIdx.x)), "l"(mine_w) : "memory");
+        cluster_barrier();
+        W = 0;
+        for (int r = 0; r < C; ++r) {
+          if (r < rank) before_me += sh.x_sum[xphase][r];
+          W += sh.x_sum[xphase][r];
+        }
+        xphase ^= 1;
+      }
       if (W != 0 || !use_q) break;
       use_q = false;   // residual mass zero (p <= q everywhere after rounding): draw from p itself
       __syncthreads();
     }
     // ---- inverse CDF: tgt = (U' * W) >> 32, first v whose running sum exceeds tgt
     const unsigned long long tgt = __umul64hi(W, static_cast<unsigned long long>(u_smp) << 32);
-    int tl_hit = 0;
-    unsigned long long before = 0;
-    for (int tl = 0; tl < n_tiles; ++tl) {
+    unsigned long long my_w = 0;
+    for (int tl = tl_lo; tl < tl_hi; ++tl) my_w += sh.tile_sum[tl];
+    if (!(before_me <= tgt && tgt < before_me + my_w)) return;   // the crossing lies in another block's range
+    int tl_hit = tl_lo;
+    unsigned long long before = before_me;
+    for (int tl = tl_lo; tl < tl_hi; ++tl) {
       const unsigned long long nx = before + sh.tile_sum[tl];
       if (nx > tgt) { tl_hit = tl; break; }
       before = nx;
-      tl_hit = tl;  // only left at the last tile if nothing exceeded (cannot happen for W > 0)
+      tl_hit = tl;
     }
     unsigned long long r[kVec];
     unsigned long long mine = 0;
@@ -259,8 +326,24 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a) {
 int launch_accept(const AcceptArgs& a, cudaStream_t s) {
   if (a.B <= 0) return 0;
   if (a.V > kTile * kMaxTiles) return -1;
-  SLED_LAUNCH_PDL(accept_kernel, dim3(a.B), dim3(kThreads), 0, s, a);
-  return 1;
+  // blocks per request: enough to occupy the machine when the batch is small
+  int C = 1;
+  while (C < kMaxCluster && a.B * C < 128 && (a.V + kTile - 1) / kTile >= 2 * C) C *= 2;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(a.B * C, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, accept_kernel, a, C) == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace sled
