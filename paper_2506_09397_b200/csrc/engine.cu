@@ -159,7 +159,8 @@ int linear_split(const sled_engine* e, int T, const Linear& L) {
 }
 
 // out partial sums [split][T][N] into e->partial (or into `dst` when given, then split must be 1)
-int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Linear& L, int T, float* dst, int* split_out) {
+int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Linear& L, int T, float* dst, int* split_out,
+               const TcEpilogue& epi = TcEpilogue()) {
   int split = dst ? 1 : linear_split(e, T, L);
   float* out = dst ? dst : e->partial;
   const int64_t stride = static_cast<int64_t>(T) * L.N;
@@ -167,7 +168,7 @@ int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Lin
   e->mark(K_LINEAR);
   int n;
   if (e->cfg.weight_dtype == SLED_BF16)
-    n = tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_ws, e->tc_error, e->n_sm, e->stream);
+    n = tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_ws, e->tc_error, e->n_sm, epi, e->stream);
   else
     n = launch_gemm_simt(A, e->adtype(), L.w, e->cfg.weight_dtype, T, L.N, L.K, split, out, stride, e->stream);
   if (n < 0) return SLED_ERR_DEVICE;
@@ -361,11 +362,21 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
                            e->stream);
     e->count(n, K_OTHER);
     int s_gu;
-    rc = run_linear(e, e->act_norm, &e->tc_norm, L.gate_up, T, nullptr, &s_gu);
-    if (rc) return rc;
-    e->mark(K_OTHER);
-    n = launch_swiglu(e->partial, s_gu, static_cast<int64_t>(T) * L.gate_up.N, T, c.ffn_dim, e->act_ffn, ad, e->stream);
-    e->count(n, K_OTHER);
+    if (c.weight_dtype == SLED_BF16 && linear_split(e, T, L.gate_up) == 1) {
+      // the whole sum is formed in one place: SwiGLU is applied there, act_ffn comes straight out of the GEMM
+      TcEpilogue epi;
+      epi.mode = kEpiSwiglu;
+      epi.act_out = static_cast<__nv_bfloat16*>(e->act_ffn);
+      epi.act_ld = c.ffn_dim;
+      rc = run_linear(e, e->act_norm, &e->tc_norm, L.gate_up, T, nullptr, &s_gu, epi);
+      if (rc) return rc;
+    } else {
+      rc = run_linear(e, e->act_norm, &e->tc_norm, L.gate_up, T, nullptr, &s_gu);
+      if (rc) return rc;
+      e->mark(K_OTHER);
+      n = launch_swiglu(e->partial, s_gu, static_cast<int64_t>(T) * L.gate_up.N, T, c.ffn_dim, e->act_ffn, ad, e->stream);
+      e->count(n, K_OTHER);
+    }
     rc = run_linear(e, e->act_ffn, &e->tc_ffn, L.down, T, nullptr, &split);
     if (rc) return rc;
     stride = static_cast<int64_t>(T) * L.down.N;
@@ -478,6 +489,21 @@ int make_linear(sled_engine* e, Linear* L, std::initializer_list<std::pair<const
   return SLED_OK;
 }
 
+// gate and up projections as one matrix with their rows interleaved (row 2f = gate f, row 2f+1 = up f),
+// so that a pair sits in neighbouring rows of an output tile and SwiGLU can be applied where the sums end up
+int make_gate_up(sled_engine* e, Linear* L, const void* gate, const void* up, int F, int K) {
+  if (!gate || !up) return SLED_ERR_ARG;
+  const size_t row = static_cast<size_t>(K) * dtype_size(e->cfg.weight_dtype);
+  int rc = dmalloc(e, &L->w, 2 * static_cast<size_t>(F) * row);
+  if (rc) return rc;
+  CU_TRY(cudaMemcpy2D(L->w, 2 * row, gate, row, row, F, cudaMemcpyDefault));
+  CU_TRY(cudaMemcpy2D(static_cast<char*>(L->w) + row, 2 * row, up, row, row, F, cudaMemcpyDefault));
+  L->N = 2 * F;
+  L->K = K;
+  if (e->cfg.weight_dtype == SLED_BF16 && tc_weight_init(&L->tc, L->w, L->N, K) != 0) return SLED_ERR_ARG;
+  return SLED_OK;
+}
+
 int check_cfg(const sled_config& c) {
   if (c.n_layers <= 0 || c.d_model <= 0 || c.n_q_heads <= 0 || c.n_kv_heads <= 0 || c.head_dim <= 0 || c.ffn_dim <= 0 ||
       c.vocab <= 0)
@@ -565,7 +591,7 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
     if ((rc = upload(e, w->ffn_norm[l], d * es, &L.ffn_norm))) return fail(rc);
     if ((rc = make_linear(e, &L.qkv, {{w->wq[l], qd}, {w->wk[l], kd}, {w->wv[l], kd}}, d))) return fail(rc);
     if ((rc = make_linear(e, &L.o, {{w->wo[l], d}}, qd))) return fail(rc);
-    if ((rc = make_linear(e, &L.gate_up, {{w->w_gate[l], F}, {w->w_up[l], F}}, d))) return fail(rc);
+    if ((rc = make_gate_up(e, &L.gate_up, w->w_gate[l], w->w_up[l], F, d))) return fail(rc);
     if ((rc = make_linear(e, &L.down, {{w->w_down[l], d}}, F))) return fail(rc);
   }
 

@@ -99,7 +99,38 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 
 
+// What the epilogue does with a finished 16-token run of one output row n:
+//   kEpiStore : out[t][n] = value
+//   kEpiSwiglu: rows come in (gate, up) pairs (2f, 2f+1); act[t][f] = silu(gate) * up as bf16
+__device__ __forceinline__ void emit16(const TcEpilogue& e, float* out, int N, int T, int n, int t_first, const float (&val)[16]) {
+  if (e.mode == kEpiSwiglu) {
+    // lane pairs (gate, up) -> one value per even lane; two neighbouring results are packed so that
+    // every fourth lane writes one 4-byte bf16 pair
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float other = __shfl_xor_sync(0xffffffffu, val[i], 1);   // the up value sits in the next lane
+      const float gate = val[i];
+      const float r = __fdividef(gate, 1.f + __expf(-gate)) * other;
+      const float r2 = __shfl_down_sync(0xffffffffu, r, 2);          // result of the next (gate, up) pair
+      const int t = t_first + i;
+      if ((n & 3) == 0 && n + 3 < N && t < T) {
+        __nv_bfloat162 pr = __floats2bfloat162_rn(r, r2);
+        *reinterpret_cast<__nv_bfloat162*>(e.act_out + static_cast<long long>(t) * e.act_ld + (n >> 1)) = pr;
+      } else if ((n & 3) == 0 && n < N && t < T) {
+        e.act_out[static_cast<long long>(t) * e.act_ld + (n >> 1)] = __float2bfloat16_rn(r);
+      }
+    }
+  } else if (n < N) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int t = t_first + i;
+      if (t < T) out[static_cast<long long>(t) * N + n] = val[i];
+    }
+  }
+}
+
 struct GemmArgs {
+  TcEpilogue epi;
   int T, N, kb_total, m_tiles, t_tiles;
   float* out;        // [T][N]
   float* ws;         // partial tiles: [2 * gridDim.x][TN_MAX][128]
@@ -273,13 +304,10 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
             : "r"(acc + static_cast<uint32_t>(c0)));
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (whole) {
-          if (n < g.N) {
+          float val[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const int t = t0 + c0 + i;
-              if (t < g.T) g.out[static_cast<long long>(t) * g.N + n] = __uint_as_float(v[i]);
-            }
-          }
+          for (int i = 0; i < 16; ++i) val[i] = __uint_as_float(v[i]);
+          emit16(g.epi, g.out, g.N, g.T, n, t0 + c0, val);
         } else {
 #pragma unroll
           for (int i = 0; i < 16; ++i) __stcg(part + (c0 + i) * 128 + row, __uint_as_float(v[i]));
@@ -313,13 +341,7 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
 #pragma unroll
               for (int j = 0; j < 16; ++j) sum[j] += __ldcg(src + j * 128);
             }
-            if (n < g.N) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const int t = t0 + c0 + j;
-                if (t < g.T) g.out[static_cast<long long>(t) * g.N + n] = sum[j];
-              }
-            }
+            emit16(g.epi, g.out, g.N, g.T, n, t0 + c0, sum);
           }
           if (warp == 2 && lane == 0) g.counters[tile] = 0;   // ready for the next launch
         }
@@ -361,7 +383,7 @@ template <int TN_MAX, int STAGES>
 __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constant__ CUtensorMap map_w,
                                                        const __grid_constant__ CUtensorMap map_a, int T, int N,
                                                        int kb_total, int kb_per_split, float* __restrict__ out,
-                                                       long long split_stride, int32_t* error) {
+                                                       long long split_stride, int32_t* error, TcEpilogue epi) {
   using L = SplitSmemLayout<TN_MAX, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -453,7 +475,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int n = m_tile * kBlockM + quad * 32 + lane;
-      float* dst = out + static_cast<long long>(split) * split_stride + n;
+      float* dst = out + static_cast<long long>(split) * split_stride;
       for (int c0 = 0; c0 < tn; c0 += 16) {
         uint32_t v[16];
         if (nkb > 0) {
@@ -467,13 +489,10 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
 #pragma unroll
           for (int i = 0; i < 16; ++i) v[i] = 0u;
         }
-        if (n < N) {
+        float val[16];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int t = t0 + c0 + i;
-            if (t < T) dst[static_cast<long long>(t) * N] = __uint_as_float(v[i]);
-          }
-        }
+        for (int i = 0; i < 16; ++i) val[i] = __uint_as_float(v[i]);
+        emit16(epi, dst, N, T, n, t0 + c0, val);
       }
     }
   }
@@ -530,7 +549,7 @@ int make_map(CUtensorMap* map, const void* ptr, long long rows, int K, int box_r
 
 template <int TN_MAX, int STAGES>
 int launch_one(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K, float* out, const TcWorkspace& wsp,
-               int32_t* error, int n_sm, cudaStream_t s) {
+               int32_t* error, int n_sm, const TcEpilogue& epi, cudaStream_t s) {
   using L = SmemLayout<TN_MAX, STAGES>;
   static bool configured = false;
   if (!configured) {
@@ -539,6 +558,7 @@ int launch_one(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K
     configured = true;
   }
   GemmArgs g{};
+  g.epi = epi;
   g.T = T;
   g.N = N;
   g.kb_total = (K + kBlockK - 1) / kBlockK;
@@ -625,7 +645,7 @@ int tc_gemm_split(int T, int N, int K, int n_sm) {
 
 template <int TN_MAX, int STAGES>
 static int launch_split(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K, int n_split, float* out,
-                        int64_t split_stride, int32_t* error, cudaStream_t s) {
+                        int64_t split_stride, int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
   using L = SplitSmemLayout<TN_MAX, STAGES>;
   static bool configured = false;
   if (!configured) {
@@ -646,17 +666,18 @@ static int launch_split(const CUtensorMap& mw, const CUtensorMap& ma, int T, int
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   const long long stride = split_stride;
-  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_split_kernel<TN_MAX, STAGES>, mw, ma, T, N, kb_total, kb_per, out, stride, error);
+  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_split_kernel<TN_MAX, STAGES>, mw, ma, T, N, kb_total, kb_per, out, stride, error, epi);
   return err == cudaSuccess ? 1 : -1;
 }
 
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
-                   const TcWorkspace& wsp, int32_t* error, int n_sm, cudaStream_t s) {
+                   const TcWorkspace& wsp, int32_t* error, int n_sm, const TcEpilogue& epi, cudaStream_t s) {
   if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
-  if (T <= 64) return launch_split<64, 4>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, s);
-  if (T <= 128) return launch_split<128, 3>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, s);
+  if (epi.mode != kEpiStore && n_split != 1) return -1;   // a fused epilogue needs the complete sum
+  if (T <= 64) return launch_split<64, 4>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (T <= 128) return launch_split<128, 3>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (n_split != 1) return -1;
-  return launch_one<256, 4>(w.map, a.map[2], T, w.N, w.K, out, wsp, error, n_sm, s);
+  return launch_one<256, 4>(w.map, a.map[2], T, w.N, w.K, out, wsp, error, n_sm, epi, s);
 }
 
 }  // namespace sled

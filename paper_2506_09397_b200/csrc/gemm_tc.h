@@ -3,6 +3,7 @@
 // side, operands brought to shared memory by TMA, fp32 accumulators in tensor memory.
 #pragma once
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -18,6 +19,13 @@ struct TcWeight {       // [N][K] bf16, row-major, device memory
 struct TcActivation {   // [rows][K] bf16, row-major, device memory; rows is a multiple of 256
   CUtensorMap map[3];   // boxes of 64 (k) x {64, 128, 256} rows
   int rows = 0, K = 0;
+};
+
+enum { kEpiStore = 0, kEpiSwiglu = 1 };
+struct TcEpilogue {       // what happens to the finished sums (see emit16 in gemm_tc.cu)
+  int mode = kEpiStore;
+  __nv_bfloat16* act_out = nullptr;   // kEpiSwiglu: [T][act_ld] activations for the down projection
+  int act_ld = 0;
 };
 
 struct TcWorkspace {    // shared by all linear layers of an engine (one launch at a time on its stream)
@@ -38,6 +46,6 @@ int tc_gemm_split(int T, int N, int K, int n_sm);
 // out[slice][T][N] = A[T][K slice] . W[N][K slice]^T; returns kernels launched (1) or a negative value;
 // `error` is a device word set if a bounded wait ran out
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
-                   const TcWorkspace& wsp, int32_t* error, int n_sm, cudaStream_t s);
+                   const TcWorkspace& wsp, int32_t* error, int n_sm, const TcEpilogue& epi, cudaStream_t s);
 
 }  // namespace sled

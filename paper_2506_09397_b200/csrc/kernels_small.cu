@@ -96,7 +96,7 @@ int launch_rope_table(const int32_t* tok_pos, int T, int h, float theta, float2*
 }
 
 // ------------------------------------------------------ RoPE + cache write --
-// grid (T, Hq + 2 Hkv), h/2 threads: thread i owns the pair (2i, 2i+1) of one head.
+// grid (T, (Hq + 2 Hkv) / 4), blocks of (h/2, 4) threads: thread (i, y) owns the pair (2i, 2i+1) of one head.
 // Cache layout of one layer: [page][Hkv][page_size][h]; slot = page * page_size + offset.
 template <typename AT, typename KT>
 __global__ void rope_kv_kernel(const float* __restrict__ partial, int n_split, int64_t split_stride,
@@ -104,7 +104,8 @@ __global__ void rope_kv_kernel(const float* __restrict__ partial, int n_split, i
                                int h, int page_size, AT* __restrict__ q_out, KT* __restrict__ kpool,
                                KT* __restrict__ vpool) {
   pdl_enter();
-  const int t = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
+  const int t = blockIdx.x, head = blockIdx.y * blockDim.y + threadIdx.y, i = threadIdx.x;
+  if (head >= Hq + 2 * Hkv) return;
   const int n_cols = (Hq + 2 * Hkv) * h;
   const int64_t src = static_cast<int64_t>(t) * n_cols + head * h + 2 * i;
   float a = 0.f, b = 0.f;
@@ -139,15 +140,15 @@ int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, cons
                    int T, int Hq, int Hkv, int h, int page_size, void* q_out, int adtype, void* kpool, void* vpool,
                    int kvdtype, cudaStream_t s) {
   if (T <= 0) return 0;
-  dim3 grid(T, Hq + 2 * Hkv);
+  dim3 grid(T, (Hq + 2 * Hkv + 3) / 4);
   if (adtype == BF16 && kvdtype == BF16)
-    SLED_LAUNCH_PDL((rope_kv_kernel<__nv_bfloat16, __nv_bfloat16>), grid, dim3(h / 2), 0, s, partial, n_split, split_stride, cs, tok_slot,
+    SLED_LAUNCH_PDL((rope_kv_kernel<__nv_bfloat16, __nv_bfloat16>), grid, dim3(h / 2, 4), 0, s, partial, n_split, split_stride, cs, tok_slot,
                     Hq, Hkv, h, page_size, static_cast<__nv_bfloat16*>(q_out), static_cast<__nv_bfloat16*>(kpool), static_cast<__nv_bfloat16*>(vpool));
   else if (adtype == F32 && kvdtype == F32)
-    SLED_LAUNCH_PDL((rope_kv_kernel<float, float>), grid, dim3(h / 2), 0, s, partial, n_split, split_stride, cs, tok_slot,
+    SLED_LAUNCH_PDL((rope_kv_kernel<float, float>), grid, dim3(h / 2, 4), 0, s, partial, n_split, split_stride, cs, tok_slot,
                     Hq, Hkv, h, page_size, static_cast<float*>(q_out), static_cast<float*>(kpool), static_cast<float*>(vpool));
   else if (adtype == F32 && kvdtype == BF16)
-    SLED_LAUNCH_PDL((rope_kv_kernel<float, __nv_bfloat16>), grid, dim3(h / 2), 0, s, partial, n_split, split_stride, cs, tok_slot,
+    SLED_LAUNCH_PDL((rope_kv_kernel<float, __nv_bfloat16>), grid, dim3(h / 2, 4), 0, s, partial, n_split, split_stride, cs, tok_slot,
                     Hq, Hkv, h, page_size, static_cast<float*>(q_out), static_cast<__nv_bfloat16*>(kpool), static_cast<__nv_bfloat16*>(vpool));
   else
     return -1;
@@ -155,7 +156,7 @@ int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, cons
 }
 
 // --------------------------------------------------------------------- SwiGLU --
-// partial: [split][T][2F], gate in columns [0, F), up in [F, 2F):  out = silu(gate) * up
+// partial: [split][T][2F], gate and up interleaved (columns 2f and 2f+1):  out = silu(gate) * up
 template <typename AT>
 __global__ void swiglu_kernel(const float* __restrict__ partial, int n_split, int64_t split_stride, int F,
                               AT* __restrict__ out) {
@@ -166,8 +167,9 @@ __global__ void swiglu_kernel(const float* __restrict__ partial, int n_split, in
   const int64_t row = static_cast<int64_t>(t) * 2 * F;
   float g = 0.f, u = 0.f;
   for (int sp = 0; sp < n_split; ++sp) {
-    g += partial[sp * split_stride + row + f];
-    u += partial[sp * split_stride + row + F + f];
+    const float2 gu = __ldcg(reinterpret_cast<const float2*>(partial + sp * split_stride + row + 2 * f));
+    g += gu.x;
+    u += gu.y;
   }
   out[static_cast<int64_t>(t) * F + f] = from_f32<AT>(g / (1.f + __expf(-g)) * u);
 }
