@@ -158,6 +158,50 @@ def test_synthetic_cache_and_long_context_split():
     eng.shutdown()
 
 
+def test_large_step_uses_several_token_tiles():
+    # more than 256 tokens in one step: the linear layers run as several token tiles per weight tile
+    # (and tiles shared between blocks); a long prefill chunk goes the same way
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=4)
+    eng = _engine(shape, w, n_pages=600, max_batch=40, max_k=8, max_step_tokens=400)
+    orc = O.OracleModel(shape, oracle_weights(w))
+    ctxs = list(range(40))
+    for c in ctxs:
+        n = 3 + (7 * c) % 29
+        p = I.make_prompt(shape.vocab, n, 4, c)
+        eng.prefill(c, p)
+        if c % 9 == 0:
+            orc.prefill(c, p)
+    reqs = []
+    for c in ctxs:
+        d, q = I.make_drafts(shape.vocab, 8 if c % 3 else 5, 4, c)
+        reqs.append((c, d, q))
+    T = sum(len(d) + 1 for _, d, _ in reqs)
+    assert T > 256
+    eng.set_commit(False)
+    got = eng.verify_batch([(c, d.numpy(), q.numpy()) for c, d, q in reqs], 9)
+    glog = eng.logits(T)
+    row = 0
+    for (c, d, q), g in zip(reqs, got):
+        k = len(d)
+        if c in orc.ctx:
+            st, n_acc, nxt, ol, mg = orc.verify(c, d.numpy(), q.numpy(), 9, commit=False)
+            assert np.max(np.abs(glog[row:row + k + 1] - ol)) <= 2e-2
+            st2, n2, x2, _ = O.accept(glog[row:row + k + 1], q.numpy(), d.numpy(), 1.0, False, 9, c, orc.ctx[c].n_kv)
+            assert (n2, x2, 0) == g
+        row += k + 1
+    # a prompt longer than one step: prefilled in chunks of max_step_tokens (> 256 tokens per chunk)
+    long_prompt = I.make_prompt(shape.vocab, 700, 4, 99)
+    eng.prefill(99, long_prompt)
+    orc.prefill(99, long_prompt)
+    K, V = eng.read_kv(99, shape.n_layers - 1, 699)
+    assert np.max(np.abs(K.float().numpy() - orc.ctx[99].K[shape.n_layers - 1, :699])) <= 2e-2
+    d, q = I.make_drafts(shape.vocab, 4, 4, 99)
+    eng.set_commit(True)
+    _verify_both(eng, orc, [(99, d, q)], seed=2, tau=1.0, greedy=False, tol=2e-2, explain=[])
+    eng.shutdown()
+
+
 def test_errors_leave_everything_unchanged():
     shape = I.TINY
     w = I.make_weights(shape, seed=0)
