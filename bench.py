@@ -264,6 +264,8 @@ def run_sled(args):
             raise SystemExit(f"sled_verify_batch failed: {B.strerror(rc)}")
         committed = 0
         for i in range(Bn):
+            if res[i].status != 0:
+                raise SystemExit(f"request {i} came back with status {res[i].status}")
             committed += res[i].n_accepted + 1
             L.sled_debug_truncate(eng.h, i, ctx[i], 1)   # same state for every step (host bookkeeping only)
         return committed

@@ -14,7 +14,9 @@
  * engine handle.  Unless a parameter says otherwise a pointer is a HOST pointer.
  * Every function returns SLED_OK (0) or a negative sled_status; a failed call
  * changes no context, page or counter.  An engine is used by one thread at a
- * time.  All device work is issued on the engine's stream.
+ * time.  All device work is issued on the engine's stream, which does not wait for
+ * any other stream: a DEVICE pointer passed in must refer to data that is already
+ * complete (synchronise the stream that produced it first).
  */
 #ifndef SLED_H_
 #define SLED_H_

@@ -75,7 +75,7 @@ def lib():
                                  C.POINTER(Margin)]
         L.orc_accept.restype = C.c_int
         L.orc_forward_token.argtypes = [C.POINTER(_Cfg), C.POINTER(_Weights), C.c_int32, C.c_int64, C.c_void_p,
-                                        C.c_void_p, C.c_int64, C.c_void_p]
+                                        C.c_void_p, C.c_int64, C.c_void_p, C.c_int32]
         L.orc_forward_token.restype = C.c_int
         L.orc_attend_one.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p]
         L.orc_attend_one.restype = None
@@ -176,9 +176,11 @@ class Context:
 class OracleModel:
     """Target model + per-context caches, driven one token at a time."""
 
-    def __init__(self, shape, weights: dict):
-        """shape: any object with the config attributes; weights: name -> array (per-layer names -> list)."""
+    def __init__(self, shape, weights: dict, round_acts: bool = False):
+        """shape: any object with the config attributes; weights: name -> array (per-layer names -> list).
+        round_acts: the separately reported mode that rounds matrix-product inputs to bf16 (see the C++ file)."""
         self.shape = shape
+        self.round_acts = int(bool(round_acts))
         wd = 1 if shape.weight_dtype == "bf16" else 0
         kd = 1 if shape.kv_dtype == "bf16" else 0
         self.cfg = _Cfg(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
@@ -212,7 +214,7 @@ class OracleModel:
         self._grow(c, pos + 1)
         out = np.empty(self.shape.vocab, dtype=np.float32)
         rc = lib().orc_forward_token(C.byref(self.cfg), C.byref(self.w), int(token), int(pos), c.K.ctypes.data,
-                                     c.V.ctypes.data, c.K.shape[1], out.ctypes.data)
+                                     c.V.ctypes.data, c.K.shape[1], out.ctypes.data, self.round_acts)
         assert rc == 0
         return out
 

@@ -316,12 +316,22 @@ static void rope(double* v, int n_heads, int h, int64_t pos, double theta) {
     }
 }
 
+static void round_vec(double* v, int64_t n) {
+  for (int64_t i = 0; i < n; ++i) v[i] = static_cast<double>(round_to_bf16(v[i]));
+}
+
 // One token through the whole model.  kcache / vcache: [n_layers][cap][Hkv][h]
 // floats holding values already rounded to the cache format, rows 0..pos-1
 // filled; row pos is written here.  logits_out: [vocab] fp32.
 // Returns 0, or -1 if pos >= cap.
+//
+// round_acts = 0 is the reference evaluation.  round_acts = 1 is a second, separately reported mode for
+// the 16-bit configurations: every vector that a 16-bit implementation has to hand to a matrix product
+// in 16 bits (the two normalised inputs of a layer, the rotated query, the attention output, the SwiGLU
+// output, the final normalised vector) is rounded to bf16 at that point and nowhere else.  Comparing
+// against it separates rounding of the activations, which grows with depth, from everything else.
 int orc_forward_token(const orc_config* cfg, const orc_weights* w, int32_t token, int64_t pos,
-                      float* kcache, float* vcache, int64_t cap, float* logits_out) {
+                      float* kcache, float* vcache, int64_t cap, float* logits_out, int32_t round_acts) {
   const int L = cfg->n_layers, d = cfg->d_model, Hq = cfg->n_q_heads, Hkv = cfg->n_kv_heads;
   const int h = cfg->head_dim, F = cfg->ffn_dim, V = cfg->vocab, wd = cfg->weight_dtype;
   if (pos >= cap || pos < 0) return -1;
@@ -333,11 +343,13 @@ int orc_forward_token(const orc_config* cfg, const orc_weights* w, int32_t token
   const int64_t layer_stride = cap * Hkv * h;
   for (int l = 0; l < L; ++l) {
     rmsnorm(x.data(), Tensor{w->attn_norm[l], wd}, d, cfg->rms_eps, a.data());
+    if (round_acts) round_vec(a.data(), d);
     matvec(Tensor{w->wq[l], wd}, static_cast<int64_t>(Hq) * h, d, a.data(), qv.data());
     matvec(Tensor{w->wk[l], wd}, static_cast<int64_t>(Hkv) * h, d, a.data(), kv.data());
     matvec(Tensor{w->wv[l], wd}, static_cast<int64_t>(Hkv) * h, d, a.data(), vv.data());
     rope(qv.data(), Hq, h, pos, cfg->rope_theta);
     rope(kv.data(), Hkv, h, pos, cfg->rope_theta);
+    if (round_acts) round_vec(qv.data(), static_cast<int64_t>(Hq) * h);
     float* kc = kcache + l * layer_stride;
     float* vc = vcache + l * layer_stride;
     for (int i = 0; i < Hkv * h; ++i) {
@@ -365,16 +377,20 @@ int orc_forward_token(const orc_config* cfg, const orc_weights* w, int32_t token
         o[static_cast<size_t>(hd) * h + i] = acc / den;
       }
     }
+    if (round_acts) round_vec(o.data(), static_cast<int64_t>(Hq) * h);
     matvec(Tensor{w->wo[l], wd}, d, static_cast<int64_t>(Hq) * h, o.data(), tmp.data());
     for (int i = 0; i < d; ++i) x[i] += tmp[i];
     rmsnorm(x.data(), Tensor{w->ffn_norm[l], wd}, d, cfg->rms_eps, a.data());
+    if (round_acts) round_vec(a.data(), d);
     matvec(Tensor{w->w_gate[l], wd}, F, d, a.data(), g.data());
     matvec(Tensor{w->w_up[l], wd}, F, d, a.data(), u.data());
     for (int i = 0; i < F; ++i) g[i] = (g[i] / (1.0 + std::exp(-g[i]))) * u[i];
+    if (round_acts) round_vec(g.data(), F);
     matvec(Tensor{w->w_down[l], wd}, d, F, g.data(), tmp.data());
     for (int i = 0; i < d; ++i) x[i] += tmp[i];
   }
   rmsnorm(x.data(), Tensor{w->final_norm, wd}, d, cfg->rms_eps, a.data());
+  if (round_acts) round_vec(a.data(), d);
   std::vector<double> lg(static_cast<size_t>(V));
   matvec(Tensor{w->lm_head, wd}, V, d, a.data(), lg.data());
   for (int v = 0; v < V; ++v) logits_out[v] = static_cast<float>(lg[v]);

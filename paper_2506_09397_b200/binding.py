@@ -127,6 +127,13 @@ def _check(code: int, what: str) -> None:
         raise SledError(code, what)
 
 
+def _settle(*tensors) -> None:
+    """The library works on its own stream and does not wait for anybody else's: device tensors handed to
+    it must be complete.  Torch fills them asynchronously on its current stream, so that stream is drained."""
+    if any(isinstance(t, torch.Tensor) and t.is_cuda for t in tensors):
+        torch.cuda.current_stream().synchronize()
+
+
 def _addr(t) -> int:
     if t is None:
         return 0
@@ -160,6 +167,7 @@ class Engine:
             keep.append(arr)
             setattr(w, name, C.cast(arr, C.POINTER(C.c_void_p)))
         h = C.c_void_p()
+        _settle(weights["tok_emb"])
         _check(lib().sled_init(C.byref(w), C.byref(cfg), C.byref(h)), "sled_init")
         self.h = h
         self.cfg = cfg
@@ -170,6 +178,7 @@ class Engine:
         """requests: list of (ctx_id, draft_tokens int32 host array [k], draft_probs [k, V] fp32 or None).
         Returns list of (n_accepted, next_token, status)."""
         n = len(requests)
+        _settle(*[r[2] for r in requests])
         reqs = (SledRequest * max(n, 1))()
         keep = []
         for i, (ctx, toks, probs) in enumerate(requests):
@@ -211,6 +220,7 @@ class Engine:
 
     def load_kv(self, ctx_id: int, K, V, pending: int) -> None:
         n = K.shape[1]
+        _settle(K, V)
         _check(lib().sled_debug_load_kv(self.h, ctx_id, _addr(K), _addr(V), n, pending), "sled_debug_load_kv")
 
     def read_kv(self, ctx_id: int, layer: int, n_tokens: int):
@@ -251,6 +261,7 @@ class Engine:
         ids = np.ascontiguousarray(np.asarray(ctx_ids, dtype=np.uint64))
         ql = np.ascontiguousarray(np.asarray(q_len, dtype=np.int32))
         ms = C.c_float()
+        _settle(q, out)
         _check(lib().sled_attention_ragged(self.h, layer, ids.ctypes.data, ql.ctypes.data, ids.size, q.data_ptr(),
                                            out.data_ptr(), C.byref(ms)), "sled_attention_ragged")
         return ms.value
@@ -278,6 +289,7 @@ def accept_rows(logits: torch.Tensor, cu_rows, drafts, q_rows, ctx_ids, pos0, te
     p0 = np.ascontiguousarray(np.asarray(pos0, dtype=np.int64))
     res = (SledResult * n)()
     ms = C.c_float()
+    _settle(logits, q_rows)
     _check(lib().sled_accept_rows(logits.data_ptr(), cu.ctypes.data, d.ctypes.data if d.size else None,
                                   _addr(q_rows) if q_rows is not None else None, ids.ctypes.data, p0.ctypes.data, n,
                                   logits.shape[1], temperature, int(greedy), seed, res, stream, C.byref(ms)),
@@ -296,6 +308,7 @@ def accept_rows_static(logits: torch.Tensor, cu_rows, drafts, q_rows, ctx_ids, p
     ids = np.ascontiguousarray(np.asarray(ctx_ids, dtype=np.uint64))
     p0 = np.ascontiguousarray(np.asarray(pos0, dtype=np.int64))
     res = (SledResult * max(n, 1))()
+    _settle(logits, q_rows)
     _check(lib().sled_accept_rows_static(logits.data_ptr(), cu.ctypes.data, d.ctypes.data if d.size else None,
                                          _addr(q_rows) if q_rows is not None else None, ids.ctypes.data,
                                          p0.ctypes.data, n, logits.shape[1], temperature, int(greedy), seed, res,

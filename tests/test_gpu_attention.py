@@ -45,8 +45,8 @@ def test_ragged_attention_matches_oracle(h, hq, hkv, kv):
             for head in rng.choice(hq, size=3, replace=False):
                 kvh = head // (hq // hkv)
                 ref = O.attend_one(q[t + j, head].float().numpy(), Ks[i][:n_vis, kvh], Vs[i][:n_vis, kvh])
-                worst = max(worst, float(np.max(np.abs(out[t + j, head] - ref))))
+                worst = max(worst, float(np.max(np.abs(out[t + j, head] - ref)) / max(1e-2, float(np.abs(ref).max()))))
         t += ql
-    # outputs are O(1/sqrt(n)) .. O(1); bf16 output rounding is 2^-9 relative
-    assert worst <= (2e-2 if kv == "bf16" else 1e-5), worst
+    # error relative to the size of the output row: bf16 output and probability rounding is 2^-9 relative
+    assert worst <= (1e-2 if kv == "bf16" else 2e-5), worst
     eng.shutdown()
