@@ -49,6 +49,10 @@ def parse_args(argv=None):
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--workload", default="step", choices=["step", "accept", "attention"],
+                    help="step: the full verification step (the headline); accept / attention: one kernel alone "
+                         "on the acceptance-only / attention-only workload")
+    ap.add_argument("--tau", type=float, default=1.0)
     return ap.parse_args(argv)
 
 
@@ -369,10 +373,95 @@ def run_sled(args):
         torch.distributed.destroy_process_group()
 
 
+def _peaks():
+    try:
+        return json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))), "measured"
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+def run_accept_only(args):
+    """Acceptance kernel alone: 512 requests x (7 drafts + 1 bonus) rows over the 128256-entry vocabulary."""
+    from paper_2506_09397_b200 import binding as B
+    n, k, V = 512, 7, 128256
+    z, q, d = I.make_accept_rows(n, k, V, tau_draft=1.0, seed=args.seed, device="cuda")
+    logits, qrows = z.reshape(n * (k + 1), V), q.reshape(n * k, V)
+    cu = [8 * i for i in range(n + 1)]
+    ctx = [10_000 + i for i in range(n)]
+    pos0 = [100 + (i % 37) for i in range(n)]
+    dh = d.cpu().numpy().reshape(-1)
+    times, got = [], None
+    for it in range(args.warmup + args.steps):
+        got, ms = B.accept_rows(logits, cu, dh, None if args.greedy else qrows, ctx, pos0, args.tau, args.greedy, seed=it)
+        if it >= args.warmup:
+            times.append(ms)
+    ms = statistics.median(times)
+    rows_read = sum(g[0] + 1 for g in got)                     # rows up to and including the deciding one
+    n_rej = sum(1 for g in got if g[0] < k)
+    alg = rows_read * V * 4 + (0 if args.greedy else n_rej * V * 4)
+    peaks, src = _peaks()
+    ach = alg / (ms / 1e3) / 1e9
+    print(json.dumps({"metric": "acceptance_rows_per_s", "value": rows_read / (ms / 1e3), "unit": "rows/s", "n_gpus": 1,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "f32/u64", "data": "synthetic",
+                      "config": {"workload": f"acceptance only: 512 requests x 8 rows, V=128256, tau={args.tau}, "
+                                             f"{'greedy' if args.greedy else 'sampling'}; {rows_read} rows examined",
+                                 "l2": "inputs larger than L2 (2.1 GB of logits)"},
+                      "acceptance_rate": sum(g[0] for g in got) / (n * k),
+                      "roofline": {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": src,
+                                   "algorithmic_bytes": alg, "all_rows_bytes": n * (k + 1) * V * 4}}))
+
+
+def run_attention_only(args):
+    """Attention kernel alone: 256 requests, query length 2..9, lognormal cache lengths, 32/8 heads of 128."""
+    from paper_2506_09397_b200 import binding as B
+    shape = I.ModelShape("attn_only", 1, 64, 32, 8, 128, 64, 64, 5e5, "bf16", "bf16")
+    nreq = 256
+    qlens = [int(x) for x in torch.randint(2, 10, (nreq,), generator=torch.Generator().manual_seed(1))]
+    lens = I.draw_lognormal_kv_lengths(nreq, 2048, 1.0, 128, 16384, args.seed + 1)
+    w = I.make_weights(shape, 0)
+    eng = B.Engine(shape, w, n_pages=sum((n + 15) // 16 for n in lens) + 8, max_batch=nreq, max_k=8,
+                   max_step_tokens=sum(qlens))
+    eng.shuffle_pages(2)
+    for i, n in enumerate(lens):
+        K, V = I.make_kv(shape, n, 6, i, device="cuda")
+        eng.load_kv(i, K, V, pending=0)
+    T = sum(qlens)
+    q = torch.randn(T, 32, 128, device="cuda").to(torch.bfloat16)
+    out = torch.zeros_like(q)
+    times = []
+    for it in range(args.warmup + args.steps):
+        ms = eng.attention_ragged(0, list(range(nreq)), qlens, q, out)
+        if it >= args.warmup:
+            times.append(ms)
+    ms = statistics.median(times)
+    alg = sum(lens) * 2 * 8 * 128 * 2 + 2 * T * 32 * 128 * 2
+    flops = 4.0 * 32 * 128 * sum(ql * (n - ql) + ql * (ql + 1) / 2 for n, ql in zip(lens, qlens))
+    peaks, src = _peaks()
+    ach = alg / (ms / 1e3) / 1e9
+    print(json.dumps({"metric": "attention_cached_tokens_per_s", "value": sum(lens) / (ms / 1e3), "unit": "tokens/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": f"attention only: 256 requests, q_len 2..9, cache lengths lognormal "
+                                             f"(median 2048, sigma 1, 128..16384; mean {sum(lens) / nreq:.0f}), "
+                                             "32/8 heads of 128, permuted 16-token pages",
+                                 "l2": "inputs larger than L2 (%.2f GB of cache)" % (alg / 1e9)},
+                      "tflops": flops / (ms / 1e3) / 1e12,
+                      "roofline": {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": src,
+                                   "algorithmic_bytes": alg}}))
+    eng.shutdown()
+
+
 def main(argv=None):
     args = parse_args(argv)
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "accept":
+        run_accept_only(args)
+    elif args.workload == "attention":
+        run_attention_only(args)
     else:
         run_sled(args)
 
