@@ -244,7 +244,7 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
 
   // attention work items: (request, KV head, chunk of keys); chunks grow until the item count is near the
   // machine size and the partial-result rows fit
-  const int64_t target = 4LL * e->n_sm;
+  const int64_t target = 2LL * e->n_sm;   // measured: about one item per resident block (two per SM) is best
   int64_t chunk = 256;
   for (;;) {
     int64_t items = 0, rows = 0;
