@@ -52,7 +52,8 @@ __device__ __forceinline__ unsigned long long fixed_exp(float x) {
   p = __fmaf_rn(p, r, 1.0f);
   p = __fmaf_rn(p, r, 1.0f);
   const int n = static_cast<int>(nf);
-  // p * 2^(n+40): p is in [0.7, 1.42], n + 40 >= -3, so the exponent add cannot leave the normal range
+  // p * 2^(n+40): p is in [0.7, 1.42], n + 40 >= -3, so the exponent add cannot leave the normal range;
+  // the product is exact and one truncating conversion gives the integer
   const float scaled = __uint_as_float(__float_as_uint(p) + (static_cast<uint32_t>(n + 40) << 23));
   return __float2ull_rz(scaled);
 }
@@ -127,11 +128,34 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a, int C) {
     float best = -INFINITY;
     int best_i = 0x7fffffff;
     int bad = 0;
-    for (int v = v_lo + threadIdx.x; v < v_hi; v += kThreads) {
-      const float x = z[v];
-      bad |= !(fabsf(x) < INFINITY);
-      const float sv = a.greedy ? x : __fmul_rn(x, a.inv_tau);
-      if (sv > best) { best = sv; best_i = v; }   // ascending v per thread: first maximum kept
+    const bool vec = ((V & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
+    if (vec) {   // four consecutive entries per thread and step (16-byte loads), four steps in flight
+      auto look = [&](int v, const float4& x4) {
+        const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          bad |= !(fabsf(xs[e]) < INFINITY);
+          const float sv = a.greedy ? xs[e] : __fmul_rn(xs[e], a.inv_tau);
+          if (sv > best) { best = sv; best_i = v + e; }   // ascending v per thread: first maximum kept
+        }
+      };
+      constexpr int kStep = kThreads * 4;
+      int v = v_lo + threadIdx.x * 4;
+      for (; v + 3 * kStep < v_hi; v += 4 * kStep) {
+        const float4 x0 = *reinterpret_cast<const float4*>(z + v);
+        const float4 x1 = *reinterpret_cast<const float4*>(z + v + kStep);
+        const float4 x2 = *reinterpret_cast<const float4*>(z + v + 2 * kStep);
+        const float4 x3 = *reinterpret_cast<const float4*>(z + v + 3 * kStep);
+        look(v, x0); look(v + kStep, x1); look(v + 2 * kStep, x2); look(v + 3 * kStep, x3);
+      }
+      for (; v < v_hi; v += kStep) look(v, *reinterpret_cast<const float4*>(z + v));
+    } else {
+      for (int v = v_lo + threadIdx.x; v < v_hi; v += kThreads) {
+        const float x = z[v];
+        bad |= !(fabsf(x) < INFINITY);
+        const float sv = a.greedy ? x : __fmul_rn(x, a.inv_tau);
+        if (sv > best) { best = sv; best_i = v; }   // ascending v per thread: first maximum kept
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -180,7 +204,24 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a, int C) {
     const float m = best;
     // ---- pass 2: Z = sum of the integer numerators
     unsigned long long zsum = 0;
-    for (int v = v_lo + threadIdx.x; v < v_hi; v += kThreads) zsum += fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
+    if (vec) {
+      auto add4 = [&](const float4& x4) {
+        zsum += fixed_exp(__fsub_rn(__fmul_rn(x4.x, a.inv_tau), m)) + fixed_exp(__fsub_rn(__fmul_rn(x4.y, a.inv_tau), m)) +
+                fixed_exp(__fsub_rn(__fmul_rn(x4.z, a.inv_tau), m)) + fixed_exp(__fsub_rn(__fmul_rn(x4.w, a.inv_tau), m));
+      };
+      constexpr int kStep = kThreads * 4;
+      int v = v_lo + threadIdx.x * 4;
+      for (; v + 3 * kStep < v_hi; v += 4 * kStep) {
+        const float4 x0 = *reinterpret_cast<const float4*>(z + v);
+        const float4 x1 = *reinterpret_cast<const float4*>(z + v + kStep);
+        const float4 x2 = *reinterpret_cast<const float4*>(z + v + 2 * kStep);
+        const float4 x3 = *reinterpret_cast<const float4*>(z + v + 3 * kStep);
+        add4(x0); add4(x1); add4(x2); add4(x3);
+      }
+      for (; v < v_hi; v += kStep) add4(*reinterpret_cast<const float4*>(z + v));
+    } else {
+      for (int v = v_lo + threadIdx.x; v < v_hi; v += kThreads) zsum += fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
+    }
     unsigned long long Z = block_sum_u64(zsum, sh.sum_scratch);
     if (C > 1) {
       if (threadIdx.x < C)
@@ -225,13 +266,27 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a, int C) {
       for (int tl = tl_lo; tl < tl_hi; ++tl) {
         unsigned long long mine = 0;
         const int v0 = tl * kTile + threadIdx.x * kVec;
+        float zs[kVec], qs[kVec];
+        if (vec && v0 + kVec <= V) {
+          const float4 z4 = *reinterpret_cast<const float4*>(z + v0);
+          zs[0] = z4.x; zs[1] = z4.y; zs[2] = z4.z; zs[3] = z4.w;
+          if (use_q) {
+            const float4 q4 = *reinterpret_cast<const float4*>(qrow + v0);
+            qs[0] = q4.x; qs[1] = q4.y; qs[2] = q4.z; qs[3] = q4.w;
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < kVec; ++e) {
+            zs[e] = v0 + e < V ? z[v0 + e] : 0.f;
+            qs[e] = (use_q && v0 + e < V) ? qrow[v0 + e] : 0.f;
+          }
+        }
 #pragma unroll
         for (int e = 0; e < kVec; ++e) {
-          const int v = v0 + e;
-          if (v < V) {
-            unsigned long long E = fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
+          if (v0 + e < V) {
+            unsigned long long E = fixed_exp(__fsub_rn(__fmul_rn(zs[e], a.inv_tau), m));
             if (use_q) {
-              const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(qrow[v]), Zd));
+              const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(qs[e]), Zd));
               E = E > Q ? E - Q : 0ull;
             }
             mine += E;
