@@ -202,6 +202,45 @@ def test_large_step_uses_several_token_tiles():
     eng.shutdown()
 
 
+def test_edge_batches():
+    # empty batch, a batch of plain decoding steps (k = 0 everywhere), the largest allowed batch, page reuse
+    shape = I.TINY
+    w = I.make_weights(shape, seed=0)
+    eng = _engine(shape, w, n_pages=16, max_batch=3, max_k=4, max_step_tokens=15)
+    orc = O.OracleModel(shape, oracle_weights(w))
+    assert eng.verify_batch([], 0) == []
+    for c in (1, 2, 3):
+        p = I.make_prompt(shape.vocab, 1 if c == 1 else 17 + c, 0, c)     # context 1: only a pending token, empty cache
+        eng.prefill(c, p)
+        orc.prefill(c, p)
+    explain = []
+    got = _verify_both(eng, orc, [(c, torch.zeros(0, dtype=torch.int32), torch.zeros(0, shape.vocab)) for c in (1, 2, 3)],
+                       seed=1, tau=1.0, greedy=False, tol=1e-4, explain=explain)
+    assert all(g[0] == 0 for g in got)
+    reqs = []
+    for c in (1, 2, 3):                                                   # max_batch requests of max_k drafts = max_step_tokens
+        d, q = I.make_drafts(shape.vocab, 4, 0, c, step=1)
+        reqs.append((c, d, q))
+    eng.set_sampling(0.9, False)
+    _verify_both(eng, orc, reqs, seed=2, tau=0.9, greedy=False, tol=1e-4, explain=explain)
+    for c in (1, 2, 3):
+        assert eng.query_ctx(c)[0] == orc.ctx[c].n_kv
+    used = 16 - eng.stats().pages_free
+    assert used == sum((orc.ctx[c].n_kv + 15) // 16 for c in (1, 2, 3))
+    eng.release(2)
+    p = I.make_prompt(shape.vocab, 40, 0, 4)                               # takes over the pages just returned
+    eng.prefill(4, p)
+    orc.release(2)
+    orc.prefill(4, p)
+    d, q = I.make_drafts(shape.vocab, 3, 0, 4)
+    eng.set_sampling(1.0, True)
+    _verify_both(eng, orc, [(4, d, q), (1,) + tuple(I.make_drafts(shape.vocab, 2, 0, 1, step=2))], seed=3, tau=1.0,
+                 greedy=True, tol=1e-4, explain=explain)
+    st = eng.stats()
+    assert st.steps == 3 and st.requests == 8 and st.contexts_open == 3
+    eng.shutdown()
+
+
 def test_errors_leave_everything_unchanged():
     shape = I.TINY
     w = I.make_weights(shape, seed=0)
