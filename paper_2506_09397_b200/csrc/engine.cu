@@ -600,8 +600,8 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->kpool), e->kv_layer_bytes * c.n_layers))) return fail(rc);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->vpool), e->kv_layer_bytes * c.n_layers))) return fail(rc);
 
-  CU_TRY(cudaMemset(e->kpool, 0, e->kv_layer_bytes * c.n_layers));  // never-written slots are read (and masked): keep them finite
-  CU_TRY(cudaMemset(e->vpool, 0, e->kv_layer_bytes * c.n_layers));
+  if ((cudaMemset(e->kpool, 0, e->kv_layer_bytes * c.n_layers)) != cudaSuccess) return fail(SLED_ERR_DEVICE);  // never-written slots are read (and masked): keep them finite
+  if ((cudaMemset(e->vpool, 0, e->kv_layer_bytes * c.n_layers)) != cudaSuccess) return fail(SLED_ERR_DEVICE);
 
   // step workspaces
   const size_t maxT = c.max_step_tokens, as = dtype_size(e->adtype());
@@ -611,9 +611,9 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if ((rc = dmalloc(e, &e->q_buf, maxT * qd * as))) return fail(rc);
   if ((rc = dmalloc(e, &e->attn_out, padT * qd * as))) return fail(rc);
   if ((rc = dmalloc(e, &e->act_ffn, padT * F * as))) return fail(rc);
-  CU_TRY(cudaMemset(e->act_norm, 0, padT * d * as));
-  CU_TRY(cudaMemset(e->attn_out, 0, padT * qd * as));
-  CU_TRY(cudaMemset(e->act_ffn, 0, padT * F * as));
+  if ((cudaMemset(e->act_norm, 0, padT * d * as)) != cudaSuccess) return fail(SLED_ERR_DEVICE);
+  if ((cudaMemset(e->attn_out, 0, padT * qd * as)) != cudaSuccess) return fail(SLED_ERR_DEVICE);
+  if ((cudaMemset(e->act_ffn, 0, padT * F * as)) != cudaSuccess) return fail(SLED_ERR_DEVICE);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->logits), maxT * c.vocab * 4))) return fail(rc);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->rope_cs), maxT * (c.head_dim / 2) * sizeof(float2)))) return fail(rc);
   {
@@ -632,7 +632,7 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
     if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->q_stage), maxT * c.vocab * 4))) return fail(rc);
   if (c.weight_dtype == SLED_BF16) {
     if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->tc_error), 16))) return fail(rc);
-    CU_TRY(cudaMemset(e->tc_error, 0, 16));
+    if ((cudaMemset(e->tc_error, 0, 16)) != cudaSuccess) return fail(SLED_ERR_DEVICE);
     if (tc_workspace_init(&e->tc_ws, e->n_sm, static_cast<int>(maxT), std::max(c.vocab, std::max(2 * F, qd + 2 * kd))))
       return fail(SLED_ERR_DEVICE);
     if (c.page_size == 16 && (c.head_dim == 64 || c.head_dim == 128)) {
@@ -658,7 +658,7 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if (cudaMallocHost(reinterpret_cast<void**>(&e->h_results), sizeof(int32_t) * 3 * c.max_batch) != cudaSuccess)
     return fail(SLED_ERR_DEVICE);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->d_results), sizeof(int32_t) * 3 * c.max_batch))) return fail(rc);
-  CU_TRY(cudaDeviceSynchronize());
+  if ((cudaDeviceSynchronize()) != cudaSuccess) return fail(SLED_ERR_DEVICE);
   e->st.pages_total = c.n_pages;
   *out = e;
   return SLED_OK;
