@@ -100,7 +100,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "50", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
             self.proc = None
@@ -303,7 +303,6 @@ def run_sled(args):
     sampler.start()
     reqs_dev = marshal(q_dev)
     committed, ms, launches = timed(reqs_dev, args.steps, args.warmup)
-    clocks = sampler.stop()
     tok_all, ms_all = aggregate(float(committed), ms, world)
     value = tok_all / (ms_all / 1e3)
 
@@ -315,6 +314,8 @@ def run_sled(args):
         h2d = 0 if args.greedy else sum(k * shape.vocab * 4 for k in ks)
         e2e = {"value": t2 / (m2 / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d + 64 * T,
                "d2h_bytes_per_step": 12 * Bn, "ms_per_step": m2 / args.steps}
+
+    clocks = sampler.stop()   # sampled over the warm-up and timed steps of both measurements
 
     # device time per kernel kind (events between kernels; extra steps, not the ones behind `value`)
     eng.set_timing(True)
