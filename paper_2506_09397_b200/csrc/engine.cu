@@ -84,7 +84,6 @@ struct sled_engine {
   int part_rows_cap = 0;
   float* q_stage = nullptr;
   TcActivation tc_norm, tc_attn, tc_ffn;
-  TcWorkspace tc_ws;
   int32_t* tc_error = nullptr;  // device word set by a tensor-core GEMM whose bounded wait ran out
 
   // step metadata: pinned staging + device mirror
@@ -168,7 +167,7 @@ int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Lin
   e->mark(K_LINEAR);
   int n;
   if (e->cfg.weight_dtype == SLED_BF16)
-    n = tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_ws, e->tc_error, e->n_sm, epi, e->stream);
+    n = tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_error, epi, e->stream);
   else
     n = launch_gemm_simt(A, e->adtype(), L.w, e->cfg.weight_dtype, T, L.N, L.K, split, out, stride, e->stream);
   if (n < 0) return SLED_ERR_DEVICE;
@@ -444,7 +443,6 @@ void destroy(sled_engine* e) {
     tc_weight_free(&L.qkv.tc); tc_weight_free(&L.o.tc); tc_weight_free(&L.gate_up.tc); tc_weight_free(&L.down.tc);
   }
   tc_weight_free(&e->lm_head.tc);
-  tc_workspace_free(&e->tc_ws);
   for (void* p : e->allocs) cudaFree(p);
   if (e->h_meta) cudaFreeHost(e->h_meta);
   if (e->h_results) cudaFreeHost(e->h_results);
@@ -633,8 +631,6 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if (c.weight_dtype == SLED_BF16) {
     if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->tc_error), 16))) return fail(rc);
     if ((cudaMemset(e->tc_error, 0, 16)) != cudaSuccess) return fail(SLED_ERR_DEVICE);
-    if (tc_workspace_init(&e->tc_ws, e->n_sm, static_cast<int>(maxT), std::max(c.vocab, std::max(2 * F, qd + 2 * kd))))
-      return fail(SLED_ERR_DEVICE);
     if (c.page_size == 16 && (c.head_dim == 64 || c.head_dim == 128)) {
       e->kv_maps.resize(2 * c.n_layers);
       const long long rows = static_cast<long long>(c.n_pages) * c.n_kv_heads * c.page_size;

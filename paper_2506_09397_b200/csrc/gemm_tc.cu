@@ -1,20 +1,21 @@
 // bf16 linear layers on the 5th-generation tensor cores (sm_100a).
 //
-// Persistent kernel, one CTA per SM.  The work of a linear layer is the list of (output tile,
-// 64-wide K slab) units, tile-major; CTA c takes the contiguous range [c*U/G, (c+1)*U/G) of it, so
-// every SM streams the same number of weight bytes whatever the tile count (no wave quantisation)
-// and its TMA ring never drains between tiles.  An output tile is 128 weight rows (the MMA M side)
-// by up to TN_MAX tokens (the N side; the real extent round_up(T,16) is a run-time field of the
-// instruction descriptor, so nothing is padded to a fixed tile).
-//   warp 0   : TMA producer - K slabs of W (evict-first: read once per step) and of the activations
-//              (evict-last: re-read by every tile) into a ring of 128-byte-swizzled stages
-//   warp 1   : allocates tensor memory (two accumulators), issues tcgen05.mma (M=128, N=tn, K=16)
-//              four per slab, commits stages back to the producer and accumulators to the epilogue
-//   warps 2-5: epilogue - tcgen05.ld the fp32 accumulator (lane = weight row, column = token) while
-//              the next segment's MMAs fill the other accumulator
-// A tile whose slabs are shared by several CTAs is finished by whichever of them arrives last: each
-// writes its partial tile to a workspace, takes a ticket, and the last one adds the partial tiles in
-// CTA order (so the sum does not depend on who was last) and stores the result.
+// One CTA computes a 128 (weight rows, the MMA M side) x TN (tokens, the N side) tile over one K slice;
+// the real token extent round_up(T,16) is a run-time field of the instruction descriptor, so nothing is
+// padded to a fixed tile.  Two CTAs fit on an SM; the number of K slices is chosen so that all CTAs of a
+// launch are resident at once with equal work (weight-streaming regime: they share HBM evenly and end
+// together); with many tiles the hardware scheduler hands them out as CTAs retire.  Token tiles of one
+// weight tile are neighbours in the grid, so the second reader of a weight slab finds it in L2.
+//   warp 0   : TMA producer - 64-wide K slabs of W (evict-first: read once per step) and of the activations
+//              (evict-last: re-read by every tile) into a ring of 128-byte-swizzled stages.  Weights do not
+//              depend on the previous kernel: the ring is filled with weight slabs before the
+//              programmatic-launch dependency wait, the activation slabs follow after it
+//   warp 1   : allocates tensor memory, issues tcgen05.mma (M=128, N=tn, K=16) four per slab and commits
+//              each stage back to the producer, the finished accumulator to the epilogue
+//   warps 2-5: epilogue - tcgen05.ld the fp32 accumulator (lane = weight row, column = token) and either
+//              store it transposed (32 consecutive outputs of one token per warp store) or apply SwiGLU
+// K slices leave partial sums [slice][T][N]; the kernel that consumes the layer's output adds them up in
+// slice order while doing its own work (no atomics, no extra pass).
 // Every mbarrier wait is bounded: when one runs out the CTA records a code in *error, lets copies in
 // flight land, frees its tensor memory and returns.
 #include <cuda_bf16.h>
@@ -129,248 +130,6 @@ __device__ __forceinline__ void emit16(const TcEpilogue& e, float* out, int N, i
   }
 }
 
-struct GemmArgs {
-  TcEpilogue epi;
-  int T, N, kb_total, m_tiles, t_tiles;
-  float* out;        // [T][N]
-  float* ws;         // partial tiles: [2 * gridDim.x][TN_MAX][128]
-  int* counters;     // [tiles] arrival tickets, zero between launches
-  int32_t* error;
-};
-
-template <int TN_MAX, int STAGES>
-struct SmemLayout {
-  static constexpr int kAStageBytes = TN_MAX * kBlockK * 2;
-  static constexpr int kStageBytes = kWStageBytes + kAStageBytes;
-  static constexpr int kTiles = STAGES * kStageBytes;
-  static constexpr int kBars = 2 * STAGES + 4;       // full[], empty[], tmem_full[2], tmem_empty[2]
-  static constexpr int kTotal = kTiles + 1024 /*alignment slack*/ + 8 * kBars + 64 + 4 * 160 /*slot list*/;
-};
-
-// first unit of CTA c, and the CTA that owns unit u, for U units over G CTAs
-__device__ __forceinline__ int cta_begin(int c, int U, int G) { return static_cast<int>((static_cast<long long>(c) * U) / G); }
-__device__ __forceinline__ int unit_owner(int u, int U, int G) {
-  int c = static_cast<int>((static_cast<long long>(u) * G) / U);
-  while (c + 1 < G && cta_begin(c + 1, U, G) <= u) ++c;
-  while (c > 0 && cta_begin(c, U, G) > u) --c;
-  return c;
-}
-
-template <int TN_MAX, int STAGES>
-__global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap map_w,
-                                                          const __grid_constant__ CUtensorMap map_a, GemmArgs g) {
-  using L = SmemLayout<TN_MAX, STAGES>;
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
-  uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t bars = base + L::kTiles;
-  const uint32_t bar_full = bars, bar_empty = bars + 8 * STAGES;
-  const uint32_t bar_tfull = bars + 16 * STAGES, bar_tempty = bar_tfull + 16;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kTiles + 8 * L::kBars);
-  volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * L::kBars + 8);
-  volatile int* ticket_slot = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * L::kBars + 16);
-  volatile int* epi_abort = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * L::kBars + 24);
-  volatile int* slot_list = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * L::kBars + 64);   // <= gridDim.x <= 160 entries
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its own prologue
-  const int G = gridDim.x, cta = blockIdx.x;
-  const int U = g.m_tiles * g.t_tiles * g.kb_total;        // fits 31 bits (checked by the launcher)
-  const int u0 = cta_begin(cta, U, G), u1 = cta_begin(cta + 1, U, G);
-  const int tile_first = u0 / g.kb_total, kb_first = u0 % g.kb_total;   // the only divisions on the unit index
-  constexpr uint32_t kTmemCols = 2 * TN_MAX < 32 ? 32 : 2 * TN_MAX;
-
-  if (threadIdx.x == 0) {
-    *abort_slot = 0;
-    *epi_abort = 0;
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
-    for (int s = 0; s < 2 * STAGES + 2; ++s) mbar_init(bars + 8 * s, 1);
-    mbar_init(bar_tempty, 4);       // one arrival per epilogue warp
-    mbar_init(bar_tempty + 8, 4);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 1) {  // tensor memory: two accumulator tiles of TN_MAX fp32 columns x 128 lanes
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))),
-                 "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = *tmem_slot;
-
-  if (warp == 0) {
-    if (lane == 0) {
-      uint64_t pol_first, pol_last;
-      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
-      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_last));
-      // The weights do not depend on the previous kernel: fill the ring with weight slabs first, then wait
-      // for the predecessor (its output is this kernel's activation operand), then add the activation slabs.
-      const int pre = min(STAGES, u1 - u0);
-      int tile = tile_first, kb = kb_first;
-      for (int j = 0; j < pre; ++j) {
-        mbar_expect_tx(bar_full + 8 * j, L::kStageBytes);
-        tma_load_2d(base + j * L::kStageBytes, &map_w, kb * kBlockK, (tile % g.m_tiles) * kBlockM, bar_full + 8 * j, pol_first);
-        if (++kb == g.kb_total) { kb = 0; ++tile; }
-      }
-      pdl_wait_here();
-      tile = tile_first;
-      kb = kb_first;
-      for (int j = 0; j < pre; ++j) {
-        tma_load_2d(base + j * L::kStageBytes + kWStageBytes, &map_a, kb * kBlockK, (tile / g.m_tiles) * TN_MAX,
-                    bar_full + 8 * j, pol_last);
-        if (++kb == g.kb_total) { kb = 0; ++tile; }
-      }
-      int s = pre == STAGES ? 0 : pre;
-      uint32_t ph = pre == STAGES ? 1u : 0u;    // parity of the ring pass the next stage belongs to
-      int m_row = (tile % g.m_tiles) * kBlockM, t_row = (tile / g.m_tiles) * TN_MAX;
-      for (int u = u0 + pre; u < u1; ++u) {
-        if (*abort_slot || !mbar_wait(bar_empty + 8 * s, ph ^ 1, g.error, 1)) { *abort_slot = 1; break; }
-        const uint32_t full = bar_full + 8 * s, wdst = base + s * L::kStageBytes;
-        mbar_expect_tx(full, L::kStageBytes);
-        tma_load_2d(wdst, &map_w, kb * kBlockK, m_row, full, pol_first);
-        tma_load_2d(wdst + kWStageBytes, &map_a, kb * kBlockK, t_row, full, pol_last);
-        if (++kb == g.kb_total) {
-          kb = 0;
-          ++tile;
-          m_row = (tile % g.m_tiles) * kBlockM;
-          t_row = (tile / g.m_tiles) * TN_MAX;
-        }
-        if (++s == STAGES) { s = 0; ph ^= 1u; }
-      }
-    }
-  } else if (warp == 1) {
-    if (lane == 0) {
-      int s = 0;
-      uint32_t ph = 0;
-      int seg = 0, tile = tile_first, ka = kb_first;
-      for (int u = u0; u < u1; ++seg) {
-        const int kb_end = min(g.kb_total, ka + (u1 - u));
-        const int t0 = (tile / g.m_tiles) * TN_MAX;
-        const int tn = min(TN_MAX, ((g.T - t0) + 15) & ~15);
-        const int b = seg & 1;
-        // the accumulator must have been read out by the epilogue of two segments ago
-        if (*abort_slot || !mbar_wait(bar_tempty + 8 * b, ((seg >> 1) & 1) ^ 1, g.error, 5)) { *abort_slot = 1; break; }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = tn, M = 128
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(tn >> 3) << 17) |
-                               (static_cast<uint32_t>(kBlockM >> 4) << 24);
-        const uint32_t acc = tmem_base + static_cast<uint32_t>(b * TN_MAX);
-        bool ok = true;
-        for (int kb = ka; kb < kb_end; ++kb) {
-          if (*abort_slot || !mbar_wait(bar_full + 8 * s, ph, g.error, 2)) { ok = false; break; }
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t wsrc = base + s * L::kStageBytes;
-          const uint64_t adesc = umma_desc(wsrc), bdesc = umma_desc(wsrc + kWStageBytes);
-#pragma unroll
-          for (int kk = 0; kk < kBlockK / 16; ++kk)   // 16 bf16 = 32 bytes further along K inside the swizzled row
-            umma_bf16(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb > ka || kk > 0) ? 1u : 0u);
-          umma_commit(bar_empty + 8 * s);             // stage free once these MMAs have read it
-          if (++s == STAGES) { s = 0; ph ^= 1u; }
-        }
-        if (!ok) { *abort_slot = 1; break; }
-        umma_commit(bar_tfull + 8 * b);               // accumulator complete
-        u += kb_end - ka;
-        ka = 0;
-        ++tile;
-      }
-    }
-  } else {
-    const int quad = warp & 3;                        // a warp may only touch tensor-memory lanes 32*(warp%4)..+31
-    const int row = quad * 32 + lane;
-    int seg = 0, tile = tile_first, ka = kb_first;
-    for (int u = u0; u < u1; ++seg) {
-      const int kb_end = min(g.kb_total, ka + (u1 - u));
-      const int m_tile = tile % g.m_tiles, t0 = (tile / g.m_tiles) * TN_MAX;
-      const int tn = min(TN_MAX, ((g.T - t0) + 15) & ~15);
-      const int b = seg & 1;
-      // the four epilogue warps must agree on whether to go on (they meet at named barriers below)
-      if (lane == 0 && !mbar_wait(bar_tfull + 8 * b, (seg >> 1) & 1, g.error, 3)) *epi_abort = 1;
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (*epi_abort) { *abort_slot = 1; break; }
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t acc = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(b * TN_MAX);
-      const int n = m_tile * kBlockM + row;
-      const bool whole = ka == 0 && kb_end == g.kb_total;
-      float* part = g.ws + (static_cast<long long>(cta) * 2 + (tile == tile_first ? 0 : 1)) * (TN_MAX * 128);
-      for (int c0 = 0; c0 < tn; c0 += 16) {
-        uint32_t v[16];
-        asm volatile(
-            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-            : "r"(acc + static_cast<uint32_t>(c0)));
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (whole) {
-          float val[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) val[i] = __uint_as_float(v[i]);
-          emit16(g.epi, g.out, g.N, g.T, n, t0 + c0, val);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) __stcg(part + (c0 + i) * 128 + row, __uint_as_float(v[i]));
-        }
-      }
-      // the accumulator has been read: hand it back to the MMA warp
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_tempty + 8 * b) : "memory");
-      if (!whole) {
-        // ticket: the last of the CTAs sharing this tile adds all partial tiles, in CTA order
-        const int uf = tile * g.kb_total;
-        const int c_first = unit_owner(uf, U, G), c_last = unit_owner(uf + g.kb_total - 1, U, G);
-        __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (warp == 2 && lane == 0) *ticket_slot = atomicAdd(g.counters + tile, 1);
-        // where each sharer left its partial tile: slot 0 if this is its first tile, else slot 1
-        for (int c = c_first + static_cast<int>(threadIdx.x) - 64; c <= c_last; c += 128)
-          slot_list[c - c_first] = c * 2 + (tile == cta_begin(c, U, G) / g.kb_total ? 0 : 1);
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        const int ticket = *ticket_slot;
-        if (ticket == c_last - c_first) {
-          __threadfence();
-          const int n_seg = c_last - c_first + 1;
-          for (int c0 = 0; c0 < tn; c0 += 16) {      // 16 independent loads in flight per thread and sharer
-            float sum[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) sum[j] = 0.f;
-            for (int i = 0; i < n_seg; ++i) {
-              const float* src = g.ws + static_cast<long long>(slot_list[i]) * (TN_MAX * 128) + c0 * 128 + row;
-#pragma unroll
-              for (int j = 0; j < 16; ++j) sum[j] += __ldcg(src + j * 128);
-            }
-            emit16(g.epi, g.out, g.N, g.T, n, t0 + c0, sum);
-          }
-          if (warp == 2 && lane == 0) g.counters[tile] = 0;   // ready for the next launch
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");   // ticket_slot is reused by the next segment
-      }
-      u += kb_end - ka;
-      ka = 0;
-      ++tile;
-    }
-  }
-
-  // teardown
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  if (warp == 1) {
-    if (*abort_slot != 0) {
-      // something timed out: give copies and MMAs still in flight time to land before the memory goes away
-      const long long t1 = clock64();
-      while (clock64() - t1 < 2000000LL) __nanosleep(1000);
-    }
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Small-T kernel (T <= 128, the weight-streaming regime): one CTA per (128-row weight tile, K slice),
-// two CTAs per SM, all CTAs of a launch resident at once with equal work, so they share the HBM
-// bandwidth evenly and finish together.  K slices leave partial sums [slice][T][N]; the kernel that
-// consumes the layer's output adds them up (fixed order) while doing its own work.
 template <int TN_MAX, int STAGES>
 struct SplitSmemLayout {
   static constexpr int kAStageBytes = TN_MAX * kBlockK * 2;
@@ -395,7 +154,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its own prologue
-  const int m_tile = blockIdx.x, t_tile = blockIdx.y, split = blockIdx.z;
+  const int t_tile = blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
   const int kb0 = split * kb_per_split;
   const int nkb = min(kb_per_split, kb_total - kb0);
   const int t0 = t_tile * TN_MAX;
@@ -547,46 +306,6 @@ int make_map(CUtensorMap* map, const void* ptr, long long rows, int K, int box_r
 }
 
 
-template <int TN_MAX, int STAGES>
-int launch_one(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K, float* out, const TcWorkspace& wsp,
-               int32_t* error, int n_sm, const TcEpilogue& epi, cudaStream_t s) {
-  using L = SmemLayout<TN_MAX, STAGES>;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(tc_gemm_kernel<TN_MAX, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess)
-      return -1;
-    configured = true;
-  }
-  GemmArgs g{};
-  g.epi = epi;
-  g.T = T;
-  g.N = N;
-  g.kb_total = (K + kBlockK - 1) / kBlockK;
-  g.m_tiles = (N + kBlockM - 1) / kBlockM;
-  g.t_tiles = (T + TN_MAX - 1) / TN_MAX;
-  g.out = out;
-  g.ws = wsp.partial;
-  g.counters = wsp.counters;
-  g.error = error;
-  const long long units = static_cast<long long>(g.m_tiles) * g.t_tiles * g.kb_total;
-  const int grid = static_cast<int>(std::min<long long>(n_sm, units));
-  if (g.m_tiles * g.t_tiles > wsp.max_tiles || grid > wsp.max_ctas || grid > 160 || TN_MAX > wsp.tn_max || units >= (1ll << 31)) return -1;
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(grid, 1, 1);
-  cfg.blockDim = dim3(192, 1, 1);
-  cfg.dynamicSmemBytes = L::kTotal;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while the previous kernel drains
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<TN_MAX, STAGES>, mw, ma, g);
-  return err == cudaSuccess ? 1 : -1;
-}
-
-int tile_tokens(int T) { return T <= 64 ? 64 : (T <= 128 ? 128 : 256); }
-
 }  // namespace
 
 int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int cols, int box_rows) {
@@ -613,28 +332,10 @@ int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K) {
   return 0;
 }
 
-int tc_workspace_init(TcWorkspace* w, int n_sm, int max_T, int max_N) {
-  w->max_ctas = n_sm;
-  w->tn_max = 256;
-  w->max_tiles = ((max_N + kBlockM - 1) / kBlockM) * ((max_T + 63) / 64);
-  if (cudaMalloc(reinterpret_cast<void**>(&w->partial), static_cast<size_t>(n_sm) * 2 * 256 * 128 * sizeof(float)) != cudaSuccess) return -1;
-  if (cudaMalloc(reinterpret_cast<void**>(&w->counters), static_cast<size_t>(w->max_tiles) * sizeof(int)) != cudaSuccess) return -1;
-  if (cudaMemset(w->counters, 0, static_cast<size_t>(w->max_tiles) * sizeof(int)) != cudaSuccess) return -1;
-  return 0;
-}
-
-void tc_workspace_free(TcWorkspace* w) {
-  if (w->partial) cudaFree(w->partial);
-  if (w->counters) cudaFree(w->counters);
-  w->partial = nullptr;
-  w->counters = nullptr;
-}
-
-// K slices for the small-T kernel: as many as keep every CTA resident at once (two per SM), each with
-// at least 4 slabs; the returned count is the number of slices that actually get work.
+// K slices: as many as keep every CTA of the launch resident at once (two per SM), each with at least 4 slabs;
+// the returned count is the number of slices that actually get work.
 int tc_gemm_split(int T, int N, int K, int n_sm) {
-  if (T > 128) return 1;   // persistent kernel: slices are summed inside
-  const int tiles = (N + kBlockM - 1) / kBlockM;
+  const int tiles = ((N + kBlockM - 1) / kBlockM) * (T > 128 ? (T + 255) / 256 : 1);
   const int kb_total = (K + kBlockK - 1) / kBlockK;
   int s = std::max(1, (2 * n_sm) / tiles);
   s = std::min(s, std::max(1, kb_total / 4));
@@ -656,7 +357,7 @@ static int launch_split(const CUtensorMap& mw, const CUtensorMap& ma, int T, int
   const int kb_total = (K + kBlockK - 1) / kBlockK;
   const int kb_per = (kb_total + n_split - 1) / n_split;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((N + kBlockM - 1) / kBlockM, 1, n_split);
+  cfg.gridDim = dim3((T + TN_MAX - 1) / TN_MAX, (N + kBlockM - 1) / kBlockM, n_split);   // token tiles of one weight tile are neighbours
   cfg.blockDim = dim3(192, 1, 1);
   cfg.dynamicSmemBytes = L::kTotal;
   cfg.stream = s;
@@ -671,13 +372,12 @@ static int launch_split(const CUtensorMap& mw, const CUtensorMap& ma, int T, int
 }
 
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
-                   const TcWorkspace& wsp, int32_t* error, int n_sm, const TcEpilogue& epi, cudaStream_t s) {
+                   int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
   if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
   if (epi.mode != kEpiStore && n_split != 1) return -1;   // a fused epilogue needs the complete sum
   if (T <= 64) return launch_split<64, 4>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (T <= 128) return launch_split<128, 3>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
-  if (n_split != 1) return -1;
-  return launch_one<256, 4>(w.map, a.map[2], T, w.N, w.K, out, wsp, error, n_sm, epi, s);
+  return launch_split<256, 2>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
 }
 
 }  // namespace sled

@@ -28,24 +28,16 @@ struct TcEpilogue {       // what happens to the finished sums (see emit16 in ge
   int act_ld = 0;
 };
 
-struct TcWorkspace {    // shared by all linear layers of an engine (one launch at a time on its stream)
-  float* partial = nullptr;   // partial tiles of CTAs that share an output tile
-  int* counters = nullptr;    // one arrival counter per output tile, zero between launches
-  int max_ctas = 0, max_tiles = 0, tn_max = 0;
-};
-
 // 2D bf16 tensor map over a row-major [rows][cols] array: boxes of 64 columns x box_rows rows, 128-byte swizzle
 int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int cols, int box_rows);
 int tc_weight_init(TcWeight* w, const void* dev_ptr, int N, int K);
 void tc_weight_free(TcWeight* w);
 int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K);
-int tc_workspace_init(TcWorkspace* w, int n_sm, int max_T, int max_N);
-void tc_workspace_free(TcWorkspace* w);
-// number of partial-sum slices [slice][T][N] a launch leaves behind for this shape (1 when T > 128)
+// number of partial-sum slices [slice][T][N] a launch leaves behind for this shape
 int tc_gemm_split(int T, int N, int K, int n_sm);
 // out[slice][T][N] = A[T][K slice] . W[N][K slice]^T; returns kernels launched (1) or a negative value;
 // `error` is a device word set if a bounded wait ran out
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
-                   const TcWorkspace& wsp, int32_t* error, int n_sm, const TcEpilogue& epi, cudaStream_t s);
+                   int32_t* error, const TcEpilogue& epi, cudaStream_t s);
 
 }  // namespace sled
