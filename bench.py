@@ -32,12 +32,12 @@ import torch
 
 from paper_2506_09397_b200 import inputs as I
 
-# DRAM traffic of the linear-layer kernel per launch at the default workload (ncu: dram__bytes_read.sum +
-# dram__bytes_write.sum, summed over the 129 launches of a step, see
-# profiles/ncu_tc_gemm_split_kernel_and_attn_mma_kernel_llama8b_2layer_b16.txt).  Only valid for the kernel source
-# it was taken from: reported as null when that file has changed since.
-TRAFFIC_LINEAR = {"workload": ("llama8b", 32, 16), "bytes_per_launch": 120.5e6,
-                  "source_sha1": "07b045a432a122b7659399d6f83144f72493ef9d"}
+# DRAM traffic of the linear-layer kernel per launch (ncu: dram__bytes_read.sum + dram__bytes_write.sum, summed over
+# the 129 launches of a step; profiles/ncu_linear_and_attention_kernels_llama8b_2layer_b{16,64}.txt), keyed by
+# (shape, layers, batch).  Only valid for the kernel source it was taken from: reported as null when that file has
+# changed since.
+TRAFFIC_LINEAR = {"bytes_per_launch": {("llama8b", 32, 16): 120.6e6, ("llama8b", 32, 64): 128.9e6},
+                  "source_sha1": "4932f71e1cca39f68c3c2164eb9167b6f8ba5763"}
 
 METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
@@ -350,9 +350,8 @@ def run_sled(args):
     try:
         import hashlib
         src = open(os.path.join(ROOT, "paper_2506_09397_b200", "csrc", "gemm_tc.cu"), "rb").read()
-        if (shape.name, shape.n_layers, Bn) == TRAFFIC_LINEAR["workload"] and \
-                hashlib.sha1(src).hexdigest() == TRAFFIC_LINEAR["source_sha1"]:
-            traffic = TRAFFIC_LINEAR["bytes_per_launch"]
+        if hashlib.sha1(src).hexdigest() == TRAFFIC_LINEAR["source_sha1"]:
+            traffic = TRAFFIC_LINEAR["bytes_per_launch"].get((shape.name, shape.n_layers, Bn))
     except Exception:
         pass
     roof.update({"traffic": traffic, "algorithmic_bytes_per_launch": lb / max(n_lin, 1), "kernel": "linear-layer kernel (all linear layers of a step)", "peak_source": peak_src,
