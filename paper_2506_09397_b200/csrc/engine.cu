@@ -326,6 +326,7 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
   const sled_config& c = e->cfg;
   const int T = pk.T, d = c.d_model, ad = e->adtype();
   int n;
+
   e->mark(K_OTHER);
   n = launch_embed(e->tok_emb, c.weight_dtype, pk.ids, T, d, e->x, e->stream);
   e->count(n, K_OTHER);
@@ -465,26 +466,41 @@ int upload(sled_engine* e, const void* src, size_t bytes, void** dst) {
   return SLED_OK;
 }
 
+// bf16 weights: replaces the row-major matrix `rowmajor` (a plain cudaMalloc that this call frees) by its tiled copy
+int finish_linear(sled_engine* e, Linear* L, void* rowmajor, int N, int K) {
+  L->N = N;
+  L->K = K;
+  if (e->cfg.weight_dtype != SLED_BF16) {
+    L->w = rowmajor;
+    e->allocs.push_back(rowmajor);
+    return SLED_OK;
+  }
+  int rc = dmalloc(e, &L->w, tc_weight_tiled_bytes(N, K));
+  if (!rc && tc_weight_init(&L->tc, rowmajor, L->w, N, K) != 0) rc = SLED_ERR_ARG;
+  cudaFree(rowmajor);
+  return rc;
+}
+
 int make_linear(sled_engine* e, Linear* L, std::initializer_list<std::pair<const void*, int>> parts, int K) {
   // concatenates the row blocks of `parts` into one [N][K] matrix
   const size_t es = dtype_size(e->cfg.weight_dtype);
   int N = 0;
-  for (auto& p : parts) N += p.second;
-  int rc = dmalloc(e, &L->w, static_cast<size_t>(N) * K * es);
-  if (rc) return rc;
-  size_t off = 0;
   for (auto& p : parts) {
     if (!p.first) return SLED_ERR_ARG;
+    N += p.second;
+  }
+  void* tmp = nullptr;
+  CU_TRY(cudaMalloc(&tmp, static_cast<size_t>(N) * K * es));
+  size_t off = 0;
+  for (auto& p : parts) {
     const size_t bytes = static_cast<size_t>(p.second) * K * es;
-    CU_TRY(cudaMemcpy(static_cast<char*>(L->w) + off, p.first, bytes, cudaMemcpyDefault));
+    if (cudaMemcpy(static_cast<char*>(tmp) + off, p.first, bytes, cudaMemcpyDefault) != cudaSuccess) {
+      cudaFree(tmp);
+      return SLED_ERR_DEVICE;
+    }
     off += bytes;
   }
-  L->N = N;
-  L->K = K;
-  if (e->cfg.weight_dtype == SLED_BF16) {
-    if (tc_weight_init(&L->tc, L->w, N, K) != 0) return SLED_ERR_ARG;
-  }
-  return SLED_OK;
+  return finish_linear(e, L, tmp, N, K);
 }
 
 // gate and up projections as one matrix with their rows interleaved (row 2f = gate f, row 2f+1 = up f),
@@ -492,14 +508,14 @@ int make_linear(sled_engine* e, Linear* L, std::initializer_list<std::pair<const
 int make_gate_up(sled_engine* e, Linear* L, const void* gate, const void* up, int F, int K) {
   if (!gate || !up) return SLED_ERR_ARG;
   const size_t row = static_cast<size_t>(K) * dtype_size(e->cfg.weight_dtype);
-  int rc = dmalloc(e, &L->w, 2 * static_cast<size_t>(F) * row);
-  if (rc) return rc;
-  CU_TRY(cudaMemcpy2D(L->w, 2 * row, gate, row, row, F, cudaMemcpyDefault));
-  CU_TRY(cudaMemcpy2D(static_cast<char*>(L->w) + row, 2 * row, up, row, row, F, cudaMemcpyDefault));
-  L->N = 2 * F;
-  L->K = K;
-  if (e->cfg.weight_dtype == SLED_BF16 && tc_weight_init(&L->tc, L->w, L->N, K) != 0) return SLED_ERR_ARG;
-  return SLED_OK;
+  void* tmp = nullptr;
+  CU_TRY(cudaMalloc(&tmp, 2 * static_cast<size_t>(F) * row));
+  if (cudaMemcpy2D(tmp, 2 * row, gate, row, row, F, cudaMemcpyDefault) != cudaSuccess ||
+      cudaMemcpy2D(static_cast<char*>(tmp) + row, 2 * row, up, row, row, F, cudaMemcpyDefault) != cudaSuccess) {
+    cudaFree(tmp);
+    return SLED_ERR_DEVICE;
+  }
+  return finish_linear(e, L, tmp, 2 * F, K);
 }
 
 int check_cfg(const sled_config& c) {

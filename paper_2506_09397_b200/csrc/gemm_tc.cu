@@ -135,7 +135,7 @@ struct SplitSmemLayout {
   static constexpr int kAStageBytes = TN_MAX * kBlockK * 2;
   static constexpr int kStageBytes = kWStageBytes + kAStageBytes;
   static constexpr int kTiles = STAGES * kStageBytes;
-  static constexpr int kTotal = kTiles + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kTotal = kTiles + 256 /*barriers*/;   // two CTAs per SM: 2 * (kTotal + 1 KB) <= 228 KB
 };
 
 template <int TN_MAX, int STAGES>
@@ -144,10 +144,10 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
                                                        int kb_total, int kb_per_split, float* __restrict__ out,
                                                        long long split_stride, int32_t* error, TcEpilogue epi) {
   using L = SplitSmemLayout<TN_MAX, STAGES>;
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
-  uint8_t* base_ptr = smem_raw + (base - raw);
+  constexpr int kTmemCols = TN_MAX <= 32 ? 32 : TN_MAX <= 64 ? 64 : TN_MAX <= 128 ? 128 : 256;   // a power of two
+  extern __shared__ __align__(1024) uint8_t smem_raw[];    // swizzled tiles need 1024-byte alignment
+  const uint32_t base = smem_u32(smem_raw);
+  uint8_t* base_ptr = smem_raw;
   const uint32_t bars = base + L::kTiles;                 // full[STAGES], empty[STAGES], tmem_full, then the tmem address
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kTiles + 8 * (2 * STAGES + 1));
   volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * (2 * STAGES + 1) + 8);
@@ -160,7 +160,10 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
   const int t0 = t_tile * TN_MAX;
   const int tn = min(TN_MAX, ((T - t0) + 15) & ~15);     // token columns of this tile, multiple of 16
 
-  if (threadIdx.x == 0) *abort_slot = *reinterpret_cast<volatile int32_t*>(error);
+  if (threadIdx.x == 0) {
+    if (base & 1023u) atomicCAS(error, 0, 5);              // the stage layout below would be wrong: refuse to run
+    *abort_slot = *reinterpret_cast<volatile int32_t*>(error);
+  }
   __syncthreads();
   if (*abort_slot != 0) return;                           // an earlier CTA gave up: do not start
 
@@ -172,7 +175,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
   }
   if (warp == 1) {  // tensor memory for the accumulator tile: TN_MAX fp32 columns x 128 lanes
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))),
-                 "r"(static_cast<uint32_t>(TN_MAX < 32 ? 32 : TN_MAX)) : "memory");
+                 "r"(static_cast<uint32_t>(kTmemCols)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -192,7 +195,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
       for (int kb = 0; kb < pre; ++kb) {
         const uint32_t full = bars + 8 * kb;
         mbar_expect_tx(full, L::kStageBytes);
-        tma_load_2d(base + kb * L::kStageBytes, &map_w, (kb0 + kb) * kBlockK, m_tile * kBlockM, full, pol_first);
+        tma_load_2d(base + kb * L::kStageBytes, &map_w, 0, (m_tile * kb_total + kb0 + kb) * kBlockM, full, pol_first);
       }
       pdl_wait_here();
       for (int kb = 0; kb < pre; ++kb)
@@ -204,7 +207,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
         const uint32_t full = bars + 8 * s;
         mbar_expect_tx(full, L::kStageBytes);
         const uint32_t wdst = base + s * L::kStageBytes;
-        tma_load_2d(wdst, &map_w, (kb0 + kb) * kBlockK, m_tile * kBlockM, full, pol_first);
+        tma_load_2d(wdst, &map_w, 0, (m_tile * kb_total + kb0 + kb) * kBlockM, full, pol_first);
         tma_load_2d(wdst + kWStageBytes, &map_a, (kb0 + kb) * kBlockK, t0, full, pol_last);
       }
     }
@@ -267,7 +270,23 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
       while (clock64() - t1 < 2000000LL) __nanosleep(1000);
     }
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                 "r"(static_cast<uint32_t>(TN_MAX < 32 ? 32 : TN_MAX)) : "memory");
+                 "r"(static_cast<uint32_t>(kTmemCols)) : "memory");
+  }
+}
+
+// Weights are kept tile by tile: block (m, kb) of the tiled array is the 128 x 64 piece W[128m .. +127][64kb .. +63]
+// as 128 rows of 128 bytes, zero where the matrix ends.  One pipeline stage is then one contiguous 16 KB read, and
+// the stages of a CTA follow each other in memory (DRAM pages are read whole instead of 128 bytes at a time).
+__global__ void __launch_bounds__(256) retile_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst,
+                                                     int N, int K, int n_kslabs) {
+  const int kb = blockIdx.x, mt = blockIdx.y;
+  uint4* out = reinterpret_cast<uint4*>(dst + (static_cast<long long>(mt) * n_kslabs + kb) * (kBlockM * kBlockK));
+  for (int i = threadIdx.x; i < kBlockM * (kBlockK / 8); i += blockDim.x) {
+    const int r = i / (kBlockK / 8), c = i % (kBlockK / 8);
+    const int n = mt * kBlockM + r, k = kb * kBlockK + c * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (n < N && k < K) v = *reinterpret_cast<const uint4*>(src + static_cast<long long>(n) * K + k);   // K is a multiple of 8
+    out[i] = v;
   }
 }
 
@@ -312,8 +331,16 @@ int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int
   return make_map(map, dev_ptr, rows, cols, box_rows);
 }
 
-int tc_weight_init(TcWeight* w, const void* dev_ptr, int N, int K) {
-  if (make_map(&w->map, dev_ptr, N, K, kBlockM)) return -1;
+size_t tc_weight_tiled_bytes(int N, int K) {
+  return static_cast<size_t>((N + kBlockM - 1) / kBlockM) * ((K + kBlockK - 1) / kBlockK) * kWStageBytes;
+}
+
+int tc_weight_init(TcWeight* w, const void* rowmajor, void* tiled, int N, int K) {
+  if (K % 8 || (reinterpret_cast<uintptr_t>(rowmajor) & 15) || (reinterpret_cast<uintptr_t>(tiled) & 15)) return -1;
+  const int n_mtiles = (N + kBlockM - 1) / kBlockM, n_kslabs = (K + kBlockK - 1) / kBlockK;
+  retile_kernel<<<dim3(n_kslabs, n_mtiles), 256>>>(static_cast<const __nv_bfloat16*>(rowmajor), static_cast<__nv_bfloat16*>(tiled), N, K, n_kslabs);
+  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+  if (make_map(&w->map, tiled, static_cast<long long>(n_mtiles) * n_kslabs * kBlockM, kBlockK, kBlockM)) return -1;
   w->N = N;
   w->K = K;
   w->ready = true;
@@ -324,8 +351,8 @@ void tc_weight_free(TcWeight* w) { w->ready = false; }
 
 int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K) {
   if (rows % 256) return -1;
-  const int boxes[3] = {64, 128, 256};
-  for (int i = 0; i < 3; ++i)
+  const int boxes[kTokenTiles] = {32, 64, 96, 128, 256};
+  for (int i = 0; i < kTokenTiles; ++i)
     if (make_map(&a->map[i], dev_ptr, rows, K, boxes[i])) return -1;
   a->rows = rows;
   a->K = K;
@@ -375,9 +402,12 @@ int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split,
                    int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
   if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
   if (epi.mode != kEpiStore && n_split != 1) return -1;   // a fused epilogue needs the complete sum
-  if (T <= 64) return launch_split<64, 4>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
-  if (T <= 128) return launch_split<128, 3>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
-  return launch_split<256, 2>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  // token tile = the smallest box that holds the step; what the narrower activation stage saves goes into ring depth
+  if (T <= 32) return launch_split<32, 5>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (T <= 64) return launch_split<64, 4>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (T <= 96) return launch_split<96, 4>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (T <= 128) return launch_split<128, 3>(w.map, a.map[3], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  return launch_split<256, 2>(w.map, a.map[4], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
 }
 
 }  // namespace sled

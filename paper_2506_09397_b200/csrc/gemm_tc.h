@@ -10,14 +10,15 @@
 
 namespace sled {
 
-struct TcWeight {       // [N][K] bf16, row-major, device memory
-  CUtensorMap map;      // box 64 (k) x 128 (rows), 128-byte swizzle
+struct TcWeight {       // [N][K] bf16 weights, stored as 128 x 64 tiles of 16 KB (see tc_weight_init)
+  CUtensorMap map;      // over the tiled array seen as rows of 128 bytes; box = one tile, 128-byte swizzle
   int N = 0, K = 0;
   bool ready = false;
 };
 
+constexpr int kTokenTiles = 5;
 struct TcActivation {   // [rows][K] bf16, row-major, device memory; rows is a multiple of 256
-  CUtensorMap map[3];   // boxes of 64 (k) x {64, 128, 256} rows
+  CUtensorMap map[kTokenTiles];   // boxes of 64 (k) x {32, 64, 96, 128, 256} rows
   int rows = 0, K = 0;
 };
 
@@ -30,7 +31,11 @@ struct TcEpilogue {       // what happens to the finished sums (see emit16 in ge
 
 // 2D bf16 tensor map over a row-major [rows][cols] array: boxes of 64 columns x box_rows rows, 128-byte swizzle
 int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int cols, int box_rows);
-int tc_weight_init(TcWeight* w, const void* dev_ptr, int N, int K);
+// Bytes of the tiled copy of an [N][K] matrix, and its construction from the row-major matrix (both in
+// device memory; `tiled` 16-byte aligned, tc_weight_tiled_bytes(N, K) long).  The row-major copy is not
+// needed afterwards.  Synchronises the device.
+size_t tc_weight_tiled_bytes(int N, int K);
+int tc_weight_init(TcWeight* w, const void* rowmajor, void* tiled, int N, int K);
 void tc_weight_free(TcWeight* w);
 int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K);
 // number of partial-sum slices [slice][T][N] a launch leaves behind for this shape
