@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(AttnArgs a) {
   const KT* vpool = static_cast<const KT*>(a.vpool);
   const AT* qbuf = static_cast<const AT*>(a.q);
   const bool split = a.req_chunks[req] > 1;
-  const int chunk_idx = key_start / a.chunk_keys;
+  const int chunk_idx = key_start / a.req_chunk_keys[req];
   const float scale = rsqrtf(static_cast<float>(H)) * 1.4426950408889634f;  // scores in log2 units
 
   const int part = threadIdx.x & 3;

@@ -331,7 +331,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(AttnArgs a, const __gr
   c.n_rows = (a.cu_q[c.req + 1] - c.row0) * c.group;
   c.kv_base = a.kv_base[c.req];
   c.split = a.req_chunks[c.req] > 1;
-  c.chunk_idx = c.key_start / a.chunk_keys;
+  c.chunk_idx = c.key_start / a.req_chunk_keys[c.req];
   c.scale = rsqrtf(static_cast<float>(H)) * 1.4426950408889634f;
   const int n_pass = (c.n_rows + 63) / 64;
 

@@ -178,9 +178,9 @@ int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Lin
 
 struct Packed {
   int T = 0, B = 0;
-  int32_t *ids, *tok_req, *tok_pos, *tok_slot, *tok_part, *cu_q, *kv_base, *pt_off, *req_chunks, *page_table;
+  int32_t *ids, *tok_req, *tok_pos, *tok_slot, *tok_part, *cu_q, *kv_base, *pt_off, *req_chunks, *req_chunk_keys, *page_table;
   int4* items;
-  int n_items = 0, chunk_keys = 0;
+  int n_items = 0;
   bool any_split = false;
   // host views
   int32_t *h_cu_q, *h_kv_base;
@@ -204,6 +204,8 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
   int32_t* h_base = e->meta_alloc<int32_t>(B, &pk->kv_base);
   int32_t* h_ptoff = e->meta_alloc<int32_t>(B + 1, &pk->pt_off);
   int32_t* h_chunks = e->meta_alloc<int32_t>(B, &pk->req_chunks);
+  int32_t* h_chunk_keys = e->meta_alloc<int32_t>(B, &pk->req_chunk_keys);
+  if (!h_chunk_keys) return SLED_ERR_BATCH_TOO_LARGE;
   if (!h_ids || !h_req || !h_pos || !h_slot || !h_part || !h_cu || !h_base || !h_ptoff || !h_chunks)
     return SLED_ERR_BATCH_TOO_LARGE;
   pk->h_cu_q = h_cu;
@@ -241,32 +243,81 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
     std::memcpy(h_pt + h_ptoff[i], c->pages.data(), sizeof(int32_t) * np);
   }
 
-  // attention work items: (request, KV head, chunk of keys); chunks grow until the item count is near the
-  // machine size and the partial-result rows fit
-  const int64_t target = 2LL * e->n_sm;   // measured: about one item per resident block (two per SM) is best
-  int64_t chunk = 256;
-  for (;;) {
-    int64_t items = 0, rows = 0;
+  // Attention work items: (request, KV head, chunk of keys).  The chunk length is chosen per request.
+  // Few requests (every item can be resident at once, two blocks per SM): a request gets chunks in proportion to
+  // its cost - key tiles, weighted up when it has more than 32 query rows, whose tiles take the tensor pipes
+  // longer - so that all blocks end together.  Many requests: one common chunk length, doubled until the item
+  // count is near the machine size; the hardware hands items out as blocks retire.
+  const int group = e->cfg.n_q_heads / Hkv;
+  const int64_t slots = 2LL * e->n_sm;
+  std::vector<int64_t> chunk_of(B, 256);
+  std::vector<double> cost(B);
+  auto heavy = [&](int i) { return plan[i].n * group > 32; };
+  for (int i = 0; i < B; ++i) {
+    const double passes = (plan[i].n * group + 63) / 64;
+    cost[i] = static_cast<double>((n_keys[i] + 63) / 64) * passes * (heavy(i) ? 1.3 : 1.0);
+  }
+  auto part_rows_of = [&]() {
+    int64_t rows = 0;
     for (int i = 0; i < B; ++i) {
-      const int64_t nc = (n_keys[i] + chunk - 1) / chunk;
-      items += nc * Hkv;
+      const int64_t nc = (n_keys[i] + chunk_of[i] - 1) / chunk_of[i];
       if (nc > 1) rows += nc * plan[i].n;
     }
-    const bool fits = rows <= e->part_rows_cap;
-    if ((items <= 2 * target && fits) || chunk >= (1 << 30)) break;
-    // doubling would still leave enough items, or we must shrink the partial rows
-    int64_t items2 = 0;
-    for (int i = 0; i < B; ++i) items2 += ((n_keys[i] + 2 * chunk - 1) / (2 * chunk)) * Hkv;
-    if (!fits || items2 >= target) chunk *= 2;
-    else break;
+    return rows;
+  };
+  if (static_cast<int64_t>(B) * Hkv <= slots) {
+    // smallest cost per item for which the items still fit the slots (bisection on a monotone count)
+    auto chunks_at = [&](int i, double per_item) {
+      const int64_t tiles = (n_keys[i] + 63) / 64;
+      const int64_t want = static_cast<int64_t>(std::ceil(cost[i] / per_item));
+      return std::max<int64_t>(1, std::min(want, std::max<int64_t>(1, tiles / 4)));   // chunks of at least 4 tiles
+    };
+    auto items_at = [&](double per_item) {
+      int64_t n = 0;
+      for (int i = 0; i < B; ++i) n += chunks_at(i, per_item) * Hkv;
+      return n;
+    };
+    double lo = 1.0, hi = 1.0;
+    for (int i = 0; i < B; ++i) hi = std::max(hi, cost[i]);
+    for (int it = 0; it < 30 && items_at(lo) > slots; ++it) {
+      const double mid = 0.5 * (lo + hi);
+      if (items_at(mid) > slots) lo = mid; else hi = mid;
+    }
+    double per_item = items_at(lo) <= slots ? lo : hi;
+    for (;;) {
+      for (int i = 0; i < B; ++i) {
+        const int64_t tiles = (n_keys[i] + 63) / 64;
+        const int64_t nc = chunks_at(i, per_item);
+        chunk_of[i] = (tiles + nc - 1) / nc * 64;
+      }
+      if (part_rows_of() <= e->part_rows_cap) break;
+      per_item *= 1.5;   // fewer, longer chunks until the partial results fit
+    }
+  } else {
+    int64_t chunk = 256;
+    for (;;) {
+      int64_t items = 0;
+      for (int i = 0; i < B; ++i) {
+        chunk_of[i] = chunk;
+        items += (n_keys[i] + chunk - 1) / chunk * Hkv;
+      }
+      const bool fits = part_rows_of() <= e->part_rows_cap;
+      if ((items <= 2 * slots && fits) || chunk >= (1 << 30)) break;
+      // doubling would still leave enough items, or we must shrink the partial rows
+      int64_t items2 = 0;
+      for (int i = 0; i < B; ++i) items2 += ((n_keys[i] + 2 * chunk - 1) / (2 * chunk)) * Hkv;
+      if (!fits || items2 >= slots) chunk *= 2;
+      else break;
+    }
   }
-  pk->chunk_keys = static_cast<int>(chunk);
-  struct It { int req, kvh, start, count; };
+  struct It { int req, kvh, start, count; double cost; bool heavy; };
   std::vector<It> its;
   int part_rows = 0;
   for (int i = 0; i < B; ++i) {
+    const int64_t chunk = chunk_of[i];
     const int nc = static_cast<int>((n_keys[i] + chunk - 1) / chunk);
     h_chunks[i] = nc;
+    h_chunk_keys[i] = static_cast<int32_t>(std::min<int64_t>(chunk, 1 << 30));
     if (nc > 1) {
       pk->any_split = true;
       for (int tt = h_cu[i]; tt < h_cu[i + 1]; ++tt) {
@@ -277,10 +328,14 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
     for (int c = 0; c < nc; ++c) {
       const int start = static_cast<int>(c * chunk);
       const int cnt = static_cast<int>(std::min<int64_t>(chunk, n_keys[i] - start));
-      for (int kvh = 0; kvh < Hkv; ++kvh) its.push_back({i, kvh, start, cnt});
+      for (int kvh = 0; kvh < Hkv; ++kvh) its.push_back({i, kvh, start, cnt, cost[i] * cnt / static_cast<double>(n_keys[i]), heavy(i)});
     }
   }
-  std::stable_sort(its.begin(), its.end(), [](const It& a, const It& b) { return a.count > b.count; });
+  // heavy items first, then by cost: blocks are handed to the SMs in turn, so an SM's second block is a light one
+  std::stable_sort(its.begin(), its.end(), [](const It& a, const It& b) {
+    if (a.heavy != b.heavy) return a.heavy;
+    return a.cost > b.cost;
+  });
   int4* h_items = e->meta_alloc<int4>(its.size(), &pk->items);
   if (!h_items) return SLED_ERR_BATCH_TOO_LARGE;
   for (size_t i = 0; i < its.size(); ++i) h_items[i] = make_int4(its[i].req, its[i].kvh, its[i].start, its[i].count);
@@ -310,7 +365,7 @@ AttnArgs attn_args(sled_engine* e, const Packed& pk, int layer, const void* q, v
   a.Hkv = e->cfg.n_kv_heads;
   a.h = e->cfg.head_dim;
   a.page_size = e->cfg.page_size;
-  a.chunk_keys = pk.chunk_keys;
+  a.req_chunk_keys = pk.req_chunk_keys;
   a.adtype = e->adtype();
   a.kvdtype = e->cfg.kv_dtype;
   if (!e->kv_maps.empty()) {
@@ -326,7 +381,6 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
   const sled_config& c = e->cfg;
   const int T = pk.T, d = c.d_model, ad = e->adtype();
   int n;
-
   e->mark(K_OTHER);
   n = launch_embed(e->tok_emb, c.weight_dtype, pk.ids, T, d, e->x, e->stream);
   e->count(n, K_OTHER);
@@ -663,7 +717,7 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
 
   // metadata staging: tokens, requests, page table (every page at most once, plus one partial page per request), items
   const size_t max_items = static_cast<size_t>(c.n_kv_heads) * (static_cast<size_t>(c.n_pages) * c.page_size / 256 + c.max_batch + 1);
-  e->meta_cap = 5 * maxT * 4 + 6 * (c.max_batch + 1) * 4 + (static_cast<size_t>(c.n_pages) + c.max_batch) * 4 +
+  e->meta_cap = 5 * maxT * 4 + 7 * (c.max_batch + 1) * 4 + 64 + (static_cast<size_t>(c.n_pages) + c.max_batch) * 4 +
                 max_items * sizeof(int4) + 6 * c.max_batch * 8 + 64 * 16;
   if (cudaMallocHost(reinterpret_cast<void**>(&e->h_meta), e->meta_cap) != cudaSuccess) return fail(SLED_ERR_DEVICE);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->d_meta), e->meta_cap))) return fail(rc);

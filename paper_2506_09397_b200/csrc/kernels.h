@@ -47,9 +47,10 @@ struct AttnArgs {
   const int32_t* tok_req;    // [T]
   const int32_t* tok_part;   // [T] first partial-result row of a token (tokens of split requests only)
   const int32_t* req_chunks; // [B] number of key chunks of a request
+  const int32_t* req_chunk_keys; // [B] keys per chunk of a request (a multiple of 64)
   float* part_acc;           // [rows][Hq][h]
   float* part_ml;            // [rows][Hq][2]
-  int T, Hq, Hkv, h, page_size, chunk_keys;
+  int T, Hq, Hkv, h, page_size;
   int adtype, kvdtype;
   // tensor-core path (bf16 cache, 16-token pages): tensor maps over this layer's K and V pool
   // viewed as [page*Hkv*16 + slot][h], and a device word that records a bounded wait running out
