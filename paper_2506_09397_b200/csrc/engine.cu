@@ -255,7 +255,7 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
   auto heavy = [&](int i) { return plan[i].n * group > 32; };
   for (int i = 0; i < B; ++i) {
     const double passes = (plan[i].n * group + 63) / 64;
-    cost[i] = static_cast<double>((n_keys[i] + 63) / 64) * passes * (heavy(i) ? 1.3 : 1.0);
+    cost[i] = static_cast<double>((n_keys[i] + 63) / 64) * passes * (heavy(i) ? 1.75 : 1.0);
   }
   auto part_rows_of = [&]() {
     int64_t rows = 0;
@@ -270,7 +270,7 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
     auto chunks_at = [&](int i, double per_item) {
       const int64_t tiles = (n_keys[i] + 63) / 64;
       const int64_t want = static_cast<int64_t>(std::ceil(cost[i] / per_item));
-      return std::max<int64_t>(1, std::min(want, std::max<int64_t>(1, tiles / 4)));   // chunks of at least 4 tiles
+      return std::max<int64_t>(1, std::min(want, std::max<int64_t>(1, tiles / 2)));   // chunks of at least 2 tiles
     };
     auto items_at = [&](double per_item) {
       int64_t n = 0;
