@@ -307,9 +307,9 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(AttnArgs a, const __gr
   volatile int* s_abort = &s_abort_mem;
 
   const int warp = threadIdx.x >> 5;
-  pdl_enter();
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
-    *s_abort = *reinterpret_cast<volatile int32_t*>(a.error);
+    *s_abort = 0;
     for (int s = 0; s < kStages; ++s) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_full + 8 * s), "r"(1));
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_empty + 8 * s), "r"(4));   // one arrival per computing warp
@@ -319,8 +319,6 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(AttnArgs a, const __gr
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
   }
   __syncthreads();
-  if (*s_abort != 0) return;   // an earlier kernel gave up (read once, before anyone can change it)
-
   const int4 item = a.items[blockIdx.x];
   ItemCtx c;
   c.req = item.x; c.kvh = item.y; c.key_start = item.z; c.key_count = item.w;
@@ -334,6 +332,12 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(AttnArgs a, const __gr
   c.chunk_idx = c.key_start / a.req_chunk_keys[c.req];
   c.scale = rsqrtf(static_cast<float>(H)) * 1.4426950408889634f;
   const int n_pass = (c.n_rows + 63) / 64;
+  // everything above reads only what the host wrote before the step; the queries and the newest cache entries
+  // come from the preceding kernel
+  pdl_wait();
+  // an earlier kernel that gave up has left a code in *error: the copy-issuing warp's second lane (idle otherwise)
+  // looks, so that nobody waits for this load; every loop below polls the flag
+  if (threadIdx.x == 129 && *reinterpret_cast<volatile int32_t*>(a.error) != 0) *s_abort = 1;
 
   if (warp == 4) {
     if ((threadIdx.x & 31) == 0) {

@@ -52,11 +52,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // bounded wait: false (and *error = code) when the phase did not complete in time
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* error, int code) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* error, int code, volatile int* stop) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (*stop != 0) return false;            // another warp of this block gave up, or an earlier kernel did
     if (clock64() - t0 > kWaitCycles) {
       atomicCAS(error, 0, code);
       return false;
@@ -162,10 +163,8 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
 
   if (threadIdx.x == 0) {
     if (base & 1023u) atomicCAS(error, 0, 5);              // the stage layout below would be wrong: refuse to run
-    *abort_slot = *reinterpret_cast<volatile int32_t*>(error);
+    *abort_slot = (base & 1023u) ? 1 : 0;
   }
-  __syncthreads();
-  if (*abort_slot != 0) return;                           // an earlier CTA gave up: do not start
 
   if (warp == 0 && lane == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
@@ -183,9 +182,12 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
   bool ok = true;
+  // An earlier kernel or CTA that gave up has left a code in *error: stop early then.  The word is read by a
+  // thread that has nothing to do until the accumulator is complete, so the load's latency delays nobody.
+  if (threadIdx.x == 64 && *reinterpret_cast<volatile int32_t*>(error) != 0) *abort_slot = 1;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (lane == 0 && *abort_slot == 0) {
       uint64_t pol_first, pol_last;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_last));
@@ -203,7 +205,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
       for (int kb = pre; kb < nkb; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(bars + 8 * (STAGES + s), ph ^ 1, error, 1)) { ok = false; break; }
+        if (!mbar_wait(bars + 8 * (STAGES + s), ph ^ 1, error, 1, abort_slot)) { ok = false; break; }
         const uint32_t full = bars + 8 * s;
         mbar_expect_tx(full, L::kStageBytes);
         const uint32_t wdst = base + s * L::kStageBytes;
@@ -219,7 +221,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
       for (int kb = 0; kb < nkb; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(bars + 8 * s, ph, error, 2)) { ok = false; break; }
+        if (!mbar_wait(bars + 8 * s, ph, error, 2, abort_slot)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t wsrc = base + s * L::kStageBytes;
         const uint64_t adesc = umma_desc(wsrc), bdesc = umma_desc(wsrc + kWStageBytes);
@@ -232,7 +234,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
     }
   } else {
     const int quad = warp & 3;                      // a warp may only touch tensor-memory lanes 32*(warp%4)..+31
-    if (nkb > 0) ok = mbar_wait(bars + 8 * (2 * STAGES), 0, error, 3);
+    if (nkb > 0) ok = mbar_wait(bars + 8 * (2 * STAGES), 0, error, 3, abort_slot);
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
