@@ -848,6 +848,8 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   const float** h_qptr = e->meta_alloc<const float*>(n_reqs, &d_qptr);
   if (!h_lo || !h_hi || !h_qptr) return rollback(SLED_ERR_BATCH_TOO_LARGE);
   bool staged = false;
+  struct QCopy { float* dst; const float* src; size_t bytes; };
+  std::vector<QCopy> copies;
   {
     size_t row = 0;
     for (int i = 0; i < n_reqs; ++i) {
@@ -864,9 +866,7 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
         else {
           // draft distributions travel on the copy stream while the forward pass runs
           float* dst = e->q_stage + row * c.vocab;
-          if (cudaMemcpyAsync(dst, reqs[i].draft_probs, static_cast<size_t>(reqs[i].k) * c.vocab * 4,
-                              cudaMemcpyHostToDevice, e->copy_stream) != cudaSuccess)
-            return rollback(SLED_ERR_DEVICE);
+          copies.push_back({dst, reqs[i].draft_probs, static_cast<size_t>(reqs[i].k) * c.vocab * 4});
           h_qptr[i] = dst;
           row += reqs[i].k;
           staged = true;
@@ -874,8 +874,13 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
       }
     }
   }
-  if (staged && cudaEventRecord(e->ev_copy, e->copy_stream) != cudaSuccess) return rollback(SLED_ERR_DEVICE);
+  // the step's description goes first: the forward pass waits for it, the draft rows are not needed before the
+  // acceptance kernel (copies in one direction are served in the order they were issued)
   if ((rc = upload_meta(e))) return rollback(rc);
+  for (const QCopy& qc : copies)
+    if (cudaMemcpyAsync(qc.dst, qc.src, qc.bytes, cudaMemcpyHostToDevice, e->copy_stream) != cudaSuccess)
+      return rollback(SLED_ERR_DEVICE);
+  if (staged && cudaEventRecord(e->ev_copy, e->copy_stream) != cudaSuccess) return rollback(SLED_ERR_DEVICE);
 
   // ---- forward + acceptance
   if ((rc = run_forward(e, pk, true))) { cudaStreamSynchronize(e->stream); return rollback(rc); }
