@@ -276,6 +276,249 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// CTA-pair kernel for steps of more than 128 tokens (the tensor-bound regime).
+//
+// Two CTAs of a cluster own two neighbouring 128-row weight tiles and the same token tile; one
+// tcgen05.mma.cta_group::2 (M = 256) drives both SMs' tensor cores.  Each CTA loads its own weight slab and only
+// HALF of the token tile's activations (its tn/2 rows of the N side; the instruction reads the two halves from the
+// two CTAs' shared memory): a stage is 32 KB instead of 48 KB, the activations cross L2 -> SM once per 256 weight
+// rows instead of once per 128, and shared memory is read at about half the rate per flop.
+// The kernel is persistent: one pair per two SMs walks over its units (weight-tile pair, K slice, token tile) - token
+// tile fastest, so the pairs that share a weight slab run at the same time and the second reader finds it in
+// L2 - with the accumulator double-buffered in tensor memory (2 x 256 columns): the epilogue of one unit runs
+// under the main loop of the next.  One CTA per SM by construction (192 KB ring, all 512 tensor-memory columns).
+//   both CTAs : warp 0 loads (TMA without multicast; the bytes are counted on the leader's "full" barrier),
+//               warps 2-5 read their own 128 accumulator rows from tensor memory, store them and hand the
+//               accumulator buffer back to the leader
+//   leader    : warp 1 issues the MMAs and commits every stage to BOTH CTAs' "empty" barriers
+// All waits on mbarriers are bounded as in the kernel above; the two cluster-wide barriers (after set-up, before
+// the tensor memory is freed) are reached by every thread of both CTAs on every path.
+constexpr int kPairTN = 256;
+constexpr int kPairStages = 6;
+constexpr int kPairAStageBytes = 128 * kBlockK * 2;
+constexpr int kPairStageBytes = kWStageBytes + kPairAStageBytes;
+constexpr int kPairTiles = kPairStages * kPairStageBytes;
+constexpr int kPairSmem = kPairTiles + 256;
+constexpr int kPairBars = 2 * kPairStages + 4;   // full[S], empty[S], acc_full[2], acc_empty[2]
+
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t leader_bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(leader_bar), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+// arrives (once the MMAs issued so far have completed) on the barrier at this shared-memory offset in both CTAs
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t leader_address(uint32_t local) {   // the same offset in the leader CTA's shared memory
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(0));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+struct PairUnit { int m_pair, t_tile, split; };
+__device__ __forceinline__ PairUnit pair_unit(int u, int n_t, int n_split) {
+  PairUnit r;
+  r.t_tile = u % n_t;
+  const int q = u / n_t;
+  r.split = q % n_split;
+  r.m_pair = q / n_split;
+  return r;
+}
+
+__global__ void __launch_bounds__(192) tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w,
+                                                      const __grid_constant__ CUtensorMap map_a, int T, int N,
+                                                      int kb_total, int kb_per_split, int n_split, int n_units,
+                                                      float* __restrict__ out, long long split_stride, int32_t* error,
+                                                      TcEpilogue epi) {
+  constexpr int S = kPairStages;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t base = smem_u32(smem_raw);
+  uint8_t* base_ptr = smem_raw;
+  const uint32_t bars = base + kPairTiles;
+  const uint32_t bar_full = bars, bar_empty = bars + 8 * S, bar_acc_full = bars + 16 * S, bar_acc_empty = bars + 16 * S + 16;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kPairTiles + 8 * kPairBars);
+  volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + kPairTiles + 8 * kPairBars + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int n_t = (T + kPairTN - 1) / kPairTN;
+
+  if (threadIdx.x == 0) {
+    if (base & 1023u) atomicCAS(error, 0, 5);
+    *abort_slot = (base & 1023u) ? 1 : 0;
+  }
+  if (warp == 0 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    for (int s = 0; s < 2 * S + 2; ++s) mbar_init(bars + 8 * s, 1);
+    mbar_init(bar_acc_empty, 8);        // the four epilogue warps of both CTAs
+    mbar_init(bar_acc_empty + 8, 8);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // the pair's two accumulator buffers: 2 x 256 fp32 columns x 128 lanes in each CTA
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))),
+                 "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();                                      // both CTAs' barriers exist before anything arrives on them
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  bool ok = true;
+  if (threadIdx.x == 64 && *reinterpret_cast<volatile int32_t*>(error) != 0) *abort_slot = 1;
+
+  if (warp == 0) {
+    if (lane == 0 && *abort_slot == 0) {
+      uint64_t pol_w, pol_last;
+      // a weight slab is read by the pairs of all token tiles at about the same time: no "evict first" here
+      asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol_w));
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_last));
+      const uint32_t leader_full = leader_address(bar_full);
+      int it = 0;                                          // slabs loaded so far, over all units
+      bool waited = false;                                 // griddepcontrol.wait done (before the first activation load)
+      for (int u = pair_id; ok && u < n_units; u += n_pairs) {
+        const PairUnit pu = pair_unit(u, n_t, n_split);
+        const int m_tile = 2 * pu.m_pair + static_cast<int>(rank);
+        const int kb0 = pu.split * kb_per_split;
+        const int nkb = min(kb_per_split, kb_total - kb0);
+        const int t0 = pu.t_tile * kPairTN;
+        const int tn = min(kPairTN, ((T - t0) + 31) & ~31);
+        const int a_row = t0 + static_cast<int>(rank) * (tn >> 1);
+        int kb = 0;
+        if (!waited) {
+          // weights do not depend on the previous kernel: fill the ring with weight slabs, then wait, then the activations
+          const int pre = min(S, nkb);
+          for (int k2 = 0; k2 < pre; ++k2) {
+            if (rank == 0) mbar_expect_tx(bar_full + 8 * k2, 2 * kPairStageBytes);   // this CTA's and the peer's bytes
+            tma_load_2d_pair(base + k2 * kPairStageBytes, &map_w, 0, (m_tile * kb_total + kb0 + k2) * kBlockM, leader_full + 8 * k2, pol_w);
+          }
+          pdl_wait_here();
+          waited = true;
+          for (int k2 = 0; k2 < pre; ++k2)
+            tma_load_2d_pair(base + k2 * kPairStageBytes + kWStageBytes, &map_a, (kb0 + k2) * kBlockK, a_row, leader_full + 8 * k2, pol_last);
+          kb = pre;
+          it = pre;
+        }
+        for (; kb < nkb; ++kb, ++it) {
+          const int s = it % S;
+          const uint32_t ph = (it / S) & 1;
+          if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, error, 1, abort_slot)) { ok = false; break; }
+          if (rank == 0) mbar_expect_tx(bar_full + 8 * s, 2 * kPairStageBytes);
+          const uint32_t wdst = base + s * kPairStageBytes;
+          tma_load_2d_pair(wdst, &map_w, 0, (m_tile * kb_total + kb0 + kb) * kBlockM, leader_full + 8 * s, pol_w);
+          tma_load_2d_pair(wdst + kWStageBytes, &map_a, (kb0 + kb) * kBlockK, a_row, leader_full + 8 * s, pol_last);
+        }
+      }
+      if (!waited) pdl_wait_here();
+      // every stage handed back: no arrival from the leader's commits is still on its way to this CTA's barriers
+      for (int j = max(it - S, 0); ok && j < it; ++j)
+        if (!mbar_wait(bar_empty + 8 * (j % S), (j / S) & 1, error, 6, abort_slot)) ok = false;
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      int it = 0, iter = 0;
+      for (int u = pair_id; ok && u < n_units; u += n_pairs, ++iter) {
+        const PairUnit pu = pair_unit(u, n_t, n_split);
+        const int kb0 = pu.split * kb_per_split;
+        const int nkb = min(kb_per_split, kb_total - kb0);
+        const int t0 = pu.t_tile * kPairTN;
+        const int tn = min(kPairTN, ((T - t0) + 31) & ~31);
+        // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = tn, M = 256 over the pair
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(tn >> 3) << 17) |
+                               (static_cast<uint32_t>(256 >> 4) << 24);
+        const int b = iter & 1;
+        // the epilogue warps of both CTAs have read what the unit before last left in this buffer
+        if (!mbar_wait(bar_acc_empty + 8 * b, ((iter >> 1) & 1) ^ 1, error, 7, abort_slot)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t acc = tmem_base + static_cast<uint32_t>(b * kPairTN);
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % S;
+          const uint32_t ph = (it / S) & 1;
+          if (!mbar_wait(bar_full + 8 * s, ph, error, 2, abort_slot)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t wsrc = base + s * kPairStageBytes;
+          const uint64_t adesc = umma_desc(wsrc), bdesc = umma_desc(wsrc + kWStageBytes);
+#pragma unroll
+          for (int kk = 0; kk < kBlockK / 16; ++kk)
+            umma_bf16_pair(acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+          umma_commit_pair(bar_empty + 8 * s);          // the stage is free in both CTAs once these MMAs have read it
+        }
+        if (ok) umma_commit_pair(bar_acc_full + 8 * b);  // this unit's accumulators are complete, in both CTAs
+      }
+    }
+  } else {
+    const int quad = warp & 3;
+    const uint32_t leader_acc_empty = leader_address(bar_acc_empty);
+    int iter = 0;
+    for (int u = pair_id; u < n_units; u += n_pairs, ++iter) {
+      const PairUnit pu = pair_unit(u, n_t, n_split);
+      const int m_tile = 2 * pu.m_pair + static_cast<int>(rank);
+      const int t0 = pu.t_tile * kPairTN;
+      const int tn = min(kPairTN, ((T - t0) + 31) & ~31);
+      const int b = iter & 1;
+      if (ok) ok = mbar_wait(bar_acc_full + 8 * b, (iter >> 1) & 1, error, 3, abort_slot);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int n = m_tile * kBlockM + quad * 32 + lane;
+      float* dst = out + static_cast<long long>(pu.split) * split_stride;
+      for (int c0 = 0; c0 < tn; c0 += 16) {
+        uint32_t v[16];
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+            : "r"(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(b * kPairTN + c0)));
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        float val[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) val[i] = __uint_as_float(v[i]);
+        emit16(epi, dst, N, T, n, t0 + c0, val);
+      }
+      // this warp is done with the buffer: tell the leader's MMA warp (eight such arrivals free it)
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(leader_acc_empty + 8 * b);
+    }
+  }
+
+  // teardown
+  if (!ok) *abort_slot = 1;
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1 && *abort_slot != 0) {
+    // something timed out: give copies and MMAs still in flight time to land before the memory goes away
+    const long long t1 = clock64();
+    while (clock64() - t1 < 2000000LL) __nanosleep(1000);
+  }
+  cluster_sync_all();                                      // neither CTA leaves while the other may still use its memory
+  if (warp == 1)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+}
+
 // Weights are kept tile by tile: block (m, kb) of the tiled array is the 128 x 64 piece W[128m .. +127][64kb .. +63]
 // as 128 rows of 128 bytes, zero where the matrix ends.  One pipeline stage is then one contiguous 16 KB read, and
 // the stages of a CTA follow each other in memory (DRAM pages are read whole instead of 128 bytes at a time).
@@ -400,6 +643,47 @@ static int launch_split(const CUtensorMap& mw, const CUtensorMap& ma, int T, int
   return err == cudaSuccess ? 1 : -1;
 }
 
+static int launch_pair(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K, int n_split, float* out,
+                       int64_t split_stride, int32_t* error, const TcEpilogue& epi, int n_sm, cudaStream_t s) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e0 = cudaFuncSetAttribute(tc_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmem);
+    if (e0 != cudaSuccess) {
+      std::fprintf(stderr, "sled: shared-memory size of the CTA-pair kernel refused: %s\n", cudaGetErrorString(e0));
+      return -1;
+    }
+    configured = true;
+  }
+  const int kb_total = (K + kBlockK - 1) / kBlockK;
+  const int kb_per = (kb_total + n_split - 1) / n_split;
+  const int n_t = (T + kPairTN - 1) / kPairTN;
+  const int n_units = ((N + kBlockM - 1) / kBlockM / 2) * n_split * n_t;
+  // one pair per two SMs; an odd number of pairs, so that a pair's successive units rotate through the token tiles
+  // (whose widths differ) instead of always getting the same one
+  int n_pairs = std::max(1, n_sm / 2);
+  if (n_pairs > 1 && n_pairs % 2 == 0) --n_pairs;
+  n_pairs = std::min(n_pairs, n_units);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(2 * n_pairs, 1, 1);
+  cfg.blockDim = dim3(192, 1, 1);
+  cfg.dynamicSmemBytes = kPairSmem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;   // a pair = two consecutive blocks
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  const long long stride = split_stride;
+  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_pair_kernel, mw, ma, T, N, kb_total, kb_per, n_split, n_units, out, stride, error, epi);
+  if (err != cudaSuccess)
+    std::fprintf(stderr, "sled: launch of the CTA-pair linear-layer kernel failed: %s\n", cudaGetErrorString(err));
+  return err == cudaSuccess ? 1 : -1;
+}
+
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
                    int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
   if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
@@ -409,6 +693,16 @@ int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split,
   if (T <= 64) return launch_split<64, 4>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (T <= 96) return launch_split<96, 4>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (T <= 128) return launch_split<128, 3>(w.map, a.map[3], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (((w.N + kBlockM - 1) / kBlockM) % 2 == 0 && (w.K + kBlockK - 1) / kBlockK / n_split >= 1) {
+    static int n_sm = 0;
+    if (n_sm == 0) {
+      int dev = 0;
+      cudaDeviceProp prop;
+      if (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess) n_sm = prop.multiProcessorCount;
+    }
+    if (n_sm >= 2)   // weight tiles pair up: persistent CTA pairs, half of the token tile staged by each CTA
+      return launch_pair(w.map, a.map[3], T, w.N, w.K, n_split, out, split_stride, error, epi, n_sm, s);
+  }
   return launch_split<256, 2>(w.map, a.map[4], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
 }
 
