@@ -334,6 +334,9 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
+// Unit u = ((weight-tile pair * K slices) + slice) * token tiles + token tile.  In round r the pair with index q
+// takes unit r * n_pairs + (q + r) % n_pairs: neighbouring pairs work on the token tiles of one weight slab at
+// the same time, and the rotation by r gives every pair a mix of wide and narrow token tiles.
 struct PairUnit { int m_pair, t_tile, split; };
 __device__ __forceinline__ PairUnit pair_unit(int u, int n_t, int n_split) {
   PairUnit r;
@@ -399,7 +402,9 @@ __global__ void __launch_bounds__(192) tc_gemm_pair_kernel(const __grid_constant
       const uint32_t leader_full = leader_address(bar_full);
       int it = 0;                                          // slabs loaded so far, over all units
       bool waited = false;                                 // griddepcontrol.wait done (before the first activation load)
-      for (int u = pair_id; ok && u < n_units; u += n_pairs) {
+      for (int r = 0; ok && r * n_pairs < n_units; ++r) {
+        const int u = r * n_pairs + (pair_id + r) % n_pairs;   // round r, rotated: see pair_unit
+        if (u >= n_units) break;                               // only the last round is incomplete
         const PairUnit pu = pair_unit(u, n_t, n_split);
         const int m_tile = 2 * pu.m_pair + static_cast<int>(rank);
         const int kb0 = pu.split * kb_per_split;
@@ -440,7 +445,9 @@ __global__ void __launch_bounds__(192) tc_gemm_pair_kernel(const __grid_constant
   } else if (warp == 1) {
     if (lane == 0 && rank == 0) {
       int it = 0, iter = 0;
-      for (int u = pair_id; ok && u < n_units; u += n_pairs, ++iter) {
+      for (int r = 0; ok && r * n_pairs < n_units; ++r, ++iter) {
+        const int u = r * n_pairs + (pair_id + r) % n_pairs;
+        if (u >= n_units) break;
         const PairUnit pu = pair_unit(u, n_t, n_split);
         const int kb0 = pu.split * kb_per_split;
         const int nkb = min(kb_per_split, kb_total - kb0);
@@ -473,7 +480,9 @@ __global__ void __launch_bounds__(192) tc_gemm_pair_kernel(const __grid_constant
     const int quad = warp & 3;
     const uint32_t leader_acc_empty = leader_address(bar_acc_empty);
     int iter = 0;
-    for (int u = pair_id; u < n_units; u += n_pairs, ++iter) {
+    for (int r = 0; r * n_pairs < n_units; ++r, ++iter) {
+      const int u = r * n_pairs + (pair_id + r) % n_pairs;
+      if (u >= n_units) break;
       const PairUnit pu = pair_unit(u, n_t, n_split);
       const int m_tile = 2 * pu.m_pair + static_cast<int>(rank);
       const int t0 = pu.t_tile * kPairTN;
@@ -658,11 +667,7 @@ static int launch_pair(const CUtensorMap& mw, const CUtensorMap& ma, int T, int 
   const int kb_per = (kb_total + n_split - 1) / n_split;
   const int n_t = (T + kPairTN - 1) / kPairTN;
   const int n_units = ((N + kBlockM - 1) / kBlockM / 2) * n_split * n_t;
-  // one pair per two SMs; an odd number of pairs, so that a pair's successive units rotate through the token tiles
-  // (whose widths differ) instead of always getting the same one
-  int n_pairs = std::max(1, n_sm / 2);
-  if (n_pairs > 1 && n_pairs % 2 == 0) --n_pairs;
-  n_pairs = std::min(n_pairs, n_units);
+  const int n_pairs = std::min(std::max(1, n_sm / 2), n_units);   // one pair per two SMs
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(2 * n_pairs, 1, 1);
   cfg.blockDim = dim3(192, 1, 1);
