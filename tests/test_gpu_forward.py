@@ -202,6 +202,39 @@ def test_large_step_uses_several_token_tiles():
     eng.shutdown()
 
 
+def test_large_step_ragged_matrix_shapes():
+    # more than 128 tokens with matrices whose row counts are not multiples of the 128-row weight tile and whose
+    # inner sizes are not multiples of the 64-wide k-slab: an even number of weight tiles runs as CTA pairs (QKV: 960
+    # rows -> 8 tiles, the last one half empty), an odd number as single CTAs (O and down: 3 tiles, gate/up: 13,
+    # LM head: 33); the down projection has a k tail (776 = 12 slabs + 8)
+    shape = I.ModelShape("odd_bf16", 2, 320, 5, 5, 64, 776, 4200, 5e5, "bf16", "bf16")
+    w = I.make_weights(shape, seed=6)
+    eng = _engine(shape, w, n_pages=400, max_batch=30, max_k=8, max_step_tokens=300)
+    orc = O.OracleModel(shape, oracle_weights(w))
+    ctxs = list(range(30))
+    for c in ctxs:
+        p = I.make_prompt(shape.vocab, 2 + (5 * c) % 23, 6, c)
+        eng.prefill(c, p)
+        if c % 7 == 0:
+            orc.prefill(c, p)
+    reqs = [(c,) + tuple(I.make_drafts(shape.vocab, 5 + c % 4, 6, c)) for c in ctxs]
+    T = sum(len(d) + 1 for _, d, _ in reqs)
+    assert T > 128
+    eng.set_commit(False)
+    got = eng.verify_batch([(c, d.numpy(), q.numpy()) for c, d, q in reqs], 5)
+    glog = eng.logits(T)
+    row = 0
+    for (c, d, q), g in zip(reqs, got):
+        k = len(d)
+        if c in orc.ctx:
+            st, n_acc, nxt, ol, mg = orc.verify(c, d.numpy(), q.numpy(), 5, commit=False)
+            assert np.max(np.abs(glog[row:row + k + 1] - ol)) <= 2e-2
+            st2, n2, x2, _ = O.accept(glog[row:row + k + 1], q.numpy(), d.numpy(), 1.0, False, 5, c, orc.ctx[c].n_kv)
+            assert (n2, x2, 0) == g
+        row += k + 1
+    eng.shutdown()
+
+
 def test_edge_batches():
     # empty batch, a batch of plain decoding steps (k = 0 everywhere), the largest allowed batch, page reuse
     shape = I.TINY
