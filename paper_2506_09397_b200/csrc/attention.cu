@@ -90,6 +90,11 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(AttnArgs a) {
           const int64_t off = ((static_cast<int64_t>(page) * a.Hkv + kvh) * a.page_size + kk % a.page_size) * H + cv * EPV;
           load_row_chunk<KT>(kpool + off, &Ks[kr][cv * EPV]);
           load_row_chunk<KT>(vpool + off, &Vs[kr][cv * EPV]);
+        } else {
+          // past the chunk: these rows are masked below, but their probability 0 still multiplies what is stored
+          // here, and shared memory left by an earlier block may hold NaN
+#pragma unroll
+          for (int z = 0; z < EPV; ++z) { Ks[kr][cv * EPV + z] = 0.f; Vs[kr][cv * EPV + z] = 0.f; }
         }
       }
       __syncthreads();

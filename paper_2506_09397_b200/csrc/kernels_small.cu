@@ -64,7 +64,16 @@ int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t spli
                        float eps, int T, int d, void* out, int adtype, cudaStream_t s) {
   if (T <= 0) return 0;
   if (!partial) n_split = 0;
-  const int nt = d >= 4096 ? 1024 : (d >= 2048 ? 512 : 256);   // d is a multiple of 8 (checked at init)
+  int nt = d >= 4096 ? 1024 : (d >= 2048 ? 512 : 256);   // d is a multiple of 8 (checked at init)
+  // many tokens: smaller blocks, so that all of them are resident at once (2048 threads per SM) instead of running
+  // as a full wave followed by a short one
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    cudaDeviceProp prop;
+    n_sm = (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess) ? prop.multiProcessorCount : 1;
+  }
+  while (nt > 128 && static_cast<long long>(T) * nt > 2048LL * n_sm) nt /= 2;
   if (wdtype == BF16 && adtype == BF16)
     SLED_LAUNCH_PDL((add_rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16>), dim3(T), dim3(nt), 0, s, x, partial, n_split,
                     split_stride, static_cast<const __nv_bfloat16*>(gain), eps, d, static_cast<__nv_bfloat16*>(out));
