@@ -615,9 +615,28 @@ int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K) {
 
 // K slices: as many as keep every CTA of the launch resident at once (two per SM), each with at least 4 slabs;
 // the returned count is the number of slices that actually get work.
+// Above 128 tokens, when the weight tiles pair up, the CTA-pair kernel runs (see tc_gemm_launch): its n_sm / 2 pairs
+// work round by round over (weight-tile pairs x token tiles x slices) units, so the slice count is chosen to
+// minimise rounds x (k-slabs per unit + a unit's fixed cost) + what the consumer pays for adding up the slices
+// (both in units of one k-slab's main-loop time).
+static bool pair_kernel_applies(int T, int N) { return T > 128 && ((N + kBlockM - 1) / kBlockM) % 2 == 0; }
+
 int tc_gemm_split(int T, int N, int K, int n_sm) {
   const int tiles = ((N + kBlockM - 1) / kBlockM) * (T > 128 ? (T + 255) / 256 : 1);
   const int kb_total = (K + kBlockK - 1) / kBlockK;
+  if (pair_kernel_applies(T, N) && n_sm >= 2) {
+    const int n_pairs = n_sm / 2, base = tiles / 2;
+    int best = 1;
+    double best_cost = 0.0;
+    for (int cand = 1; cand <= 8 && cand <= std::max(1, kb_total / 8); ++cand) {
+      const int kb_per = (kb_total + cand - 1) / cand;
+      if ((kb_total + kb_per - 1) / kb_per != cand) continue;          // this count leaves a slice without work
+      const int rounds = (base * cand + n_pairs - 1) / n_pairs;
+      const double cost = rounds * (kb_per + 8.0) + cand * 3e-6 * static_cast<double>(T) * N;
+      if (cand == 1 || cost < best_cost) { best = cand; best_cost = cost; }
+    }
+    return best;
+  }
   int s = std::max(1, (2 * n_sm) / tiles);
   s = std::min(s, std::max(1, kb_total / 4));
   s = std::min(s, 16);
@@ -698,7 +717,7 @@ int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split,
   if (T <= 64) return launch_split<64, 4>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (T <= 96) return launch_split<96, 4>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (T <= 128) return launch_split<128, 3>(w.map, a.map[3], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
-  if (((w.N + kBlockM - 1) / kBlockM) % 2 == 0 && (w.K + kBlockK - 1) / kBlockK / n_split >= 1) {
+  if (pair_kernel_applies(T, w.N)) {
     static int n_sm = 0;
     if (n_sm == 0) {
       int dev = 0;
