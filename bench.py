@@ -98,6 +98,40 @@ class ClockSampler:
         self.gpu = gpu_index
 
     def start(self):
+        # NVML from a thread (a sample every 10 ms from the first millisecond on); nvidia-smi as the fallback, whose
+        # start-up alone can outlast a short timed region
+        self.stop_flag = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            try:
+                uuid = str(torch.cuda.get_device_properties(self.gpu).uuid)
+                h = pynvml.nvmlDeviceGetHandleByUUID(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+            except Exception:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.gpu)
+            mx = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+            bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+
+            def poll():
+                while not self.stop_flag:
+                    try:
+                        clk = pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)
+                        try:
+                            r = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                        except Exception:
+                            r = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                        self.rows.append([str(self.gpu), str(clk), str(mx), "", ""] +
+                                         ["Active" if r & bits[n] else "Not Active" for n in
+                                          ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")])
+                    except Exception:
+                        pass
+                    time.sleep(0.01)
+
+            self.thread = threading.Thread(target=poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.thread = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
                                           "-lms", "50", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
@@ -110,6 +144,9 @@ class ClockSampler:
             self.rows.append([x.strip() for x in line.split(",")])
 
     def stop(self):
+        self.stop_flag = True
+        if getattr(self, "thread", None):
+            self.thread.join(timeout=1)
         if self.proc:
             self.proc.terminate()
             try:
