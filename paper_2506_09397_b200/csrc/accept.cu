@@ -13,9 +13,7 @@ namespace sled {
 
 namespace {
 
-constexpr int kThreads = 1024;
 constexpr int kVec = 4;                       // consecutive vocabulary entries per thread per tile
-constexpr int kTile = kThreads * kVec;        // 4096 entries per tile
 constexpr int kMaxTiles = 1024;               // vocabularies up to 4M entries
 
 enum { ST_OK = 0, ST_NONFINITE = -8 };
@@ -65,6 +63,7 @@ __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v)
 }
 
 // block-wide sum, result to every thread; scratch holds 32 values
+template <int kThreads>
 __device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v, unsigned long long* scratch) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   v = warp_sum_u64(v);
@@ -106,7 +105,9 @@ __device__ __forceinline__ void cluster_barrier() {
 // One cluster of C blocks per request; block `rank` owns a contiguous run of 4096-entry vocabulary tiles.
 // Per examined row the blocks exchange (maximum, argmax, finiteness), then the integer sums, through
 // each other's shared memory; every block then takes the same decision from the same numbers.
+template <int kThreads>
 __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a, int C) {
+  constexpr int kTile = kThreads * kVec;        // entries per tile: 4096 with 1024 threads, 2048 with 512
   __shared__ Shared sh;
   pdl_enter();
   const int req = blockIdx.x / C, rank = blockIdx.x % C;
@@ -222,7 +223,7 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a, int C) {
     } else {
       for (int v = v_lo + threadIdx.x; v < v_hi; v += kThreads) zsum += fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
     }
-    unsigned long long Z = block_sum_u64(zsum, sh.sum_scratch);
+    unsigned long long Z = block_sum_u64<kThreads>(zsum, sh.sum_scratch);
     if (C > 1) {
       if (threadIdx.x < C)
         asm volatile("st.shared::cluster.b64 [%0], %1;" ::"r"(map_to_rank(smem_addr(&sh.x_sum[xphase][rank]), threadIdx.x)), "l"(Z) : "memory");
@@ -378,12 +379,8 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a, int C) {
 
 }  // namespace
 
-int launch_accept(const AcceptArgs& a, cudaStream_t s) {
-  if (a.B <= 0) return 0;
-  if (a.V > kTile * kMaxTiles) return -1;
-  // blocks per request: enough to occupy the machine when the batch is small
-  int C = 1;
-  while (C < kMaxCluster && a.B * C < 128 && (a.V + kTile - 1) / kTile >= 2 * C) C *= 2;
+template <int kThreads>
+static int launch_accept_t(const AcceptArgs& a, int C, cudaStream_t s) {
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(a.B * C, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -398,7 +395,31 @@ int launch_accept(const AcceptArgs& a, cudaStream_t s) {
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, accept_kernel, a, C) == cudaSuccess ? 1 : -1;
+  return cudaLaunchKernelEx(&cfg, accept_kernel<kThreads>, a, C) == cudaSuccess ? 1 : -1;
+}
+
+int launch_accept(const AcceptArgs& a, cudaStream_t s) {
+  if (a.B <= 0) return 0;
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    cudaDeviceProp prop;
+    n_sm = (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess) ? prop.multiProcessorCount : 1;
+  }
+  // Small batches: blocks of 1024 threads, as many blocks per request (a cluster) as it takes to occupy the machine.
+  // Large batches: blocks of 512 threads - four fit an SM instead of one (registers), so several requests hide each
+  // other's latencies - and two blocks per request while that still leaves every block resident or nearly so.
+  if (a.B * kMaxCluster >= 2 * n_sm && a.V <= 512 * kVec * kMaxTiles) {
+    constexpr int kTile = 512 * kVec;
+    int C = 1;
+    while (C < kMaxCluster && a.B * C < 6 * n_sm && (a.V + kTile - 1) / kTile >= 2 * C) C *= 2;
+    return launch_accept_t<512>(a, C, s);
+  }
+  constexpr int kTile = 1024 * kVec;
+  if (a.V > kTile * kMaxTiles) return -1;
+  int C = 1;
+  while (C < kMaxCluster && a.B * C < 128 && (a.V + kTile - 1) / kTile >= 2 * C) C *= 2;
+  return launch_accept_t<1024>(a, C, s);
 }
 
 }  // namespace sled
