@@ -106,7 +106,7 @@ __device__ __forceinline__ void cluster_barrier() {
 // Per examined row the blocks exchange (maximum, argmax, finiteness), then the integer sums, through
 // each other's shared memory; every block then takes the same decision from the same numbers.
 template <int kThreads>
-__global__ void __launch_bounds__(kThreads) accept_kernel(AcceptArgs a, int C) {
+__global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kernel(AcceptArgs a, int C) {
   constexpr int kTile = kThreads * kVec;        // entries per tile: 4096 with 1024 threads, 2048 with 512
   __shared__ Shared sh;
   pdl_enter();
@@ -407,8 +407,8 @@ int launch_accept(const AcceptArgs& a, cudaStream_t s) {
     n_sm = (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess) ? prop.multiProcessorCount : 1;
   }
   // Small batches: blocks of 1024 threads, as many blocks per request (a cluster) as it takes to occupy the machine.
-  // Large batches: blocks of 512 threads - four fit an SM instead of one (registers), so several requests hide each
-  // other's latencies - and two blocks per request while that still leaves every block resident or nearly so.
+  // Large batches: blocks of 512 threads, compiled for three per SM (one 1024-thread block fits otherwise), so that
+  // several requests hide each other's latencies - and two blocks per request (measured best among 1 / 2 / 4).
   if (a.B * kMaxCluster >= 2 * n_sm && a.V <= 512 * kVec * kMaxTiles) {
     constexpr int kTile = 512 * kVec;
     int C = 1;
