@@ -841,8 +841,8 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   }
   Packed pk;
   if ((rc = pack_step(e, plan, false, &pk))) return rollback(rc);
-  uint32_t *d_lo, *d_hi;
-  const float** d_qptr;
+  uint32_t *d_lo = nullptr, *d_hi = nullptr;
+  const float** d_qptr = nullptr;
   uint32_t* h_lo = e->meta_alloc<uint32_t>(n_reqs, &d_lo);
   uint32_t* h_hi = e->meta_alloc<uint32_t>(n_reqs, &d_hi);
   const float** h_qptr = e->meta_alloc<const float*>(n_reqs, &d_qptr);
