@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
 // tile fastest, so the pairs that share a weight slab run at the same time and the second reader finds it in
 // L2 - with the accumulator double-buffered in tensor memory (2 x 256 columns): the epilogue of one unit runs
 // under the main loop of the next.  One CTA per SM by construction (192 KB ring, all 512 tensor-memory columns).
-//   both CTAs : warp 0 loads (TMA without multicast; the bytes are counted on the leader's "full" barrier),
+//   both CTAs : warp 0 loads (plain TMA loads; the bytes are counted on the leader's "full" barrier),
 //               warps 2-5 read their own 128 accumulator rows from tensor memory, store them and hand the
 //               accumulator buffer back to the leader
 //   leader    : warp 1 issues the MMAs and commits every stage to BOTH CTAs' "empty" barriers
@@ -317,10 +317,13 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, 
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
       : "memory");
 }
-// arrives (once the MMAs issued so far have completed) on the barrier at this shared-memory offset in both CTAs
+// arrives (once the MMAs issued so far have completed) on the barrier at this shared-memory offset in both CTAs:
+// one commit per CTA, each naming that CTA's barrier by its cluster address
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
+  uint32_t peer_bar;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(peer_bar) : "r"(bar), "r"(1));
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(peer_bar) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
