@@ -176,12 +176,14 @@ int sled_accept_rows(const float* logits, const int32_t* cu_rows, const int32_t*
  * allocation would stall the device, or a caller between two points of a fixed schedule cannot
  * afford the cudaMalloc / cudaFree pair that sled_accept_rows performs for its small device-side
  * description of the batch.  Here that description lives in a fixed array inside the library
- * image: SLED_STATIC_MAX_REQS requests and SLED_STATIC_MAX_ROWS rows at most (about 90 KB, held
- * by every GPU that loads the library until the process ends).  Larger batches are refused with
+ * image: SLED_STATIC_MAX_REQS requests and SLED_STATIC_MAX_ROWS rows at most (just under 69 KB, held
+ * by every GPU that loads the library until the process ends; the call also builds a host image
+ * of that size on the caller's stack).  Larger batches are refused with
  * SLED_ERR_BATCH_TOO_LARGE.  The call allocates nothing on the device and nothing on the host
  * heap; it does not measure time.  Arguments and results are those of sled_accept_rows.
- * The first call on a device looks up the array's device address (with that device current);
- * make that first call before starting any stream capture.  All calls on a device share the one
+ * Every call must be made with the device that holds `logits` current (checked: SLED_ERR_ARG
+ * otherwise).  The first call on a device looks up the array's device address; make that first
+ * call before starting any stream capture, and from one thread.  All calls on a device share the one
  * array and every call rewrites it completely, so two calls must not overlap on the GPU: issue
  * them from one thread, one after the other (the call synchronises `stream` before returning). */
 #define SLED_STATIC_MAX_REQS 1024

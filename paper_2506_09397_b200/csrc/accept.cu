@@ -130,6 +130,8 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     int best_i = 0x7fffffff;
     int bad = 0;
     const bool vec = ((V & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
+    // the draft rows are the caller's memory: any 4-byte aligned address is legal, 16-byte loads need more
+    const bool q_vec = vec && ((reinterpret_cast<uintptr_t>(qbase) & 15) == 0);
     if (vec) {   // four consecutive entries per thread and step (16-byte loads), four steps in flight
       auto look = [&](int v, const float4& x4) {
         const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
@@ -271,9 +273,12 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
         if (vec && v0 + kVec <= V) {
           const float4 z4 = *reinterpret_cast<const float4*>(z + v0);
           zs[0] = z4.x; zs[1] = z4.y; zs[2] = z4.z; zs[3] = z4.w;
-          if (use_q) {
+          if (use_q && q_vec) {
             const float4 q4 = *reinterpret_cast<const float4*>(qrow + v0);
             qs[0] = q4.x; qs[1] = q4.y; qs[2] = q4.z; qs[3] = q4.w;
+          } else if (use_q) {
+#pragma unroll
+            for (int e = 0; e < kVec; ++e) qs[e] = qrow[v0 + e];
           }
         } else {
 #pragma unroll

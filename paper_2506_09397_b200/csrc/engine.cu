@@ -49,6 +49,8 @@ struct PlanReq {     // tokens fed for one context in one forward pass
 
 enum Kind { K_LINEAR = 0, K_ATTN = 1, K_ACCEPT = 2, K_OTHER = 3, K_KINDS = 4 };
 
+constexpr int kResultsHead = 4;   // words in front of the per-request results: [0] = device error word
+
 }  // namespace
 
 struct sled_engine {
@@ -84,7 +86,8 @@ struct sled_engine {
   int part_rows_cap = 0;
   float* q_stage = nullptr;
   TcActivation tc_norm, tc_attn, tc_ffn;
-  int32_t* tc_error = nullptr;  // device word set by a tensor-core GEMM whose bounded wait ran out
+  int32_t* tc_error = nullptr;  // device word set by a kernel whose bounded wait ran out: the first word of the
+                                // results block (d_results), so the step's one result copy brings it along
 
   // step metadata: pinned staging + device mirror
   char* h_meta = nullptr;
@@ -698,9 +701,13 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->part_ml), static_cast<size_t>(e->part_rows_cap) * c.n_q_heads * 8))) return fail(rc);
   if (!c.probs_on_device && !c.greedy)
     if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->q_stage), maxT * c.vocab * 4))) return fail(rc);
+  // results block: [0] error word (+3 words of padding), then 3 words per request
+  if (cudaMallocHost(reinterpret_cast<void**>(&e->h_results), sizeof(int32_t) * (kResultsHead + 3 * c.max_batch)) != cudaSuccess)
+    return fail(SLED_ERR_DEVICE);
+  if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->d_results), sizeof(int32_t) * (kResultsHead + 3 * c.max_batch)))) return fail(rc);
+  if ((cudaMemset(e->d_results, 0, sizeof(int32_t) * kResultsHead)) != cudaSuccess) return fail(SLED_ERR_DEVICE);
   if (c.weight_dtype == SLED_BF16) {
-    if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->tc_error), 16))) return fail(rc);
-    if ((cudaMemset(e->tc_error, 0, 16)) != cudaSuccess) return fail(SLED_ERR_DEVICE);
+    e->tc_error = e->d_results;
     if (c.page_size == 16 && (c.head_dim == 64 || c.head_dim == 128)) {
       e->kv_maps.resize(2 * c.n_layers);
       const long long rows = static_cast<long long>(c.n_pages) * c.n_kv_heads * c.page_size;
@@ -721,9 +728,6 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
                 max_items * sizeof(int4) + 6 * c.max_batch * 8 + 64 * 16;
   if (cudaMallocHost(reinterpret_cast<void**>(&e->h_meta), e->meta_cap) != cudaSuccess) return fail(SLED_ERR_DEVICE);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->d_meta), e->meta_cap))) return fail(rc);
-  if (cudaMallocHost(reinterpret_cast<void**>(&e->h_results), sizeof(int32_t) * 3 * c.max_batch) != cudaSuccess)
-    return fail(SLED_ERR_DEVICE);
-  if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->d_results), sizeof(int32_t) * 3 * c.max_batch))) return fail(rc);
   if ((cudaDeviceSynchronize()) != cudaSuccess) return fail(SLED_ERR_DEVICE);
   e->st.pages_total = c.n_pages;
   *out = e;
@@ -821,7 +825,13 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   if (rc) return rc;
   std::vector<int32_t> old_pending(n_reqs);
   for (int i = 0; i < n_reqs; ++i) old_pending[i] = e->kvm->find(ctxs[i])->pending;
+  bool issued = false;   // device work of this call is queued (copies or kernels)
   auto rollback = [&](int code) {
+    if (issued) {        // nothing may still read the staging buffers or write the pages that go back to the pool
+      cudaStreamSynchronize(e->copy_stream);
+      cudaStreamSynchronize(e->stream);
+      cudaGetLastError();
+    }
     for (int i = 0; i < n_reqs; ++i) e->kvm->commit(ctxs[i], 0, old_pending[i]);
     return code;
   };
@@ -861,6 +871,7 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
         const bool on_device = cudaPointerGetAttributes(&attr, reqs[i].draft_probs) == cudaSuccess &&
                                attr.type == cudaMemoryTypeDevice;
         cudaGetLastError();
+        if (on_device && attr.device != c.device_index) return rollback(SLED_ERR_ARG);   // another GPU's memory
         if (on_device) h_qptr[i] = reqs[i].draft_probs;   // read in place by the acceptance kernel
         else if (!e->q_stage) return rollback(SLED_ERR_ARG);  // engine was created for device-resident rows only
         else {
@@ -876,6 +887,7 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   }
   // the step's description goes first: the forward pass waits for it, the draft rows are not needed before the
   // acceptance kernel (copies in one direction are served in the order they were issued)
+  issued = true;
   if ((rc = upload_meta(e))) return rollback(rc);
   for (const QCopy& qc : copies)
     if (cudaMemcpyAsync(qc.dst, qc.src, qc.bytes, cudaMemcpyHostToDevice, e->copy_stream) != cudaSuccess)
@@ -883,7 +895,7 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   if (staged && cudaEventRecord(e->ev_copy, e->copy_stream) != cudaSuccess) return rollback(SLED_ERR_DEVICE);
 
   // ---- forward + acceptance
-  if ((rc = run_forward(e, pk, true))) { cudaStreamSynchronize(e->stream); return rollback(rc); }
+  if ((rc = run_forward(e, pk, true))) return rollback(rc);
   if (staged && cudaStreamWaitEvent(e->stream, e->ev_copy, 0) != cudaSuccess) return rollback(SLED_ERR_DEVICE);
   AcceptArgs aa{};
   aa.logits = e->logits;
@@ -893,7 +905,7 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   aa.ctx_lo = d_lo;
   aa.ctx_hi = d_hi;
   aa.pos0 = pk.kv_base;
-  aa.results = e->d_results;
+  aa.results = e->d_results + kResultsHead;
   aa.B = n_reqs;
   aa.V = c.vocab;
   aa.inv_tau = 1.0f / c.temperature;
@@ -901,17 +913,23 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   aa.seed = seed;
   e->mark(K_ACCEPT);
   int n = launch_accept(aa, e->stream);
-  if (n < 0) { cudaStreamSynchronize(e->stream); return rollback(SLED_ERR_DEVICE); }
+  if (n < 0) return rollback(SLED_ERR_DEVICE);
   e->count(n, K_ACCEPT);
   e->mark(K_OTHER);
-  cudaError_t err = cudaMemcpyAsync(e->h_results, e->d_results, sizeof(int32_t) * 3 * n_reqs, cudaMemcpyDeviceToHost, e->stream);
+  cudaError_t err = cudaMemcpyAsync(e->h_results, e->d_results, sizeof(int32_t) * (kResultsHead + 3 * n_reqs),
+                                    cudaMemcpyDeviceToHost, e->stream);
   if (err == cudaSuccess) err = cudaStreamSynchronize(e->stream);
   if (err == cudaSuccess) err = cudaGetLastError();
   if (err != cudaSuccess) {
     std::fprintf(stderr, "sled: verification step failed on the device: %s\n", cudaGetErrorString(err));
     return rollback(SLED_ERR_DEVICE);
   }
-  if ((rc = check_tc_error(e))) return rollback(rc);
+  if (e->h_results[0] != 0) {   // a bounded device-side wait ran out somewhere in the step: nothing of it is kept
+    std::fprintf(stderr, "sled: a kernel of the step gave up waiting (code %d)\n", e->h_results[0]);
+    cudaMemsetAsync(e->d_results, 0, sizeof(int32_t), e->stream);
+    cudaStreamSynchronize(e->stream);
+    return rollback(SLED_ERR_DEVICE);
+  }
   e->last_T = pk.T;
   finish_timing(e);
 
@@ -924,9 +942,10 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   e->st.linear_launches_last_step = e->lin_launches;
   e->st.attention_launches_last_step = e->attn_launches;
   for (int i = 0; i < n_reqs; ++i) {
-    results[i].n_accepted = e->h_results[3 * i];
-    results[i].next_token = e->h_results[3 * i + 1];
-    results[i].status = e->h_results[3 * i + 2];
+    const int32_t* r = e->h_results + kResultsHead + 3 * i;
+    results[i].n_accepted = r[0];
+    results[i].next_token = r[1];
+    results[i].status = r[2];
     if (results[i].status == SLED_OK && e->commit) {
       e->kvm->commit(ctxs[i], results[i].n_accepted + 1, results[i].next_token);
       e->st.drafts_accepted += results[i].n_accepted;
@@ -947,8 +966,10 @@ int sled_accept_rows(const float* logits, const int32_t* cu_rows, const int32_t*
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) { cudaGetLastError(); return SLED_ERR_NO_DEVICE; }
   const int rows = cu_rows[n_reqs];
-  if (rows < n_reqs) return SLED_ERR_ARG;
-  if (!greedy && rows > n_reqs && (!q_rows || !drafts)) return SLED_ERR_ARG;
+  if (cu_rows[0] != 0 || rows < n_reqs) return SLED_ERR_ARG;
+  if (rows > n_reqs && (!drafts || (!greedy && !q_rows))) return SLED_ERR_ARG;   // draft ids are read in both modes
+  for (int i = 0; i < n_reqs; ++i)
+    if (cu_rows[i + 1] - cu_rows[i] < 1) return SLED_ERR_ARG;                      // checked before anything is written
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // small per-call device arrays
   std::vector<int32_t> ids(rows, 0), p0(n_reqs);
@@ -1046,6 +1067,7 @@ int sled_attention_ragged(sled_engine* e, int32_t layer, const uint64_t* ctx_ids
   if (n < 0) return SLED_ERR_DEVICE;
   CU_TRY(cudaStreamSynchronize(e->stream));
   CU_TRY(cudaGetLastError());
+  if ((rc = check_tc_error(e))) return rc;
   e->st.kernels_launched += n;
   if (device_ms) CU_TRY(cudaEventElapsedTime(device_ms, e->ev_a, e->ev_b));
   return SLED_OK;

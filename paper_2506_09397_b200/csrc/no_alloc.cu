@@ -17,7 +17,7 @@
 namespace {
 
 // Layout of the block, sized for the stated maxima.  Every GPU that loads the library
-// holds this array (about 90 KB) until the process exits.
+// holds this array (a little over 68 KB; under 69 KB, checked below) until the process exits.
 constexpr int kMaxReqs = SLED_STATIC_MAX_REQS;
 constexpr int kMaxRows = SLED_STATIC_MAX_ROWS;
 struct alignas(256) StaticBlock {
@@ -29,6 +29,8 @@ struct alignas(256) StaticBlock {
   const float* qptr[kMaxReqs];    // device address of each request's draft rows
   int32_t results[3 * kMaxReqs];  // n_accepted, next_token, status
 };
+
+static_assert(sizeof(StaticBlock) < 69 * 1024, "the size stated in sled.h");
 
 // In host code this name only stands for the symbol; it is not a device address.
 static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticBlock)];
@@ -66,25 +68,36 @@ extern "C" int sled_accept_rows_static(const float* logits, const int32_t* cu_ro
     return SLED_ERR_BATCH_TOO_LARGE;
   }
   const int rows = cu_rows[n_reqs];
-  if (rows < n_reqs) return SLED_ERR_ARG;
+  if (cu_rows[0] != 0 || rows < n_reqs) return SLED_ERR_ARG;
   if (rows > kMaxRows) {
     std::fprintf(stderr, "sled_accept_rows_static: %d rows exceed the fixed maximum of %d\n", rows, kMaxRows);
     return SLED_ERR_BATCH_TOO_LARGE;
   }
-  if (!greedy && rows > n_reqs && (!q_rows || !drafts)) return SLED_ERR_ARG;
+  if (rows > n_reqs && (!drafts || (!greedy && !q_rows))) return SLED_ERR_ARG;   // draft ids are read in both modes
+  for (int i = 0; i < n_reqs; ++i)
+    if (cu_rows[i + 1] - cu_rows[i] < 1) return SLED_ERR_ARG;                      // checked before anything is written
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) { cudaGetLastError(); return SLED_ERR_NO_DEVICE; }
+  {
+    // the kernel runs on the current device: the logits must live there (the array's address is per device)
+    int cur = -1;
+    cudaPointerAttributes attr{};
+    if (cudaGetDevice(&cur) != cudaSuccess) return SLED_ERR_NO_DEVICE;
+    const bool ok = cudaPointerGetAttributes(&attr, logits) == cudaSuccess && attr.type == cudaMemoryTypeDevice &&
+                    attr.device == cur;
+    cudaGetLastError();
+    if (!ok) return SLED_ERR_ARG;
+  }
   StaticBlock* dev = nullptr;
   int rc = block_address(&dev);
   if (rc) return rc;
 
-  // host image of the block, built on the stack (nothing is allocated on either side)
+  // host image of the block, built on the stack (nothing is allocated on either side): that much of the caller's stack
   StaticBlock host;
   std::memset(&host, 0, sizeof(host));  // rows the kernel never reads and old results start from zero
   int64_t drow = 0;
   for (int i = 0; i < n_reqs; ++i) {
     const int k = cu_rows[i + 1] - cu_rows[i] - 1;
-    if (k < 0) return SLED_ERR_ARG;
     for (int j = 0; j < k; ++j) {
       const int d = drafts[drow + j];
       if (d < 0 || d >= vocab) return SLED_ERR_TOKEN_RANGE;

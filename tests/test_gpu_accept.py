@@ -90,3 +90,22 @@ def test_degenerate_rows():
     z[3] = 0.0
     got, want = _run_both(z, q, d, [2, 2, 2, 2], 1.0, True, seed=1)
     assert got == want and all(g[1] == 3 for g in got[:3]) and got[3] == (2, 0, 0)   # all-equal row: index 0
+
+
+def test_draft_rows_at_an_odd_address():
+    # draft rows are the caller's memory: a 4-byte aligned address that is not 16-byte aligned must work
+    n, k, V = 8, 3, 4096
+    z, q, d = I.make_accept_rows(n, k, V, tau_draft=1.0, seed=12, sigma=1.5)
+    logits = z.reshape(n * (k + 1), V).contiguous().cuda()
+    cu = [(k + 1) * i for i in range(n + 1)]
+    ctx, pos0 = list(range(50, 50 + n)), [9] * n
+    drafts = d.reshape(-1).numpy()
+    qa = q.reshape(n * k, V).contiguous().cuda()
+    buf = torch.zeros(n * k * V + 1, device="cuda")
+    buf[1:] = qa.reshape(-1)
+    qb = buf[1:].view(n * k, V)
+    assert qb.data_ptr() % 16 == 4
+    want, _ = B.accept_rows(logits, cu, drafts, qa, ctx, pos0, 1.0, False, seed=2)
+    got, _ = B.accept_rows(logits, cu, drafts, qb, ctx, pos0, 1.0, False, seed=2)
+    assert got == want
+    assert any(g[0] < k for g in got)            # some request reached the residual pass that reads the row

@@ -56,3 +56,19 @@ def test_sizes_beyond_the_fixed_maximum_are_refused():
         B.accept_rows_static(logits, cu, np.zeros(8192, np.int32), None, np.zeros(1, np.uint64), np.zeros(1, np.int64),
                              1.0, True, 0)
     assert ei.value.code == B.SLED_ERR_BATCH_TOO_LARGE
+
+
+def test_bad_descriptions_are_refused_before_anything_is_read():
+    V = 8
+    logits = torch.zeros(4, V, device="cuda")
+    ids, p0 = np.zeros(1, np.uint64), np.zeros(1, np.int64)
+    for fn in (lambda *a: B.accept_rows_static(*a), lambda *a: B.accept_rows(*a)[0]):
+        with pytest.raises(B.SledError) as ei:       # drafts are read in greedy mode too: a missing array is an error
+            fn(logits, np.array([0, 3], np.int32), [], None, ids, p0, 1.0, True, 0)
+        assert ei.value.code == B.SLED_ERR_ARG
+        with pytest.raises(B.SledError) as ei:       # the first row offset must be 0
+            fn(logits, np.array([1, 3], np.int32), [0], None, ids, p0, 1.0, True, 0)
+        assert ei.value.code == B.SLED_ERR_ARG
+        with pytest.raises(B.SledError) as ei:       # a request without rows
+            fn(logits, np.array([0, 0], np.int32), [], None, ids, p0, 1.0, True, 0)
+        assert ei.value.code == B.SLED_ERR_ARG
