@@ -79,6 +79,8 @@ def lib():
         L.orc_forward_token.restype = C.c_int
         L.orc_attend_one.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p]
         L.orc_attend_one.restype = None
+        L.orc_round_bf16.argtypes = [C.c_double]
+        L.orc_round_bf16.restype = C.c_float
         L.orc_num_threads.restype = C.c_int
         L.orc_set_threads.argtypes = [C.c_int]
         _lib = L
@@ -141,6 +143,10 @@ def attend_one(q: np.ndarray, keys: np.ndarray, values: np.ndarray) -> np.ndarra
     lib().orc_attend_one(q.ctypes.data, keys.ctypes.data, values.ctypes.data, keys.shape[0], q.shape[0],
                          out.ctypes.data)
     return out
+
+
+def round_bf16(x: float) -> float:
+    return float(lib().orc_round_bf16(float(x)))
 
 
 def num_threads() -> int:

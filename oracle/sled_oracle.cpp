@@ -21,7 +21,8 @@
 //
 // Parity pins live in tests/ (run with -m "not gpu"): Philox known answers and
 // a second implementation, closed forms of the acceptance rule, the chi-square
-// losslessness invariant, and an independent library forward.
+// losslessness invariant, an independent library forward (both evaluation modes of
+// orc_forward_token), and the bf16 rounding against a library conversion incl. ties.
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -65,6 +66,9 @@ struct Tensor {  // a weight array of either storage type, read as double
 }  // namespace
 
 extern "C" {
+
+// The cache format's rounding, exposed so that tests can pin it against a library conversion.
+float orc_round_bf16(double x) { return round_to_bf16(x); }
 
 // ----------------------------------------------------------------- Philox --
 // Philox4x32 with 10 rounds, as defined by Salmon, Moraes, Dror, Shaw,
