@@ -10,7 +10,9 @@
 // <= 32) the warps split each key tile among themselves instead and merge at the end.  S = Q K^T and O += P V use
 // mma.sync.m16n8k16 with fp32 accumulation; the softmax is the usual online form in fp32 with
 // base-2 exponentials.  Each chunk either writes the normalised output (request not split) or
-// its partial (max, normaliser, unnormalised output) for the merge kernel.
+// its partial (max, normaliser, unnormalised output) for the merge kernel.  The cached prefix does not depend on
+// the kernel that runs before this one (only the newest k+1 slots do): its first tiles are requested before the
+// programmatic-launch dependency wait.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -332,41 +334,52 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(AttnArgs a, const __gr
   c.chunk_idx = c.key_start / a.req_chunk_keys[c.req];
   c.scale = rsqrtf(static_cast<float>(H)) * 1.4426950408889634f;
   const int n_pass = (c.n_rows + 63) / 64;
-  // everything above reads only what the host wrote before the step; the queries and the newest cache entries
-  // come from the preceding kernel
-  pdl_wait();
-  // an earlier kernel that gave up has left a code in *error: the copy-issuing warp's second lane (idle otherwise)
-  // looks, so that nobody waits for this load; every loop below polls the flag
-  if (threadIdx.x == 129 && *reinterpret_cast<volatile int32_t*>(a.error) != 0) *s_abort = 1;
+  // Everything above reads only what the host wrote before the step.  The queries and the cache slots of the step's
+  // own tokens (key index >= kv_base) come from the preceding kernel; the cached prefix does not.
 
   if (warp == 4) {
     if ((threadIdx.x & 31) == 0) {
       const int32_t* pages = a.page_table + a.pt_off[c.req];
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-      int it = 0;
-      for (int pass = 0; pass < n_pass && !*s_abort; ++pass) {
-        for (int tile = 0; tile < c.n_tiles; ++tile, ++it) {
-          const int s = it % kStages;
-          if (*s_abort || !mbar_wait(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { *s_abort = 1; break; }
-          const uint32_t bar = bar_full + 8 * s;
-          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(L::kBytes) : "memory");
-          const uint32_t dst = base + s * L::kBytes;
+      auto load_tile = [&](int tile, int s) {
+        const uint32_t bar = bar_full + 8 * s;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(L::kBytes) : "memory");
+        const uint32_t dst = base + s * L::kBytes;
 #pragma unroll
-          for (int p = 0; p < 4; ++p) {
-            int kk = c.key_start + tile * kTile + p * 16;
-            if (kk >= c.key_end) kk = c.key_end - 1;            // past the chunk: re-read a valid page (masked later)
-            const int row = (pages[kk >> 4] * a.Hkv + c.kvh) * 16;
+        for (int p = 0; p < 4; ++p) {
+          int kk = c.key_start + tile * kTile + p * 16;
+          if (kk >= c.key_end) kk = c.key_end - 1;            // past the chunk: re-read a valid page (masked later)
+          const int row = (pages[kk >> 4] * a.Hkv + c.kvh) * 16;
 #pragma unroll
-            for (int hh = 0; hh < L::kHalves; ++hh) {
-              tma_load_2d(dst + hh * L::kSub + p * 2048, &map_k, hh * 64, row, bar, policy);
-              tma_load_2d(dst + L::kKBytes + hh * L::kSub + p * 2048, &map_v, hh * 64, row, bar, policy);
-            }
+          for (int hh = 0; hh < L::kHalves; ++hh) {
+            tma_load_2d(dst + hh * L::kSub + p * 2048, &map_k, hh * 64, row, bar, policy);
+            tma_load_2d(dst + L::kKBytes + hh * L::kSub + p * 2048, &map_v, hh * 64, row, bar, policy);
           }
         }
+      };
+      // tiles that lie wholly inside the cached prefix are requested before the dependency wait (the ring is empty:
+      // nothing to wait for), so the cache streams while the preceding kernel is still writing the new slots
+      const int safe_tiles = c.key_end <= c.kv_base ? c.n_tiles : max(0, c.kv_base - c.key_start) / kTile;
+      const int pre = min(min(kStages, c.n_tiles), safe_tiles);
+      for (int tile = 0; tile < pre; ++tile) load_tile(tile, tile);
+      pdl_wait();
+      int it = pre;
+      for (int pass = 0; pass < n_pass && !*s_abort; ++pass) {
+        for (int tile = pass == 0 ? pre : 0; tile < c.n_tiles; ++tile, ++it) {
+          const int s = it % kStages;
+          if (*s_abort || !mbar_wait(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { *s_abort = 1; break; }
+          load_tile(tile, s);
+        }
       }
+    } else {
+      pdl_wait();
+      // an earlier kernel that gave up has left a code in *error: the copy-issuing warp's second lane (idle
+      // otherwise) looks, so that nobody waits for this load; every loop below polls the flag
+      if (threadIdx.x == 129 && *reinterpret_cast<volatile int32_t*>(a.error) != 0) *s_abort = 1;
     }
   } else {
+    pdl_wait();
     int it = 0;
     float* merge_buf = reinterpret_cast<float*>(base_ptr);
     for (int pass = 0; pass < n_pass; ++pass) {   // no early exit: the warps meet at named barriers inside

@@ -478,7 +478,7 @@ int check_tc_error(sled_engine* e) {
   int32_t v = 0;
   CU_TRY(cudaMemcpy(&v, e->tc_error, sizeof(v), cudaMemcpyDeviceToHost));
   if (v != 0) {
-    std::fprintf(stderr, "sled: a tensor-core GEMM gave up waiting (code %d)\n", v);
+    std::fprintf(stderr, "sled: a kernel gave up waiting (code %d)\n", v);
     cudaMemset(e->tc_error, 0, sizeof(v));
     return SLED_ERR_DEVICE;
   }

@@ -608,7 +608,7 @@ void tc_weight_free(TcWeight* w) { w->ready = false; }
 
 int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K) {
   if (rows % 256) return -1;
-  const int boxes[kTokenTiles] = {32, 64, 96, 128, 256};
+  const int boxes[kTokenTiles] = {32, 64, 96, 128, 160, 256};
   for (int i = 0; i < kTokenTiles; ++i)
     if (make_map(&a->map[i], dev_ptr, rows, K, boxes[i])) return -1;
   a->rows = rows;
@@ -618,14 +618,15 @@ int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K) {
 
 // K slices: as many as keep every CTA of the launch resident at once (two per SM), each with at least 4 slabs;
 // the returned count is the number of slices that actually get work.
-// Above 128 tokens, when the weight tiles pair up, the CTA-pair kernel runs (see tc_gemm_launch): its n_sm / 2 pairs
+// Above 160 tokens, when the weight tiles pair up, the CTA-pair kernel runs (see tc_gemm_launch): its n_sm / 2 pairs
 // work round by round over (weight-tile pairs x token tiles x slices) units, so the slice count is chosen to
 // minimise rounds x (k-slabs per unit + a unit's fixed cost) + what the consumer pays for adding up the slices
 // (both in units of one k-slab's main-loop time).
-static bool pair_kernel_applies(int T, int N) { return T > 128 && ((N + kBlockM - 1) / kBlockM) % 2 == 0; }
+constexpr int kSingleTileMax = 160;   // widest step that one token tile of the single-CTA kernel (two CTAs per SM) holds
+static bool pair_kernel_applies(int T, int N) { return T > kSingleTileMax && ((N + kBlockM - 1) / kBlockM) % 2 == 0; }
 
 int tc_gemm_split(int T, int N, int K, int n_sm) {
-  const int tiles = ((N + kBlockM - 1) / kBlockM) * (T > 128 ? (T + 255) / 256 : 1);
+  const int tiles = ((N + kBlockM - 1) / kBlockM) * (T > kSingleTileMax ? (T + 255) / 256 : 1);
   const int kb_total = (K + kBlockK - 1) / kBlockK;
   if (pair_kernel_applies(T, N) && n_sm >= 2) {
     const int n_pairs = n_sm / 2, base = tiles / 2;
@@ -720,6 +721,7 @@ int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split,
   if (T <= 64) return launch_split<64, 4>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (T <= 96) return launch_split<96, 4>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (T <= 128) return launch_split<128, 3>(w.map, a.map[3], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (T <= kSingleTileMax) return launch_split<160, 3>(w.map, a.map[4], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (pair_kernel_applies(T, w.N)) {
     static int n_sm = 0;
     if (n_sm == 0) {
@@ -730,7 +732,7 @@ int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split,
     if (n_sm >= 2)   // weight tiles pair up: persistent CTA pairs, half of the token tile staged by each CTA
       return launch_pair(w.map, a.map[3], T, w.N, w.K, n_split, out, split_stride, error, epi, n_sm, s);
   }
-  return launch_split<256, 2>(w.map, a.map[4], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  return launch_split<256, 2>(w.map, a.map[5], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
 }
 
 }  // namespace sled

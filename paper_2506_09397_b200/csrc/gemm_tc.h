@@ -16,9 +16,9 @@ struct TcWeight {       // [N][K] bf16 weights, stored as 128 x 64 tiles of 16 K
   bool ready = false;
 };
 
-constexpr int kTokenTiles = 5;
+constexpr int kTokenTiles = 6;
 struct TcActivation {   // [rows][K] bf16, row-major, device memory; rows is a multiple of 256
-  CUtensorMap map[kTokenTiles];   // boxes of 64 (k) x {32, 64, 96, 128, 256} rows
+  CUtensorMap map[kTokenTiles];   // boxes of 64 (k) x {32, 64, 96, 128, 160, 256} rows
   int rows = 0, K = 0;
 };
 

@@ -306,3 +306,33 @@ def test_errors_leave_everything_unchanged():
     with pytest.raises(B.SledError):
         eng.verify_batch([(1, d.numpy(), q.numpy())], 0)
     eng.shutdown()
+
+
+def test_step_between_128_and_160_tokens():
+    # 129..160 tokens: the widest single token tile of the linear layers (160 columns, partly filled)
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=8)
+    eng = _engine(shape, w, n_pages=300, max_batch=20, max_k=8, max_step_tokens=160)
+    orc = O.OracleModel(shape, oracle_weights(w))
+    ctxs = list(range(20))
+    for c in ctxs:
+        p = I.make_prompt(shape.vocab, 4 + (11 * c) % 37, 8, c)
+        eng.prefill(c, p)
+        if c % 6 == 0:
+            orc.prefill(c, p)
+    reqs = [(c,) + tuple(I.make_drafts(shape.vocab, 6 if c % 2 else 7, 8, c)) for c in ctxs]
+    T = sum(len(d) + 1 for _, d, _ in reqs)
+    assert 128 < T <= 160
+    eng.set_commit(False)
+    got = eng.verify_batch([(c, d.numpy(), q.numpy()) for c, d, q in reqs], 3)
+    glog = eng.logits(T)
+    row = 0
+    for (c, d, q), g in zip(reqs, got):
+        k = len(d)
+        if c in orc.ctx:
+            st, n_acc, nxt, ol, mg = orc.verify(c, d.numpy(), q.numpy(), 3, commit=False)
+            assert np.max(np.abs(glog[row:row + k + 1] - ol)) <= 2e-2
+            st2, n2, x2, _ = O.accept(glog[row:row + k + 1], q.numpy(), d.numpy(), 1.0, False, 3, c, orc.ctx[c].n_kv)
+            assert (n2, x2, 0) == g
+        row += k + 1
+    eng.shutdown()
