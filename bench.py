@@ -7,8 +7,12 @@ synthetic device requests, commit / rollback included).
 
 Prints ONE JSON line.  Metric: verified (committed) tokens per second at the Llama-3-8B shape.
 `value` is measured with the draft distributions already in device memory, `e2e` with them in
-pinned host memory (copied in and results copied out inside the timed region).  `roofline` is for
-the tensor-core linear-layer kernel, the dominant one.  `--impl reference` times the CPU oracle.
+pinned host memory (copied in and results copied out inside the timed region).  Drafts come from
+distributions correlated with the target's own logits (`--drafts independent`: from distributions
+that ignore the target).  `roofline` is for the tensor-core linear-layer kernel, the dominant one;
+`kernel_ms` splits an untouched step by kind of kernel from per-launch device timestamps,
+`kernel_ms_serialised` is the same with events between the kernels.  `sweep` repeats the step at
+other batch sizes (fewer steps, no end-to-end leg).  `--impl reference` times the CPU oracle.
 Under torchrun every rank runs its own replica on its own requests (no data-path collective).
 """
 from __future__ import annotations
@@ -60,6 +64,11 @@ def parse_args(argv=None):
                     help="step: the full verification step (the headline); accept / attention: one kernel alone "
                          "on the acceptance-only / attention-only workload")
     ap.add_argument("--tau", type=float, default=1.0)
+    ap.add_argument("--drafts", default="correlated", choices=["correlated", "independent"],
+                    help="correlated: draft distributions built from the target's own logits (rho = 0.8), "
+                         "independent: softmax of N(0,1) logits")
+    ap.add_argument("--sweep", default="1,64,128", help="other batch sizes measured after the headline one")
+    ap.add_argument("--no-sweep", action="store_true")
     return ap.parse_args(argv)
 
 
@@ -198,19 +207,36 @@ def step_bytes(shape, ks, ctx, n_reject: int) -> float:
 
 
 # ------------------------------------------------------------------ oracle arm --
-def oracle_sample_time(shape, weights_host, ks, ctx, seed, which: int, greedy: bool):
-    """Times the CPU oracle on request `which` of the batch.  Returns (seconds, committed tokens, threads)."""
+def _oracle_model(shape, weights_host):
     from oracle import oracle as O
     conv = lambda t: t.numpy() if t.dtype == torch.float32 else t
     w = {k: [conv(t) for t in v] if isinstance(v, list) else conv(v) for k, v in weights_host.items()}
-    orc = O.OracleModel(shape, w)
+    return O, O.OracleModel(shape, w)
+
+
+def oracle_request(O, orc, shape, ks, ctx, seed, which: int, greedy: bool, drafts: str):
+    """Loads request `which` of the batch into the oracle, builds its drafts (untimed) and times its verification.
+    Correlated drafts are made from the oracle's own logits, position by position, with the generator the GPU arm
+    uses on its logits.  Returns (seconds, committed tokens)."""
     K, V = I.make_kv(shape, ctx[which], seed, which)
     orc.load_kv(which, K.float().numpy(), V.float().numpy(), pending=1)
     del K, V
-    d, q = I.make_drafts(shape.vocab, ks[which], seed, which)
+    k = ks[which]
+    if drafts == "independent":
+        d, q = I.make_drafts(shape.vocab, k, seed, which)
+        d, q = d.numpy(), q.numpy()
+    else:
+        c = orc.ctx[which]
+        d, q, tok = np.zeros(k, np.int32), np.zeros((k, shape.vocab), np.float32), c.pending
+        for j in range(k):
+            z = orc.forward_token(c, int(tok), c.n_kv + j)
+            tok, qj = I.correlated_draft(torch.from_numpy(z), seed, which, j)
+            d[j], q[j] = tok, qj.numpy()
     t0 = time.perf_counter()
-    st, n_acc, nxt, _, _ = orc.verify(which, d.numpy(), None if greedy else q.numpy(), seed, 1.0, greedy)
-    return time.perf_counter() - t0, n_acc + 1, O.num_threads()
+    st, n_acc, nxt, _, _ = orc.verify(which, d, None if greedy else q, seed, 1.0, greedy)
+    dt = time.perf_counter() - t0
+    orc.release(which)
+    return dt, n_acc + 1
 
 
 def run_reference(args):
@@ -220,10 +246,11 @@ def run_reference(args):
     shape, ks, ctx, seed = workload(args, 0)
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     w = I.weights_to(I.make_weights(shape, seed, device=dev), "cpu")
+    O, orc = _oracle_model(shape, w)
     which = int(np.argmin(ks))
-    times, toks, threads = [], 0, 1
+    times, toks = [], 0
     for i in range(args.warmup + args.steps):
-        dt, n_tok, threads = oracle_sample_time(shape, w, ks, ctx, seed, which, args.greedy)
+        dt, n_tok = oracle_request(O, orc, shape, ks, ctx, seed, which, args.greedy, args.drafts)
         if i >= args.warmup:
             times.append(dt)
             toks += n_tok
@@ -233,7 +260,7 @@ def run_reference(args):
             "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
             "config": {"workload": workload_name(args, shape, ks, ctx)},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
                              "sample": f"each step = request {which} of the batch alone (k={ks[which]}, "
                                        f"context {ctx[which]}), 1 of {args.batch} requests"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -255,6 +282,175 @@ def aggregate(local_tokens: float, local_ms: float, world: int):
     return float(t.item()), float(m.item())
 
 
+def load_peaks():
+    try:
+        return json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))), "measured"
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+class Point:
+    """One batch size of the step workload on its own engine: contexts with synthetic cache content, per-request
+    drafts (correlated with the target, or independent), and the timing loops."""
+
+    def __init__(self, B, args, shape, w_dev, batch, rank, local_rank, world, stream):
+        self.B, self.args, self.shape, self.Bn, self.world, self.stream = B, args, shape, batch, world, stream
+        sub = argparse.Namespace(**{**vars(args), "batch": batch})
+        _, self.ks, self.ctx, self.seed = workload(sub, rank)
+        self.name = workload_name(sub, shape, self.ks, self.ctx)
+        self.T = sum(k + 1 for k in self.ks)
+        self.dev = f"cuda:{local_rank}"
+        n_pages = sum((c + k + 1 + 15) // 16 for c, k in zip(self.ctx, self.ks)) + 64
+        self.eng = B.Engine(shape, w_dev, n_pages=n_pages, max_batch=batch, max_k=max(self.ks),
+                            max_step_tokens=max(self.T, 16), temperature=1.0, greedy=args.greedy,
+                            device_index=local_rank, stream=stream.cuda_stream)
+        self.eng.shuffle_pages(self.seed)
+        for i in range(batch):
+            K, V = I.make_kv(shape, self.ctx[i], self.seed, i, device=self.dev)
+            self.eng.load_kv(i, K, V, pending=1)
+            del K, V
+        self.res = (B.SledResult * batch)()
+        self.lib = B.lib()
+        self.ctx_ids = np.arange(batch, dtype=np.uint64)
+        self.ctx_len = np.asarray(self.ctx, dtype=np.int64)
+        self.pend = np.ones(batch, dtype=np.int32)
+
+    # -- drafts
+    def independent_drafts(self):
+        d_host, q_dev = [], []
+        for i in range(self.Bn):
+            d, q = I.make_drafts(self.shape.vocab, self.ks[i], self.seed, i, device=self.dev)
+            d_host.append(np.ascontiguousarray(d.cpu().numpy()))
+            q_dev.append(q)
+        return d_host, q_dev
+
+    def correlated_drafts(self):
+        """Draft j+1 of a request is drawn from a distribution built from the target's own logits at that position:
+        k_max untimed greedy passes without commit over the drafts drawn so far, logits copied out after each."""
+        eng, Bn, ks, V = self.eng, self.Bn, self.ks, self.shape.vocab
+        eng.set_sampling(1.0, True)
+        eng.set_commit(False)
+        d_host = [np.zeros(k, np.int32) for k in ks]
+        q_dev = [torch.zeros(k, V, device=self.dev) for k in ks]
+        for j in range(max(ks)):
+            have = [min(j, k) for k in ks]
+            reqs = (self.B.SledRequest * Bn)()
+            for i in range(Bn):
+                reqs[i].ctx_id, reqs[i].k = i, have[i]
+                reqs[i].draft_tokens = d_host[i].ctypes.data if have[i] else None
+            rc = eng.verify_batch_raw(reqs, Bn, 0, self.res)
+            if rc != 0:
+                raise SystemExit(f"draft construction pass failed: {self.B.strerror(rc)}")
+            n_rows = sum(h + 1 for h in have)
+            logits = torch.empty(n_rows, V, device=self.dev)
+            rc = self.lib.sled_debug_copy_logits(eng.h, logits.data_ptr(), n_rows)
+            if rc != 0:
+                raise SystemExit("sled_debug_copy_logits failed")
+            row = 0
+            for i in range(Bn):
+                if ks[i] > j:
+                    d, q = I.correlated_draft(logits[row + j], self.seed, i, j)
+                    d_host[i][j] = d
+                    q_dev[i][j] = q
+                row += have[i] + 1
+            del logits
+        eng.set_sampling(1.0, self.args.greedy)
+        eng.set_commit(True)
+        return d_host, q_dev
+
+    def marshal(self, d_host, qs):
+        reqs = (self.B.SledRequest * self.Bn)()
+        for i in range(self.Bn):
+            reqs[i].ctx_id = i
+            reqs[i].draft_tokens = d_host[i].ctypes.data if self.ks[i] else None
+            reqs[i].draft_probs = None if (self.args.greedy or not self.ks[i]) else qs[i].data_ptr()
+            reqs[i].k = self.ks[i]
+        self._keep = (d_host, qs)
+        return reqs
+
+    # -- steps
+    def one_step(self, reqs, step_seed):
+        rc = self.eng.verify_batch_raw(reqs, self.Bn, step_seed, self.res)
+        if rc != 0:
+            raise SystemExit(f"sled_verify_batch failed: {self.B.strerror(rc)}")
+        committed = 0
+        for i in range(self.Bn):
+            if self.res[i].status != 0:
+                raise SystemExit(f"request {i} came back with status {self.res[i].status}")
+            committed += self.res[i].n_accepted + 1
+        # every context back to where it was (host bookkeeping only), so that all steps do the same work
+        rc = self.lib.sled_debug_truncate_batch(self.eng.h, self.ctx_ids.ctypes.data, self.ctx_len.ctypes.data,
+                                                self.pend.ctypes.data, self.Bn)
+        if rc != 0:
+            raise SystemExit("sled_debug_truncate_batch failed")
+        return committed
+
+    def timed(self, reqs, steps, warmup):
+        for s in range(warmup):
+            self.one_step(reqs, 100 + s)
+        launches0 = self.eng.stats().kernels_launched
+        if self.world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        committed = 0
+        e0.record(self.stream)
+        for s in range(steps):
+            committed += self.one_step(reqs, 1000 + s)
+        e1.record(self.stream)
+        torch.cuda.synchronize()
+        if self.world > 1:
+            torch.distributed.barrier()
+        return committed, e0.elapsed_time(e1), self.eng.stats().kernels_launched - launches0
+
+    def kernel_times(self, reqs, mode, steps=5):
+        """Device time by kind of kernel in extra steps: mode 1 = per-launch timestamps (launches overlap as in the
+        timed steps), mode 2 = events between kernel groups (serialises them)."""
+        self.eng.set_timing(mode)
+        rows, n_rej = [], 0
+        for s in range(steps):
+            self.one_step(reqs, 2000 + s)
+            st = self.eng.stats()
+            rows.append((st.ms_linear, st.ms_attention, st.ms_accept, st.ms_other, st.ms_idle, st.ms_step))
+            n_rej = sum(1 for i in range(self.Bn) if self.res[i].n_accepted < self.ks[i])
+        self.eng.set_timing(0)
+        med = [statistics.median(c) for c in zip(*rows)]
+        names = ("linear", "attention", "accept", "other", "idle", "step")
+        return dict(zip(names, med)), self.eng.stats().linear_launches_last_step, n_rej
+
+    def summary(self, committed, ms, steps, n_rej, peaks):
+        """Whole-step figures of one timed run (this rank)."""
+        sb = step_bytes(self.shape, self.ks, self.ctx, n_rej)
+        step_s = ms / steps / 1e3
+        return {"ms_per_step": ms / steps, "tokens_per_s": committed / (ms / 1e3),
+                "scored_positions_per_s": self.T / step_s,
+                "acceptance_rate": (committed / steps - self.Bn) / max(sum(self.ks), 1),
+                "step_bytes": sb, "frac_of_hbm_peak": sb / step_s / 1e9 / peaks["hbm_gbs"]}
+
+    def linear_roofline(self, km, n_lin, peaks, peak_src):
+        lb, lf = linear_bytes(self.shape, self.T), linear_flops(self.shape, self.T)
+        lin = km["linear"]
+        hbm, tc_s, tc_b = peaks["hbm_gbs"], peaks.get("bf16_tflops_sustained", 1400.0), peaks.get("bf16_tflops", 1590.0)
+        if lb / (hbm * 1e9) >= lf / (tc_s * 1e12):
+            ach = lb / (lin / 1e3) / 1e9
+            roof = {"bound": "hbm", "achieved": ach, "peak": hbm, "unit": "GB/s", "frac": ach / hbm}
+        else:
+            ach = lf / (lin / 1e3) / 1e12
+            roof = {"bound": "tensor", "achieved": ach, "peak": tc_s, "unit": "TFLOP/s", "frac": ach / tc_s,
+                    "frac_of_burst_peak": ach / tc_b, "peak_kind": "sustained (the kernel runs inside a long step)"}
+        roof.update({"kernel": "linear-layer kernel (all linear layers of a step)", "peak_source": peak_src,
+                     "launches_per_step": n_lin, "avg_launch_ms": lin / max(n_lin, 1),
+                     "algorithmic_bytes_per_launch": lb / max(n_lin, 1), "algorithmic_bytes_per_step": lb,
+                     "algorithmic_flops_per_step": lf,
+                     "time_basis": "per-launch device timestamps inside untouched steps: a launch is charged the time "
+                                   "by which it extends the step beyond all earlier launches"})
+        return roof
+
+    def close(self):
+        self.eng.shutdown()
+        torch.cuda.empty_cache()
+
+
 def run_sled(args):
     from paper_2506_09397_b200 import binding as B
     rank = int(os.environ.get("RANK", "0"))
@@ -267,122 +463,42 @@ def run_sled(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     shape, ks, ctx, seed = workload(args, rank)
-    Bn = args.batch
-    T = sum(k + 1 for k in ks)
     dev = f"cuda:{local_rank}"
-
+    peaks, peak_src = load_peaks()
     w = I.make_weights(shape, seed, device=dev)
-    n_pages = sum((c + k + 1 + 15) // 16 for c, k in zip(ctx, ks)) + 64
-    stream = torch.cuda.Stream(device=dev)
-    eng = B.Engine(shape, w, n_pages=n_pages, max_batch=Bn, max_k=max(ks), max_step_tokens=max(T, 16),
-                   temperature=1.0, greedy=args.greedy, device_index=local_rank, stream=stream.cuda_stream)
     need_host_w = (rank == 0 and world == 1 and not args.no_cpu_baseline)
     w_host = I.weights_to(w, "cpu") if need_host_w else None
-    del w
-    torch.cuda.empty_cache()
-    eng.shuffle_pages(seed)
-    for i in range(Bn):
-        K, V = I.make_kv(shape, ctx[i], seed, i, device=dev)
-        eng.load_kv(i, K, V, pending=1)
-        del K, V
-    drafts_host, q_dev, q_host = [], [], []
-    for i in range(Bn):
-        d, q = I.make_drafts(shape.vocab, ks[i], seed, i, device=dev)
-        drafts_host.append(np.ascontiguousarray(d.cpu().numpy()))
-        q_dev.append(q)
-        if not args.no_e2e:
-            q_host.append(q.cpu().pin_memory())
+    stream = torch.cuda.Stream(device=dev)
+    correlated = args.drafts == "correlated" and not args.greedy
+
+    # ---- the headline point
+    pt = Point(B, args, shape, w, args.batch, rank, local_rank, world, stream)
+    Bn, T = pt.Bn, pt.T
+    d_host, q_dev = pt.correlated_drafts() if correlated else pt.independent_drafts()
     torch.cuda.synchronize()
-
-    def marshal(qs):
-        reqs = (B.SledRequest * Bn)()
-        for i in range(Bn):
-            reqs[i].ctx_id = i
-            reqs[i].draft_tokens = drafts_host[i].ctypes.data
-            reqs[i].draft_probs = None if args.greedy else qs[i].data_ptr()
-            reqs[i].k = ks[i]
-        return reqs
-
-    res = (B.SledResult * Bn)()
-    L = B.lib()
-
-    def one_step(reqs, step_seed):
-        rc = eng.verify_batch_raw(reqs, Bn, step_seed, res)
-        if rc != 0:
-            raise SystemExit(f"sled_verify_batch failed: {B.strerror(rc)}")
-        committed = 0
-        for i in range(Bn):
-            if res[i].status != 0:
-                raise SystemExit(f"request {i} came back with status {res[i].status}")
-            committed += res[i].n_accepted + 1
-            L.sled_debug_truncate(eng.h, i, ctx[i], 1)   # same state for every step (host bookkeeping only)
-        return committed
-
-    def timed(reqs, steps, warmup):
-        for s in range(warmup):
-            one_step(reqs, 100 + s)
-        launches0 = eng.stats().kernels_launched
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        committed = 0
-        e0.record(stream)
-        for s in range(steps):
-            committed += one_step(reqs, 1000 + s)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        if world > 1:
-            torch.distributed.barrier()
-        return committed, e0.elapsed_time(e1), eng.stats().kernels_launched - launches0
-
     sampler = ClockSampler(local_rank)
     sampler.start()
-    reqs_dev = marshal(q_dev)
-    committed, ms, launches = timed(reqs_dev, args.steps, args.warmup)
+    reqs_dev = pt.marshal(d_host, q_dev)
+    committed, ms, launches = pt.timed(reqs_dev, args.steps, args.warmup)
     tok_all, ms_all = aggregate(float(committed), ms, world)
     value = tok_all / (ms_all / 1e3)
 
     e2e = None
     if not args.no_e2e:
-        reqs_host = marshal(q_host)
-        c2, ms2, _ = timed(reqs_host, args.steps, args.warmup)
+        q_host = [q.cpu().pin_memory() for q in q_dev]
+        reqs_host = pt.marshal(d_host, q_host)
+        c2, ms2, _ = pt.timed(reqs_host, args.steps, args.warmup)
         t2, m2 = aggregate(float(c2), ms2, world)
-        h2d = 0 if args.greedy else sum(k * shape.vocab * 4 for k in ks)
+        h2d = 0 if args.greedy else sum(k * shape.vocab * 4 for k in pt.ks)
         e2e = {"value": t2 / (m2 / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d + 64 * T,
-               "d2h_bytes_per_step": 12 * Bn, "ms_per_step": m2 / args.steps}
-
+               "d2h_bytes_per_step": 16 + 12 * Bn, "ms_per_step": m2 / args.steps}
+        reqs_dev = pt.marshal(d_host, q_dev)
+        del q_host
     clocks = sampler.stop()   # sampled over the warm-up and timed steps of both measurements
 
-    # device time per kernel kind (events between kernels; extra steps, not the ones behind `value`)
-    eng.set_timing(True)
-    lin_ms, attn_ms, acc_ms, oth_ms, step_ms = [], [], [], [], []
-    n_rej = 0
-    for s in range(5):
-        one_step(reqs_dev, 2000 + s)
-        st = eng.stats()
-        lin_ms.append(st.ms_linear); attn_ms.append(st.ms_attention); acc_ms.append(st.ms_accept)
-        oth_ms.append(st.ms_other); step_ms.append(st.ms_step)
-        n_rej = sum(1 for i in range(Bn) if res[i].n_accepted < ks[i])
-    eng.set_timing(False)
-    st = eng.stats()
-    n_lin = st.linear_launches_last_step
-    lin = statistics.median(lin_ms)
-    peaks = {}
-    try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
-    except Exception:
-        pass
-    hbm_peak = peaks.get("hbm_gbs", 6650.0)
-    tc_peak = peaks.get("bf16_tflops_sustained", 1400.0)
-    peak_src = "measured" if peaks else "fallback"
-    lb, lf = linear_bytes(shape, T), linear_flops(shape, T)
-    if lb / (hbm_peak * 1e9) >= lf / (tc_peak * 1e12):
-        ach = lb / (lin / 1e3) / 1e9
-        roof = {"bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak}
-    else:
-        ach = lf / (lin / 1e3) / 1e12
-        roof = {"bound": "tensor", "achieved": ach, "peak": tc_peak, "unit": "TFLOP/s", "frac": ach / tc_peak}
+    km, n_lin, n_rej = pt.kernel_times(reqs_dev, 1)
+    km_serial, _, _ = pt.kernel_times(reqs_dev, 2, steps=3)
+    roof = pt.linear_roofline(km, n_lin, peaks, peak_src)
     traffic = None
     try:
         import hashlib
@@ -391,35 +507,82 @@ def run_sled(args):
             traffic = TRAFFIC_LINEAR["bytes_per_launch"].get((shape.name, shape.n_layers, Bn))
     except Exception:
         pass
-    roof.update({"traffic": traffic, "algorithmic_bytes_per_launch": lb / max(n_lin, 1), "kernel": "linear-layer kernel (all linear layers of a step)", "peak_source": peak_src,
-                 "launches_per_step": n_lin, "avg_launch_ms": lin / max(n_lin, 1),
-                 "algorithmic_bytes_per_step": lb, "algorithmic_flops_per_step": lf})
-    sb = step_bytes(shape, ks, ctx, n_rej)
+    roof["traffic"] = traffic
+    head = pt.summary(committed, ms, args.steps, n_rej, peaks)
     step_s = ms_all / args.steps / 1e3
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_all / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if shape.weight_dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": workload_name(args, shape, ks, ctx), "tokens_scored_per_step": T,
+            "config": {"workload": pt.name, "tokens_scored_per_step": T,
                        "l2": "inputs larger than L2 (a step streams %.2f GB of weights)" % (2e-9 * shape.streamed_params()),
-                       "draft_distributions": "independent of the target (softmax of N(0,1) logits)",
+                       "draft_distributions": ("target-correlated: draft logits = 0.8 z + 0.6 std(z) noise, z the target's "
+                                               "own logits at that position (untimed passes), q = softmax, d ~ q"
+                                               if correlated else "independent of the target (softmax of N(0,1) logits)"),
                        "kv": "synthetic N(0,1) cache content in permuted 16-token pages"},
             "clocks": clocks, "gpu_launches": int(launches),
             "scored_positions_per_s": T * world / step_s,
-            "acceptance_rate": (committed / args.steps - Bn) / max(sum(ks), 1),
-            "step_hbm": {"algorithmic_bytes": sb, "achieved_GBps": sb / step_s / 1e9,
-                         "frac_of_hbm_peak": sb / step_s / 1e9 / hbm_peak, "peak_source": peak_src},
-            "kernel_ms": {"linear": lin, "attention": statistics.median(attn_ms), "accept": statistics.median(acc_ms),
-                          "other": statistics.median(oth_ms), "step_with_events": statistics.median(step_ms)},
-            "roofline": roof}
+            "acceptance_rate": head["acceptance_rate"],
+            "step_hbm": {"algorithmic_bytes": head["step_bytes"], "achieved_GBps": head["step_bytes"] / step_s / 1e9,
+                         "frac_of_hbm_peak": head["step_bytes"] / step_s / 1e9 / peaks["hbm_gbs"], "peak_source": peak_src},
+            "kernel_ms": km, "kernel_ms_serialised": km_serial, "roofline": roof}
     if e2e:
         line["e2e"] = e2e
+    if correlated and not args.no_sweep:
+        # the same step with drafts that ignore the target (acceptance is then low: nearly every request stops at its
+        # first draft), as a second figure
+        d2, q2 = pt.independent_drafts()
+        r2 = pt.marshal(d2, q2)
+        c_i, ms_i, _ = pt.timed(r2, max(5, args.steps // 2), 3)
+        s_i = pt.summary(c_i, ms_i, max(5, args.steps // 2), Bn, peaks)
+        line["independent_drafts"] = {k: s_i[k] for k in ("ms_per_step", "tokens_per_s", "acceptance_rate", "frac_of_hbm_peak")}
+        del d2, q2, r2
+    del d_host, q_dev, reqs_dev
+    pt.close()
+
+    # ---- other batch sizes of the same workload (fewer steps; no end-to-end leg)
+    sweep = []
+    if not args.no_sweep and world == 1:
+        for b in [int(x) for x in args.sweep.split(",") if x]:
+            if b == args.batch:
+                continue
+            sp = Point(B, args, shape, w, b, rank, local_rank, world, stream)
+            dh, qd = sp.correlated_drafts() if correlated else sp.independent_drafts()
+            torch.cuda.synchronize()
+            smp = ClockSampler(local_rank)
+            smp.start()
+            rq = sp.marshal(dh, qd)
+            n_steps = max(5, args.steps // 2)
+            c_s, ms_s, _ = sp.timed(rq, n_steps, 3)
+            clk = smp.stop()
+            km_s, n_lin_s, n_rej_s = sp.kernel_times(rq, 1, steps=3)
+            entry = {"batch": b, "tokens_scored_per_step": sp.T, "steps": n_steps, "workload": sp.name}
+            entry.update(sp.summary(c_s, ms_s, n_steps, n_rej_s, peaks))
+            entry["kernel_ms"] = km_s
+            r = sp.linear_roofline(km_s, n_lin_s, peaks, peak_src)
+            entry["linear_layers"] = {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac") if k in r}
+            lf = linear_flops(shape, sp.T)
+            tf = lf / (km_s["linear"] / 1e3) / 1e12
+            entry["linear_layers"].update({"tflops": tf, "frac_of_sustained_bf16_peak": tf / peaks.get("bf16_tflops_sustained", 1400.0),
+                                           "frac_of_burst_bf16_peak": tf / peaks.get("bf16_tflops", 1590.0)})
+            entry["clocks"] = clk
+            sweep.append(entry)
+            del dh, qd, rq
+            sp.close()
+        line["sweep"] = sweep
+    del w
+    torch.cuda.empty_cache()
+
     if need_host_w:
-        which = int(np.argmin(ks))
-        dt, n_tok, threads = oracle_sample_time(shape, w_host, ks, ctx, seed, which, args.greedy)
-        line["cpu_baseline"] = {"value": n_tok / dt, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
-                                "sample": f"request {which} of the batch alone (k={ks[which]}, context {ctx[which]}), "
-                                          f"1 of {Bn} requests, one pass"}
-    eng.shutdown()
+        O, orc = _oracle_model(shape, w_host)
+        t_all, tok_all_cpu = 0.0, 0
+        for i in range(Bn):
+            dt, n_tok = oracle_request(O, orc, shape, ks, ctx, seed, i, args.greedy, args.drafts)
+            t_all += dt
+            tok_all_cpu += n_tok
+        line["cpu_baseline"] = {"value": tok_all_cpu / t_all, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+                                "seconds": t_all,
+                                "sample": f"the whole batch of {Bn} requests, one after the other, one pass "
+                                          "(drafts rebuilt from the oracle's own logits by the same generator, untimed)"}
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -427,10 +590,7 @@ def run_sled(args):
 
 
 def _peaks():
-    try:
-        return json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))), "measured"
-    except Exception:
-        return {"hbm_gbs": 6650.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+    return load_peaks()
 
 
 def run_accept_only(args):

@@ -113,9 +113,11 @@ typedef struct sled_stats {
   int32_t pages_total, pages_free, contexts_open;
   int64_t kernels_launched;    /* device kernels launched by this engine so far */
   int64_t kernels_last_step;   /* ... by the last sled_verify_batch */
-  /* device time of the last step by kind, filled when sled_debug_set_timing(1) */
+  /* device time of the last step by kind of kernel, filled while sled_debug_set_timing is on; ms_idle: stretches of
+   * the step in which no kernel ran (mode 1 only) */
   float ms_linear, ms_attention, ms_accept, ms_other, ms_step;
   int32_t linear_launches_last_step, attention_launches_last_step;
+  float ms_idle;
 } sled_stats;
 
 /* ---- the three calls of the verification service ---------------------------------- */
@@ -214,10 +216,17 @@ int sled_debug_read_kv(sled_engine* e, uint64_t ctx_id, int32_t layer, void* K, 
 int sled_debug_copy_logits(sled_engine* e, float* dst, int32_t n_rows);
 /* Sets a context back to n_kv cached tokens (<= its current count) and a pending token. */
 int sled_debug_truncate(sled_engine* e, uint64_t ctx_id, int64_t n_kv, int32_t pending);
+/* The same for n contexts in one call (ctx_ids, n_kv, pending: HOST arrays [n]); stops at the first error. */
+int sled_debug_truncate_batch(sled_engine* e, const uint64_t* ctx_ids, const int64_t* n_kv, const int32_t* pending,
+                              int32_t n);
 /* commit = 0: verification steps leave every context as it was (repeatable timing). */
 int sled_debug_set_commit(sled_engine* e, int32_t commit);
-/* on = 1: record device time per kernel kind into sled_stats (adds events between kernels). */
-int sled_debug_set_timing(sled_engine* e, int32_t on);
+/* Device time per kind of kernel into sled_stats.  mode 0: off.  mode 1: every launch stamps the GPU's global timer
+ * when its first block begins and its last block ends; launches keep overlapping as they do untimed, and a launch
+ * is charged the time by which it extends the step beyond all earlier launches (the parts add up to ms_step).
+ * mode 2: CUDA events between kernel groups, which serialises neighbouring launches (each kernel's stand-alone
+ * duration; the parts add up to more than an untimed step). */
+int sled_debug_set_timing(sled_engine* e, int32_t mode);
 /* Context state: cached tokens, pending token, owned pages (ids into pages_out, up to cap). */
 int sled_debug_query_ctx(sled_engine* e, uint64_t ctx_id, int64_t* n_kv, int32_t* pending, int32_t* n_pages,
                          int32_t* pages_out, int32_t cap);

@@ -23,7 +23,7 @@ SLED_F32, SLED_BF16 = 0, 1
 EXPORTS = (
     "sled_init", "sled_verify_batch", "sled_release", "sled_prefill", "sled_set_sampling", "sled_get_stats",
     "sled_get_stream", "sled_shutdown", "sled_strerror", "sled_accept_rows", "sled_accept_rows_static", "sled_attention_ragged",
-    "sled_debug_load_kv", "sled_debug_read_kv", "sled_debug_copy_logits", "sled_debug_truncate",
+    "sled_debug_load_kv", "sled_debug_read_kv", "sled_debug_copy_logits", "sled_debug_truncate", "sled_debug_truncate_batch",
     "sled_debug_set_commit", "sled_debug_set_timing", "sled_debug_query_ctx", "sled_debug_shuffle_pages",
     "sled_kvm_create", "sled_kvm_destroy", "sled_kvm_open", "sled_kvm_reserve_batch", "sled_kvm_commit",
     "sled_kvm_release", "sled_kvm_query", "sled_kvm_free_pages", "sled_kvm_pack",
@@ -58,7 +58,7 @@ class SledStats(C.Structure):
         (n, C.c_int32) for n in ("pages_total", "pages_free", "contexts_open")] + [
         ("kernels_launched", C.c_int64), ("kernels_last_step", C.c_int64)] + [
         (n, C.c_float) for n in ("ms_linear", "ms_attention", "ms_accept", "ms_other", "ms_step")] + [
-        ("linear_launches_last_step", C.c_int32), ("attention_launches_last_step", C.c_int32)]
+        ("linear_launches_last_step", C.c_int32), ("attention_launches_last_step", C.c_int32), ("ms_idle", C.c_float)]
 
 
 class SledError(RuntimeError):
@@ -97,6 +97,7 @@ def lib():
             "sled_debug_read_kv": (C.c_int, [P, U64, I32, P, P, I32]),
             "sled_debug_copy_logits": (C.c_int, [P, P, I32]),
             "sled_debug_truncate": (C.c_int, [P, U64, I64, I32]),
+            "sled_debug_truncate_batch": (C.c_int, [P, P, P, P, I32]),
             "sled_debug_set_commit": (C.c_int, [P, I32]),
             "sled_debug_set_timing": (C.c_int, [P, I32]),
             "sled_debug_query_ctx": (C.c_int, [P, U64, C.POINTER(I64), C.POINTER(I32), C.POINTER(I32), P, I32]),
@@ -242,8 +243,9 @@ class Engine:
     def set_commit(self, on: bool) -> None:
         _check(lib().sled_debug_set_commit(self.h, int(on)), "sled_debug_set_commit")
 
-    def set_timing(self, on: bool) -> None:
-        _check(lib().sled_debug_set_timing(self.h, int(on)), "sled_debug_set_timing")
+    def set_timing(self, mode: int) -> None:
+        """0 off, 1 device timestamps per launch (overlap untouched), 2 events between kernel groups (serialises)."""
+        _check(lib().sled_debug_set_timing(self.h, int(mode)), "sled_debug_set_timing")
 
     def shuffle_pages(self, seed: int) -> None:
         _check(lib().sled_debug_shuffle_pages(self.h, seed), "sled_debug_shuffle_pages")

@@ -109,6 +109,7 @@ template <int kThreads>
 __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kernel(AcceptArgs a, int C) {
   constexpr int kTile = kThreads * kVec;        // entries per tile: 4096 with 1024 threads, 2048 with 512
   __shared__ Shared sh;
+  StampScope scope(LaunchStamp{a.stamp.begin, a.stamp.end});
   pdl_enter();
   const int req = blockIdx.x / C, rank = blockIdx.x % C;
   const int row0 = a.cu_q[req];

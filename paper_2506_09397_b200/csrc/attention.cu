@@ -42,6 +42,7 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(AttnArgs a) {
   constexpr int EPV = 16 / sizeof(KT);  // storage elements per 16-byte load
   __shared__ __align__(16) float Ks[kTileKeys][H];
   __shared__ __align__(16) float Vs[kTileKeys][H];
+  StampScope scope(LaunchStamp{a.stamp.begin, a.stamp.end});
   pdl_enter();
 
   const int4 item = a.items[blockIdx.x];
@@ -167,6 +168,7 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(AttnArgs a) {
 // Merge of the per-chunk partial results of split requests: grid (T, Hq), h threads.
 template <typename AT>
 __global__ void attn_merge_kernel(AttnArgs a) {
+  StampScope scope(LaunchStamp{a.stamp_merge.begin, a.stamp_merge.end});
   pdl_enter();
   const int t = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
   const int n = a.req_chunks[a.tok_req[t]];

@@ -309,6 +309,8 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(AttnArgs a, const __gr
   volatile int* s_abort = &s_abort_mem;
 
   const int warp = threadIdx.x >> 5;
+  const LaunchStamp stamp{a.stamp.begin, a.stamp.end};
+  stamp_begin(stamp);
   pdl_launch_dependents();
   if (threadIdx.x == 0) {
     *s_abort = 0;
@@ -396,6 +398,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(AttnArgs a, const __gr
     const long long t1 = clock64();
     while (clock64() - t1 < 2000000LL) __nanosleep(1000);
   }
+  stamp_end(stamp);
 }
 
 template <int H>

@@ -48,6 +48,32 @@ __device__ __forceinline__ void pdl_enter() {
   pdl_wait();
 }
 
+// Optional device-side timestamps of a launch (benchmark mode): when the first block began and when the last one
+// ended, in nanoseconds of the GPU's global timer.  Unlike events between kernels they leave the overlap of
+// neighbouring launches (programmatic dependent launch) as it is.  `begin` starts at ~0, `end` at 0; a null
+// pointer switches the stamps off.
+struct LaunchStamp {
+  unsigned long long* begin;
+  unsigned long long* end;
+};
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void stamp_begin(const LaunchStamp& s) {
+  if (s.begin && threadIdx.x == 0 && threadIdx.y == 0) atomicMin(s.begin, global_ns());
+}
+__device__ __forceinline__ void stamp_end(const LaunchStamp& s) {
+  if (s.end && threadIdx.x == 0 && threadIdx.y == 0) atomicMax(s.end, global_ns());
+}
+// stamps the end when the scope is left, whichever return is taken
+struct StampScope {
+  LaunchStamp s;
+  __device__ __forceinline__ explicit StampScope(const LaunchStamp& st) : s(st) { stamp_begin(s); }
+  __device__ __forceinline__ ~StampScope() { stamp_end(s); }
+};
+
 }  // namespace sled
 
 // Launch with the programmatic-serialization attribute (host side).  `kern` must be a concrete

@@ -60,7 +60,8 @@ struct sled_engine {
   bool own_stream = false;
   cudaEvent_t ev_copy = nullptr, ev_a = nullptr, ev_b = nullptr;
   KvManager* kvm = nullptr;
-  bool commit = true, timing = false;
+  bool commit = true;
+  int timing = 0;   // 0 off, 1 device timestamps per launch (overlap untouched), 2 events between kernel groups (serialises)
 
   // device memory
   std::vector<void*> allocs;
@@ -101,6 +102,10 @@ struct sled_engine {
   std::vector<cudaEvent_t> ev_pool;
   std::vector<int> ev_kind;
   size_t ev_used = 0;
+  unsigned long long* d_stamps = nullptr;   // [2][stamp_cap]: begin times, then end times
+  unsigned long long* h_stamps = nullptr;   // pinned mirror
+  std::vector<int> stamp_kind;
+  size_t stamp_cap = 0, stamp_used = 0;
 
   sled_stats st{};
   int64_t launches_step = 0;
@@ -117,8 +122,16 @@ struct sled_engine {
     return reinterpret_cast<T*>(h_meta + off);
   }
 
-  void mark(int kind) {  // timing: an event before every kernel group, tagged with what follows
-    if (!timing || ev_used >= ev_pool.size()) return;
+  Stamp stamp(int kind) {  // timing mode 1: the next launch's pair of timestamp words
+    Stamp st;
+    if (timing != 1 || stamp_used >= stamp_cap) return st;
+    st.begin = d_stamps + stamp_used;
+    st.end = d_stamps + stamp_cap + stamp_used;
+    stamp_kind[stamp_used++] = kind;
+    return st;
+  }
+  void mark(int kind) {  // timing mode 2: an event before every kernel group, tagged with what follows
+    if (timing != 2 || ev_used >= ev_pool.size()) return;
     cudaEventRecord(ev_pool[ev_used], stream);
     ev_kind[ev_used] = kind;
     ++ev_used;
@@ -168,11 +181,16 @@ int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Lin
   const int64_t stride = static_cast<int64_t>(T) * L.N;
   if (!dst && static_cast<size_t>(split) * stride > e->partial_elems) return SLED_ERR_DEVICE;
   e->mark(K_LINEAR);
+  const Stamp st = e->stamp(K_LINEAR);
   int n;
-  if (e->cfg.weight_dtype == SLED_BF16)
-    n = tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_error, epi, e->stream);
-  else
-    n = launch_gemm_simt(A, e->adtype(), L.w, e->cfg.weight_dtype, T, L.N, L.K, split, out, stride, e->stream);
+  if (e->cfg.weight_dtype == SLED_BF16) {
+    TcEpilogue ep = epi;
+    ep.stamp_begin = st.begin;
+    ep.stamp_end = st.end;
+    n = tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_error, ep, e->stream);
+  } else {
+    n = launch_gemm_simt(A, e->adtype(), L.w, e->cfg.weight_dtype, T, L.N, L.K, split, out, stride, e->stream, st);
+  }
   if (n < 0) return SLED_ERR_DEVICE;
   e->count(n, K_LINEAR);
   *split_out = split;
@@ -376,6 +394,8 @@ AttnArgs attn_args(sled_engine* e, const Packed& pk, int layer, const void* q, v
     a.map_v = &e->kv_maps[2 * layer + 1];
     a.error = e->tc_error;
   }
+  a.stamp = e->stamp(K_ATTN);
+  if (pk.any_split) a.stamp_merge = e->stamp(K_ATTN);
   return a;
 }
 
@@ -385,9 +405,9 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
   const int T = pk.T, d = c.d_model, ad = e->adtype();
   int n;
   e->mark(K_OTHER);
-  n = launch_embed(e->tok_emb, c.weight_dtype, pk.ids, T, d, e->x, e->stream);
+  n = launch_embed(e->tok_emb, c.weight_dtype, pk.ids, T, d, e->x, e->stream, e->stamp(K_OTHER));
   e->count(n, K_OTHER);
-  n = launch_rope_table(pk.tok_pos, T, c.head_dim, c.rope_theta, e->rope_cs, e->stream);
+  n = launch_rope_table(pk.tok_pos, T, c.head_dim, c.rope_theta, e->rope_cs, e->stream, e->stamp(K_OTHER));
   e->count(n, K_OTHER);
   int split = 0;           // split count of the partial sums waiting to be added to x
   int64_t stride = 0;
@@ -395,7 +415,7 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
     Layer& L = e->layers[l];
     e->mark(K_OTHER);
     n = launch_add_rmsnorm(e->x, e->partial, split, stride, L.attn_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm,
-                           ad, e->stream);
+                           ad, e->stream, e->stamp(K_OTHER));
     if (n < 0) return SLED_ERR_DEVICE;
     e->count(n, K_OTHER);
     int s_qkv;
@@ -404,7 +424,7 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
     e->mark(K_OTHER);
     n = launch_rope_kv(e->partial, s_qkv, static_cast<int64_t>(T) * L.qkv.N, e->rope_cs, pk.tok_slot, T, c.n_q_heads,
                        c.n_kv_heads, c.head_dim, c.page_size, e->q_buf, ad, e->kpool + e->kv_layer_bytes * l,
-                       e->vpool + e->kv_layer_bytes * l, c.kv_dtype, e->stream);
+                       e->vpool + e->kv_layer_bytes * l, c.kv_dtype, e->stream, e->stamp(K_OTHER));
     if (n < 0) return SLED_ERR_DEVICE;
     e->count(n, K_OTHER);
     e->mark(K_ATTN);
@@ -416,7 +436,7 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
     stride = static_cast<int64_t>(T) * L.o.N;
     e->mark(K_OTHER);
     n = launch_add_rmsnorm(e->x, e->partial, split, stride, L.ffn_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm, ad,
-                           e->stream);
+                           e->stream, e->stamp(K_OTHER));
     e->count(n, K_OTHER);
     int s_gu;
     if (c.weight_dtype == SLED_BF16 && linear_split(e, T, L.gate_up) == 1) {
@@ -431,7 +451,8 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
       rc = run_linear(e, e->act_norm, &e->tc_norm, L.gate_up, T, nullptr, &s_gu);
       if (rc) return rc;
       e->mark(K_OTHER);
-      n = launch_swiglu(e->partial, s_gu, static_cast<int64_t>(T) * L.gate_up.N, T, c.ffn_dim, e->act_ffn, ad, e->stream);
+      n = launch_swiglu(e->partial, s_gu, static_cast<int64_t>(T) * L.gate_up.N, T, c.ffn_dim, e->act_ffn, ad, e->stream,
+                        e->stamp(K_OTHER));
       e->count(n, K_OTHER);
     }
     rc = run_linear(e, e->act_ffn, &e->tc_ffn, L.down, T, nullptr, &split);
@@ -441,7 +462,7 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
   if (need_logits) {
     e->mark(K_OTHER);
     n = launch_add_rmsnorm(e->x, e->partial, split, stride, e->final_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm,
-                           ad, e->stream);
+                           ad, e->stream, e->stamp(K_OTHER));
     e->count(n, K_OTHER);
     int s1;
     int rc = run_linear(e, e->act_norm, &e->tc_norm, e->lm_head, T, e->logits, &s1);
@@ -455,8 +476,38 @@ int upload_meta(sled_engine* e) {
   return SLED_OK;
 }
 
+// Timing mode 1.  Launches overlap (a kernel may begin while its predecessor drains), so a launch is charged the
+// time by which it extends the step beyond everything launched before it: end_i - max(begin_i, latest end so far);
+// stretches in which nothing ran go to ms_idle.  The parts add up to ms_step = last end - first begin.
+int finish_stamps(sled_engine* e) {
+  const size_t n = e->stamp_used, cap = e->stamp_cap;
+  if (n == 0) return SLED_OK;
+  CU_TRY(cudaMemcpy(e->h_stamps, e->d_stamps, sizeof(unsigned long long) * 2 * cap, cudaMemcpyDeviceToHost));
+  double acc[K_KINDS] = {0, 0, 0, 0}, idle = 0.0;
+  unsigned long long first = 0, latest = 0;
+  bool any = false;
+  for (size_t i = 0; i < n; ++i) {
+    const unsigned long long b = e->h_stamps[i], en = e->h_stamps[cap + i];
+    if (en == 0 || b == ~0ull) continue;   // nothing was launched for this slot
+    if (!any) { first = latest = b; any = true; }
+    if (b > latest) idle += static_cast<double>(b - latest);
+    const unsigned long long from = b > latest ? b : latest;
+    if (en > from) acc[e->stamp_kind[i]] += static_cast<double>(en - from);
+    if (en > latest) latest = en;
+  }
+  e->st.ms_linear = static_cast<float>(acc[K_LINEAR] * 1e-6);
+  e->st.ms_attention = static_cast<float>(acc[K_ATTN] * 1e-6);
+  e->st.ms_accept = static_cast<float>(acc[K_ACCEPT] * 1e-6);
+  e->st.ms_other = static_cast<float>(acc[K_OTHER] * 1e-6);
+  e->st.ms_idle = static_cast<float>(idle * 1e-6);
+  e->st.ms_step = static_cast<float>(static_cast<double>(latest - first) * 1e-6);
+  return SLED_OK;
+}
+
 int finish_timing(sled_engine* e) {
-  if (!e->timing || e->ev_used < 2) return SLED_OK;
+  if (e->timing == 1) return finish_stamps(e);
+  e->st.ms_idle = 0.f;
+  if (e->timing != 2 || e->ev_used < 2) return SLED_OK;
   float acc[K_KINDS] = {0, 0, 0, 0};
   for (size_t i = 0; i + 1 < e->ev_used; ++i) {
     float ms = 0.f;
@@ -488,6 +539,11 @@ int check_tc_error(sled_engine* e) {
 void begin_step(sled_engine* e) {
   e->meta_used = 0;
   e->ev_used = 0;
+  e->stamp_used = 0;
+  if (e->timing == 1) {   // begin words to all ones (a minimum is taken), end words to zero (a maximum)
+    cudaMemsetAsync(e->d_stamps, 0xFF, sizeof(unsigned long long) * e->stamp_cap, e->stream);
+    cudaMemsetAsync(e->d_stamps + e->stamp_cap, 0, sizeof(unsigned long long) * e->stamp_cap, e->stream);
+  }
   e->launches_step = 0;
   e->lin_launches = 0;
   e->attn_launches = 0;
@@ -504,6 +560,7 @@ void destroy(sled_engine* e) {
   for (void* p : e->allocs) cudaFree(p);
   if (e->h_meta) cudaFreeHost(e->h_meta);
   if (e->h_results) cudaFreeHost(e->h_results);
+  if (e->h_stamps) cudaFreeHost(e->h_stamps);
   for (auto ev : e->ev_pool) cudaEventDestroy(ev);
   if (e->ev_copy) cudaEventDestroy(e->ev_copy);
   if (e->ev_a) cudaEventDestroy(e->ev_a);
@@ -912,6 +969,7 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   aa.greedy = c.greedy;
   aa.seed = seed;
   e->mark(K_ACCEPT);
+  aa.stamp = e->stamp(K_ACCEPT);
   int n = launch_accept(aa, e->stream);
   if (n < 0) return rollback(SLED_ERR_DEVICE);
   e->count(n, K_ACCEPT);
@@ -1156,23 +1214,41 @@ int sled_debug_truncate(sled_engine* e, uint64_t ctx_id, int64_t n_kv, int32_t p
   return e->kvm->truncate(ctx_id, n_kv, pending);
 }
 
+int sled_debug_truncate_batch(sled_engine* e, const uint64_t* ctx_ids, const int64_t* n_kv, const int32_t* pending,
+                              int32_t n) {
+  if (!e || n < 0 || (n > 0 && (!ctx_ids || !n_kv || !pending))) return SLED_ERR_ARG;
+  for (int32_t i = 0; i < n; ++i) {
+    const int rc = sled_debug_truncate(e, ctx_ids[i], n_kv[i], pending[i]);
+    if (rc) return rc;
+  }
+  return SLED_OK;
+}
+
 int sled_debug_set_commit(sled_engine* e, int32_t commit) {
   if (!e) return SLED_ERR_ARG;
   e->commit = commit != 0;
   return SLED_OK;
 }
 
-int sled_debug_set_timing(sled_engine* e, int32_t on) {
-  if (!e) return SLED_ERR_ARG;
+int sled_debug_set_timing(sled_engine* e, int32_t mode) {
+  if (!e || mode < 0 || mode > 2) return SLED_ERR_ARG;
   cudaSetDevice(e->cfg.device_index);
-  if (on && e->ev_pool.empty()) {
-    const size_t n = 16 + 12 * static_cast<size_t>(e->cfg.n_layers);
+  const size_t n = 16 + 12 * static_cast<size_t>(e->cfg.n_layers);
+  if (mode == 2 && e->ev_pool.empty()) {
     e->ev_pool.resize(n);
     e->ev_kind.assign(n, K_OTHER);
     for (auto& ev : e->ev_pool)
       if (cudaEventCreate(&ev) != cudaSuccess) return SLED_ERR_DEVICE;
   }
-  e->timing = on != 0;
+  if (mode == 1 && !e->d_stamps) {
+    int rc = dmalloc(e, reinterpret_cast<void**>(&e->d_stamps), sizeof(unsigned long long) * 2 * n);
+    if (rc) return rc;
+    if (cudaMallocHost(reinterpret_cast<void**>(&e->h_stamps), sizeof(unsigned long long) * 2 * n) != cudaSuccess)
+      return SLED_ERR_DEVICE;
+    e->stamp_kind.assign(n, K_OTHER);
+    e->stamp_cap = n;
+  }
+  e->timing = mode;
   return SLED_OK;
 }
 

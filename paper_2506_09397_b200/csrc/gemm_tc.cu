@@ -96,6 +96,14 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 
 __device__ __forceinline__ void pdl_wait_here() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// benchmark mode: earliest block start / latest block end of the launch, in ns of the GPU's global timer
+__device__ __forceinline__ void stamp_time(unsigned long long* slot, bool is_end) {
+  if (slot == nullptr || threadIdx.x != 0) return;
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  if (is_end) atomicMax(slot, t); else atomicMin(slot, t);
+}
+
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -154,6 +162,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
   volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * (2 * STAGES + 1) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  stamp_time(epi.stamp_begin, false);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its own prologue
   const int t_tile = blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
   const int kb0 = split * kb_per_split;
@@ -274,6 +283,7 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                  "r"(static_cast<uint32_t>(kTmemCols)) : "memory");
   }
+  stamp_time(epi.stamp_end, true);   // thread 0 is past the block-wide barrier: every warp's work is done
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -365,6 +375,7 @@ __global__ void __launch_bounds__(192) tc_gemm_pair_kernel(const __grid_constant
   volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + kPairTiles + 8 * kPairBars + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  stamp_time(epi.stamp_begin, false);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
@@ -529,6 +540,7 @@ __global__ void __launch_bounds__(192) tc_gemm_pair_kernel(const __grid_constant
   cluster_sync_all();                                      // neither CTA leaves while the other may still use its memory
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  stamp_time(epi.stamp_end, true);
 }
 
 // Weights are kept tile by tile: block (m, kb) of the tiled array is the 128 x 64 piece W[128m .. +127][64kb .. +63]

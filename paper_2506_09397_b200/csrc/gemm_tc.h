@@ -27,6 +27,9 @@ struct TcEpilogue {       // what happens to the finished sums (see emit16 in ge
   int mode = kEpiStore;
   __nv_bfloat16* act_out = nullptr;   // kEpiSwiglu: [T][act_ld] activations for the down projection
   int act_ld = 0;
+  // benchmark mode: device words that receive the time the launch's first block began / its last block ended
+  unsigned long long* stamp_begin = nullptr;
+  unsigned long long* stamp_end = nullptr;
 };
 
 // 2D bf16 tensor map over a row-major [rows][cols] array: boxes of 64 columns x box_rows rows, 128-byte swizzle

@@ -10,18 +10,25 @@ namespace sled {
 
 enum DType { F32 = 0, BF16 = 1 };
 
+// Device addresses that receive a launch's begin / end time (see common.cuh); null members: no stamps.
+struct Stamp {
+  unsigned long long* begin = nullptr;
+  unsigned long long* end = nullptr;
+};
+
 // ---- elementwise / small kernels (kernels_small.cu)
-int launch_embed(const void* table, int wdtype, const int32_t* ids, int T, int d, float* x, cudaStream_t s);
+int launch_embed(const void* table, int wdtype, const int32_t* ids, int T, int d, float* x, cudaStream_t s,
+                 Stamp st = Stamp());
 // x += sum_s partial[s] (if partial), then out = RMSNorm(x) * gain in the activation type
 int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t split_stride, const void* gain, int wdtype,
-                       float eps, int T, int d, void* out, int adtype, cudaStream_t s);
-int launch_rope_table(const int32_t* tok_pos, int T, int h, float theta, float2* cs, cudaStream_t s);
+                       float eps, int T, int d, void* out, int adtype, cudaStream_t s, Stamp st = Stamp());
+int launch_rope_table(const int32_t* tok_pos, int T, int h, float theta, float2* cs, cudaStream_t s, Stamp st = Stamp());
 // sums the QKV partials, rotates Q and K, writes Q to q_out and K, V into their cache slots
 int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, const float2* cs, const int32_t* tok_slot,
                    int T, int Hq, int Hkv, int h, int page_size, void* q_out, int adtype, void* kpool, void* vpool,
-                   int kvdtype, cudaStream_t s);
+                   int kvdtype, cudaStream_t s, Stamp st = Stamp());
 int launch_swiglu(const float* partial, int n_split, int64_t split_stride, int T, int F, void* out, int adtype,
-                  cudaStream_t s);
+                  cudaStream_t s, Stamp st = Stamp());
 // contiguous [n][Hkv][h] <-> paged cache of one layer
 int launch_kv_scatter(const void* src, const int32_t* slots, int n, int Hkv, int h, int page_size, void* pool,
                       int kvdtype, cudaStream_t s);
@@ -30,7 +37,7 @@ int launch_kv_gather(const void* pool, const int32_t* slots, int n, int Hkv, int
 
 // ---- fp32 / generic CUDA-core GEMM (kernels_small.cu): out[s][T][N] = A[T][Kslice_s] . W[N][Kslice_s]^T
 int launch_gemm_simt(const void* A, int adtype, const void* W, int wdtype, int T, int N, int K, int n_split,
-                     float* out, int64_t split_stride, cudaStream_t s);
+                     float* out, int64_t split_stride, cudaStream_t s, Stamp st = Stamp());
 
 // ---- ragged verification attention over the paged cache (attention.cu)
 struct AttnArgs {
@@ -57,6 +64,7 @@ struct AttnArgs {
   const CUtensorMap* map_k = nullptr;
   const CUtensorMap* map_v = nullptr;
   int32_t* error = nullptr;
+  Stamp stamp, stamp_merge;   // of the attention kernel and of the merge kernel that may follow it
 };
 int launch_attention(const AttnArgs& a, cudaStream_t s);
 // tensor-core kernel alone (attention_mma.cu); returns 1 or a negative value
@@ -76,6 +84,7 @@ struct AcceptArgs {
   float inv_tau;
   int greedy;
   uint64_t seed;
+  Stamp stamp;
 };
 int launch_accept(const AcceptArgs& a, cudaStream_t s);
 

@@ -8,21 +8,25 @@
 
 namespace sled {
 
+static inline LaunchStamp dev_stamp(const Stamp& st) { return LaunchStamp{st.begin, st.end}; }
+
 // ------------------------------------------------------------------ embedding --
 template <typename WT>
-__global__ void embed_kernel(const WT* __restrict__ table, const int32_t* __restrict__ ids, int d, float* __restrict__ x) {
+__global__ void embed_kernel(const WT* __restrict__ table, const int32_t* __restrict__ ids, int d, float* __restrict__ x,
+                             LaunchStamp stamp) {
+  StampScope scope(stamp);
   pdl_enter();
   const int t = blockIdx.x;
   const WT* row = table + static_cast<int64_t>(ids[t]) * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) x[static_cast<int64_t>(t) * d + i] = to_f32(row[i]);
 }
 
-int launch_embed(const void* table, int wdtype, const int32_t* ids, int T, int d, float* x, cudaStream_t s) {
+int launch_embed(const void* table, int wdtype, const int32_t* ids, int T, int d, float* x, cudaStream_t s, Stamp st) {
   if (T <= 0) return 0;
   if (wdtype == BF16)
-    SLED_LAUNCH_PDL(embed_kernel<__nv_bfloat16>, dim3(T), dim3(256), 0, s, static_cast<const __nv_bfloat16*>(table), ids, d, x);
+    SLED_LAUNCH_PDL(embed_kernel<__nv_bfloat16>, dim3(T), dim3(256), 0, s, static_cast<const __nv_bfloat16*>(table), ids, d, x, dev_stamp(st));
   else
-    SLED_LAUNCH_PDL(embed_kernel<float>, dim3(T), dim3(256), 0, s, static_cast<const float*>(table), ids, d, x);
+    SLED_LAUNCH_PDL(embed_kernel<float>, dim3(T), dim3(256), 0, s, static_cast<const float*>(table), ids, d, x, dev_stamp(st));
   return 1;
 }
 
@@ -33,8 +37,9 @@ int launch_embed(const void* table, int wdtype, const int32_t* ids, int T, int d
 template <typename WT, typename AT>
 __global__ void add_rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ partial, int n_split,
                                    int64_t split_stride, const WT* __restrict__ gain, float eps, int d,
-                                   AT* __restrict__ out) {
+                                   AT* __restrict__ out, LaunchStamp stamp) {
   __shared__ float scratch[32];
+  StampScope scope(stamp);
   pdl_enter();
   const int64_t base = static_cast<int64_t>(blockIdx.x) * d;
   float ss = 0.f;
@@ -61,7 +66,7 @@ __global__ void add_rmsnorm_kernel(float* __restrict__ x, const float* __restric
 }
 
 int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t split_stride, const void* gain, int wdtype,
-                       float eps, int T, int d, void* out, int adtype, cudaStream_t s) {
+                       float eps, int T, int d, void* out, int adtype, cudaStream_t s, Stamp st) {
   if (T <= 0) return 0;
   if (!partial) n_split = 0;
   int nt = d >= 4096 ? 1024 : (d >= 2048 ? 512 : 256);   // d is a multiple of 8 (checked at init)
@@ -76,10 +81,10 @@ int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t spli
   while (nt > 128 && static_cast<long long>(T) * nt > 2048LL * n_sm) nt /= 2;
   if (wdtype == BF16 && adtype == BF16)
     SLED_LAUNCH_PDL((add_rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16>), dim3(T), dim3(nt), 0, s, x, partial, n_split,
-                    split_stride, static_cast<const __nv_bfloat16*>(gain), eps, d, static_cast<__nv_bfloat16*>(out));
+                    split_stride, static_cast<const __nv_bfloat16*>(gain), eps, d, static_cast<__nv_bfloat16*>(out), dev_stamp(st));
   else if (wdtype == F32 && adtype == F32)
     SLED_LAUNCH_PDL((add_rmsnorm_kernel<float, float>), dim3(T), dim3(nt), 0, s, x, partial, n_split, split_stride,
-                    static_cast<const float*>(gain), eps, d, static_cast<float*>(out));
+                    static_cast<const float*>(gain), eps, d, static_cast<float*>(out), dev_stamp(st));
   else
     return -1;
   return 1;
@@ -88,7 +93,9 @@ int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t spli
 // --------------------------------------------------------------- rotary table --
 // cs[t][i] = (cos, sin)(pos_t * theta^(-2i/h)), angle and functions in fp64, stored fp32;
 // computed once per step and shared by all layers and heads.
-__global__ void rope_table_kernel(const int32_t* __restrict__ tok_pos, int h, double log2_theta, float2* __restrict__ cs) {
+__global__ void rope_table_kernel(const int32_t* __restrict__ tok_pos, int h, double log2_theta, float2* __restrict__ cs,
+                                  LaunchStamp stamp) {
+  StampScope scope(stamp);
   pdl_enter();
   const int t = blockIdx.x, i = threadIdx.x;
   if (i >= h / 2) return;
@@ -98,9 +105,9 @@ __global__ void rope_table_kernel(const int32_t* __restrict__ tok_pos, int h, do
   cs[static_cast<int64_t>(t) * (h / 2) + i] = make_float2(static_cast<float>(c), static_cast<float>(sn));
 }
 
-int launch_rope_table(const int32_t* tok_pos, int T, int h, float theta, float2* cs, cudaStream_t s) {
+int launch_rope_table(const int32_t* tok_pos, int T, int h, float theta, float2* cs, cudaStream_t s, Stamp st) {
   if (T <= 0) return 0;
-  SLED_LAUNCH_PDL(rope_table_kernel, dim3(T), dim3(h / 2), 0, s, tok_pos, h, log2(static_cast<double>(theta)), cs);
+  SLED_LAUNCH_PDL(rope_table_kernel, dim3(T), dim3(h / 2), 0, s, tok_pos, h, log2(static_cast<double>(theta)), cs, dev_stamp(st));
   return 1;
 }
 
@@ -111,7 +118,8 @@ template <typename AT, typename KT>
 __global__ void rope_kv_kernel(const float* __restrict__ partial, int n_split, int64_t split_stride,
                                const float2* __restrict__ cs, const int32_t* __restrict__ tok_slot, int Hq, int Hkv,
                                int h, int page_size, AT* __restrict__ q_out, KT* __restrict__ kpool,
-                               KT* __restrict__ vpool) {
+                               KT* __restrict__ vpool, LaunchStamp stamp) {
+  StampScope scope(stamp);
   pdl_enter();
   const int t = blockIdx.x, head = blockIdx.y * blockDim.y + threadIdx.y, i = threadIdx.x;
   if (head >= Hq + 2 * Hkv) return;
@@ -147,18 +155,18 @@ __global__ void rope_kv_kernel(const float* __restrict__ partial, int n_split, i
 
 int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, const float2* cs, const int32_t* tok_slot,
                    int T, int Hq, int Hkv, int h, int page_size, void* q_out, int adtype, void* kpool, void* vpool,
-                   int kvdtype, cudaStream_t s) {
+                   int kvdtype, cudaStream_t s, Stamp st) {
   if (T <= 0) return 0;
   dim3 grid(T, (Hq + 2 * Hkv + 3) / 4);
   if (adtype == BF16 && kvdtype == BF16)
     SLED_LAUNCH_PDL((rope_kv_kernel<__nv_bfloat16, __nv_bfloat16>), grid, dim3(h / 2, 4), 0, s, partial, n_split, split_stride, cs, tok_slot,
-                    Hq, Hkv, h, page_size, static_cast<__nv_bfloat16*>(q_out), static_cast<__nv_bfloat16*>(kpool), static_cast<__nv_bfloat16*>(vpool));
+                    Hq, Hkv, h, page_size, static_cast<__nv_bfloat16*>(q_out), static_cast<__nv_bfloat16*>(kpool), static_cast<__nv_bfloat16*>(vpool), dev_stamp(st));
   else if (adtype == F32 && kvdtype == F32)
     SLED_LAUNCH_PDL((rope_kv_kernel<float, float>), grid, dim3(h / 2, 4), 0, s, partial, n_split, split_stride, cs, tok_slot,
-                    Hq, Hkv, h, page_size, static_cast<float*>(q_out), static_cast<float*>(kpool), static_cast<float*>(vpool));
+                    Hq, Hkv, h, page_size, static_cast<float*>(q_out), static_cast<float*>(kpool), static_cast<float*>(vpool), dev_stamp(st));
   else if (adtype == F32 && kvdtype == BF16)
     SLED_LAUNCH_PDL((rope_kv_kernel<float, __nv_bfloat16>), grid, dim3(h / 2, 4), 0, s, partial, n_split, split_stride, cs, tok_slot,
-                    Hq, Hkv, h, page_size, static_cast<float*>(q_out), static_cast<__nv_bfloat16*>(kpool), static_cast<__nv_bfloat16*>(vpool));
+                    Hq, Hkv, h, page_size, static_cast<float*>(q_out), static_cast<__nv_bfloat16*>(kpool), static_cast<__nv_bfloat16*>(vpool), dev_stamp(st));
   else
     return -1;
   return 1;
@@ -168,7 +176,8 @@ int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, cons
 // partial: [split][T][2F], gate and up interleaved (columns 2f and 2f+1):  out = silu(gate) * up
 template <typename AT>
 __global__ void swiglu_kernel(const float* __restrict__ partial, int n_split, int64_t split_stride, int F,
-                              AT* __restrict__ out) {
+                              AT* __restrict__ out, LaunchStamp stamp) {
+  StampScope scope(stamp);
   pdl_enter();
   const int t = blockIdx.y;
   const int f = blockIdx.x * blockDim.x + threadIdx.x;
@@ -184,13 +193,13 @@ __global__ void swiglu_kernel(const float* __restrict__ partial, int n_split, in
 }
 
 int launch_swiglu(const float* partial, int n_split, int64_t split_stride, int T, int F, void* out, int adtype,
-                  cudaStream_t s) {
+                  cudaStream_t s, Stamp st) {
   if (T <= 0) return 0;
   dim3 grid((F + 255) / 256, T);
   if (adtype == BF16)
-    SLED_LAUNCH_PDL(swiglu_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, partial, n_split, split_stride, F, static_cast<__nv_bfloat16*>(out));
+    SLED_LAUNCH_PDL(swiglu_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, partial, n_split, split_stride, F, static_cast<__nv_bfloat16*>(out), dev_stamp(st));
   else
-    SLED_LAUNCH_PDL(swiglu_kernel<float>, grid, dim3(256), 0, s, partial, n_split, split_stride, F, static_cast<float*>(out));
+    SLED_LAUNCH_PDL(swiglu_kernel<float>, grid, dim3(256), 0, s, partial, n_split, split_stride, F, static_cast<float*>(out), dev_stamp(st));
   return 1;
 }
 
@@ -241,7 +250,8 @@ int launch_kv_gather(const void* pool, const int32_t* slots, int n, int Hkv, int
 template <typename AT, typename WT>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const AT* __restrict__ A, const WT* __restrict__ W, int T, int N,
                                                         int K, int k_per_split, float* __restrict__ out,
-                                                        int64_t split_stride) {
+                                                        int64_t split_stride, LaunchStamp stamp) {
+  StampScope scope(stamp);
   pdl_enter();
   constexpr int BM = 32, BN = 64, BK = 32;
   __shared__ float As[BK][BM + 1];
@@ -285,18 +295,18 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const AT* __restrict__ A
 }
 
 int launch_gemm_simt(const void* A, int adtype, const void* W, int wdtype, int T, int N, int K, int n_split,
-                     float* out, int64_t split_stride, cudaStream_t s) {
+                     float* out, int64_t split_stride, cudaStream_t s, Stamp st) {
   if (T <= 0) return 0;
   if (n_split < 1) n_split = 1;
   int k_per_split = ((K + n_split - 1) / n_split + 31) / 32 * 32;
   dim3 grid((N + 63) / 64, (T + 31) / 32, n_split);
   if (adtype == F32 && wdtype == F32)
     SLED_LAUNCH_PDL((gemm_simt_kernel<float, float>), grid, dim3(256), 0, s, static_cast<const float*>(A),
-                    static_cast<const float*>(W), T, N, K, k_per_split, out, split_stride);
+                    static_cast<const float*>(W), T, N, K, k_per_split, out, split_stride, dev_stamp(st));
   else if (adtype == BF16 && wdtype == BF16)
     SLED_LAUNCH_PDL((gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16>), grid, dim3(256), 0, s,
                     static_cast<const __nv_bfloat16*>(A), static_cast<const __nv_bfloat16*>(W), T, N, K, k_per_split, out,
-                    split_stride);
+                    split_stride, dev_stamp(st));
   else
     return -1;
   return 1;

@@ -171,3 +171,16 @@ def make_accept_rows(n_requests: int, k: int, vocab: int, tau_draft: float, seed
         q[i] = qi
         d[i] = torch.multinomial(qi, 1, generator=g).reshape(k).to(torch.int32)
     return z, q, d
+
+
+def correlated_draft(z_row: torch.Tensor, seed: int, ctx_id: int, j: int, rho: float = 0.8):
+    """One draft position of a device whose draft model resembles the target: given the target's logits z at that
+    position (from whichever implementation is being driven), draft logits = rho z + sqrt(1 - rho^2) std(z) noise,
+    q = softmax(draft logits), d ~ q.  Returns (d int, q fp32 [V]) on z_row's device."""
+    dev = z_row.device
+    g = _gen(seed, 600, ctx_id, j, device=dev.type)
+    z = z_row.to(torch.float32)
+    noise = torch.randn(z.shape[0], generator=g, device=dev, dtype=torch.float32)
+    q = torch.softmax(rho * z + (1.0 - rho * rho) ** 0.5 * z.std() * noise, dim=-1)
+    d = int(torch.multinomial(q, 1, generator=g).item())
+    return d, q
