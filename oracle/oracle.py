@@ -8,7 +8,10 @@ server answers with the rejected position and the corrective token):
 
     prefill   -> KV of all prompt tokens but the last, which becomes *pending*
     verify    -> feed [pending, d_1..d_k], Eq. 1 acceptance, then commit the KV of
-                 pending and of the accepted drafts, drop the rest, pending := next
+                 pending and of the accepted drafts, drop the rest, pending := next;
+                 with base_len = m the context is first cut back to its first m tokens
+                 (Section 3.3: a device whose timer ran out sends its drafts again,
+                 extended, from the point it last heard about)
     release   -> forget the context
 
 The arithmetic is all in the C++ file; this file only moves arrays.
@@ -176,7 +179,8 @@ class Context:
     pending: int              # last committed token, not yet in the cache
     K: np.ndarray             # [L, cap, Hkv, h] fp32 values on the cache format's grid
     V: np.ndarray
-    tokens: list = field(default_factory=list)  # committed history when known (prefilled contexts)
+    tokens: list = field(default_factory=list)  # committed tokens from sequence index hist_start on; the last one is pending
+    hist_start: int = 0       # 0 for prefilled contexts; the pending token's index when only the cache was given
 
 
 class OracleModel:
@@ -241,7 +245,7 @@ class OracleModel:
         n = K.shape[1]
         Kc, Vc = self._new_cache(n + 16)
         Kc[:, :n], Vc[:, :n] = K, V
-        self.ctx[ctx_id] = Context(n, int(pending), Kc, Vc, [])
+        self.ctx[ctx_id] = Context(n, int(pending), Kc, Vc, [int(pending)], n)
 
     def release(self, ctx_id: int) -> None:
         del self.ctx[ctx_id]
@@ -253,8 +257,22 @@ class OracleModel:
         feed = [c.pending] + [int(d) for d in drafts]
         return np.stack([self.forward_token(c, t, c.n_kv + j) for j, t in enumerate(feed)])
 
-    def verify(self, ctx_id: int, drafts, q, seed: int, tau: float = 1.0, greedy: bool = False, commit: bool = True):
-        """Returns (status, n_accepted, next_token, logits [k+1, V], Margin)."""
+    def rebase(self, ctx_id: int, base_len: int) -> None:
+        """Cuts the context back to its first base_len committed tokens: the last of them becomes pending again,
+        the cache keeps the base_len - 1 entries before it.  Only as far back as the token history is known."""
+        c = self.ctx[ctx_id]
+        if not (c.hist_start + 1 <= base_len <= c.n_kv + 1):
+            raise ValueError("base_len outside the known history")
+        c.tokens = c.tokens[:base_len - c.hist_start]
+        c.n_kv = base_len - 1
+        c.pending = c.tokens[-1]
+
+    def verify(self, ctx_id: int, drafts, q, seed: int, tau: float = 1.0, greedy: bool = False, commit: bool = True,
+               base_len: int = 0):
+        """Returns (status, n_accepted, next_token, logits [k+1, V], Margin).  base_len > 0: the drafts continue the
+        first base_len tokens of the context (what the device had seen when it drafted), not its current end."""
+        if base_len:
+            self.rebase(ctx_id, base_len)
         c = self.ctx[ctx_id]
         logits = self.score(ctx_id, drafts)
         st, n_acc, nxt, mg = accept(logits, q, drafts, tau, greedy, seed, ctx_id, c.n_kv)

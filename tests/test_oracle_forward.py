@@ -293,3 +293,44 @@ def test_sampling_positions_do_not_collide_across_steps(tiny):
         for j in range(n_acc + 1):
             assert pos0 + j + 1 not in seen
             seen.add(pos0 + j + 1)
+
+
+def test_resent_drafts_continue_the_devices_view(tiny):
+    # Section 3.3: after a timeout the device sends its drafts again, extended.  If the server had in fact
+    # processed the first request, it must go back to the length the device still believes in (base_len);
+    # the outcome must be that of a context that never saw the first request.
+    shape = I.TINY
+    prompt = list(I.make_prompt(shape.vocab, 9, 0, 4))
+    a = O.OracleModel(shape, tiny)
+    a.prefill(4, prompt)
+    d1, q1 = I.make_drafts(shape.vocab, 3, 0, 4)
+    a.verify(4, d1.numpy(), q1.numpy(), seed=1)                   # processed; its answer is lost on the way back
+    assert a.ctx[4].n_kv + 1 > len(prompt)
+    d2, q2 = I.make_drafts(shape.vocab, 5, 0, 4, step=1)          # the resent, longer draft from the old position
+    ra = a.verify(4, d2.numpy(), q2.numpy(), seed=2, base_len=len(prompt))
+    b = O.OracleModel(shape, tiny)
+    b.prefill(4, prompt)
+    rb = b.verify(4, d2.numpy(), q2.numpy(), seed=2)
+    assert ra[:3] == rb[:3] and np.array_equal(ra[3], rb[3])
+    assert a.ctx[4].tokens == b.ctx[4].tokens and a.ctx[4].n_kv == b.ctx[4].n_kv and a.ctx[4].pending == b.ctx[4].pending
+    # every admissible base_len gives the state of a fresh context with that history; base_len = current length is a no-op
+    full = list(a.ctx[4].tokens)
+    for m in range(1, len(full) + 1):
+        c = O.OracleModel(shape, tiny)
+        c.prefill(4, full)
+        c.rebase(4, m)
+        assert (c.ctx[4].tokens, c.ctx[4].n_kv, c.ctx[4].pending) == (full[:m], m - 1, full[m - 1])
+    for bad in (0, len(full) + 1):
+        c = O.OracleModel(shape, tiny)
+        c.prefill(4, full)
+        with pytest.raises(ValueError):
+            c.rebase(4, bad)
+    # a context whose cache was given without its tokens can only go back to where its known history starts
+    K, V = I.make_kv(shape, 6, 0, 1)
+    c = O.OracleModel(shape, tiny)
+    c.load_kv(5, K.numpy(), V.numpy(), pending=3)
+    c.verify(5, d1.numpy(), q1.numpy(), seed=1)
+    c.rebase(5, 7)
+    assert (c.ctx[5].n_kv, c.ctx[5].pending) == (6, 3)
+    with pytest.raises(ValueError):
+        c.rebase(5, 6)
