@@ -446,6 +446,28 @@ class Point:
                                    "by which it extends the step beyond all earlier launches"})
         return roof
 
+    def e2e_with_bf16_rows(self, d_host, q_dev, w_dev, local_rank, stream):
+        """End-to-end steps on an engine that takes its draft rows in bf16 from pinned host memory.  Replaces this
+        point's engine (one copy of the weights at a time)."""
+        B, args = self.B, self.args
+        n_pages = sum((c + k + 1 + 15) // 16 for c, k in zip(self.ctx, self.ks)) + 64
+        self.eng.shutdown()
+        torch.cuda.empty_cache()
+        self.eng = B.Engine(self.shape, w_dev, n_pages=n_pages, max_batch=self.Bn, max_k=max(self.ks),
+                            max_step_tokens=max(self.T, 16), temperature=1.0, greedy=False, device_index=local_rank,
+                            stream=stream.cuda_stream, draft_probs_dtype="bf16")
+        self.eng.shuffle_pages(self.seed)
+        for i in range(self.Bn):
+            K, V = I.make_kv(self.shape, self.ctx[i], self.seed, i, device=self.dev)
+            self.eng.load_kv(i, K, V, pending=1)
+            del K, V
+        q16 = [q.to(torch.bfloat16).cpu().pin_memory() for q in q_dev]
+        reqs = self.marshal(d_host, q16)
+        n_steps = max(5, args.steps // 2)
+        c, ms, _ = self.timed(reqs, n_steps, 3)
+        return {"value": c / (ms / 1e3), "ms_per_step": ms / n_steps,
+                "h2d_bytes_per_step": sum(k * self.shape.vocab * 2 for k in self.ks) + 64 * self.T}
+
     def close(self):
         self.eng.shutdown()
         torch.cuda.empty_cache()
@@ -536,6 +558,10 @@ def run_sled(args):
         s_i = pt.summary(c_i, ms_i, max(5, args.steps // 2), Bn, peaks)
         line["independent_drafts"] = {k: s_i[k] for k in ("ms_per_step", "tokens_per_s", "acceptance_rate", "frac_of_hbm_peak")}
         del d2, q2, r2
+    if e2e and not args.greedy and not args.no_sweep:
+        # the same end-to-end step with the draft rows sent as bf16 (half the bytes; decisions then use the rounded
+        # rows); it replaces the point's engine, so it comes last
+        line["e2e"]["bf16_rows"] = pt.e2e_with_bf16_rows(d_host, q_dev, w, local_rank, stream)
     del d_host, q_dev, reqs_dev
     pt.close()
 

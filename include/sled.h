@@ -29,6 +29,7 @@ extern "C" {
 
 typedef struct sled_engine sled_engine;
 typedef struct sled_kvm sled_kvm;
+typedef struct sled_planner sled_planner;
 
 enum sled_status {
   SLED_OK = 0,
@@ -41,10 +42,18 @@ enum sled_status {
   SLED_ERR_BATCH_TOO_LARGE = -7, /* n_reqs > max_batch or sum(k_i + 1) > max_step_tokens */
   SLED_ERR_NONFINITE = -8,    /* per-request status: a logit that had to be read was NaN or Inf */
   SLED_ERR_DEVICE = -9,       /* CUDA error, or a bounded device-side wait ran out */
-  SLED_ERR_NO_DEVICE = -10    /* no usable CUDA device: there is no CPU fallback */
+  SLED_ERR_NO_DEVICE = -10,   /* no usable CUDA device: there is no CPU fallback */
+  SLED_ERR_BASE_LEN = -11     /* base_len beyond the context's end, or before the start of its known token history */
 };
 
+/* returned by sled_poll while a request is still queued (not an error) */
+#define SLED_PENDING 1
+
 enum sled_dtype { SLED_F32 = 0, SLED_BF16 = 1 };
+
+/* How the server forms batches (Section 3.4).  STATIC is the paper's scheme: requests wait until a fixed number
+ * of them is there.  CONTINUOUS runs whatever has arrived, up to the capacity of a step. */
+enum sled_batching { SLED_BATCH_STATIC = 0, SLED_BATCH_CONTINUOUS = 1 };
 
 /* Shape of the Llama-style target model and the engine's capacities.
  * (The paper fixes only "Llama family", Section 4; shapes come from the workload.) */
@@ -67,6 +76,10 @@ typedef struct sled_config {
                              allocated, host rows are then refused); 0: host or device, found out per request */
   int32_t device_index;   /* CUDA device ordinal */
   void* stream;           /* cudaStream_t to launch on; NULL: the engine creates one */
+  int32_t draft_probs_dtype; /* sled_dtype of every sled_request.draft_probs row.  SLED_F32: exact.  SLED_BF16: rows
+                             rounded to 16 bits by the device, half the bytes per request (Section 3.2 wants requests
+                             small).  Eq. 1 is then applied with the rounded q: the output follows the target's
+                             distribution up to the rounding of q (relative 2^-9 per entry), no longer exactly. */
 } sled_config;
 
 /* Target weights, row-major [out][in], all of type weight_dtype.  HOST or DEVICE
@@ -94,9 +107,18 @@ typedef struct sled_weights {
 typedef struct sled_request {
   uint64_t ctx_id;             /* context opened by sled_prefill */
   const int32_t* draft_tokens; /* [k], host */
-  const float* draft_probs;    /* [k][vocab] fp32, rows sum to 1; host (copied in during the forward pass) or
-                                  device (read in place); may be NULL when k == 0 or in greedy mode */
+  const void* draft_probs;     /* [k][vocab] of cfg.draft_probs_dtype (fp32 unless set otherwise), rows sum to 1; host
+                                  (copied in during the forward pass) or device (read in place); may be NULL when
+                                  k == 0 or in greedy mode */
   int32_t k;                   /* 0 <= k <= max_k; k = 0 is an ordinary decoding step */
+  int64_t base_len;            /* 0: the drafts continue the context's current end.  m > 0: they continue its first m
+                                  committed tokens - the length the device knew when it drafted.  Section 3.3: a device
+                                  whose timer ran out sends its drafts again, extended; if the server had processed the
+                                  first copy after all, it goes back to m before verifying, so the same request may be
+                                  sent any number of times.  m may reach back as far as the context's tokens are known
+                                  (everything for a context opened by sled_prefill) and not beyond its current end:
+                                  SLED_ERR_BASE_LEN otherwise.  The cut is made once the whole call has passed
+                                  validation and reservation; a device failure later leaves the context at m. */
 } sled_request;
 
 /* The feedback of Section 3.2: how many drafts were accepted (the first rejected
@@ -155,6 +177,36 @@ int sled_get_stats(sled_engine* e, sled_stats* out);
 void* sled_get_stream(sled_engine* e);
 void sled_shutdown(sled_engine* e);
 const char* sled_strerror(int status);
+
+/* ---- the server loop around the step (Section 3.4, Fig. 2: queue -> batch planner -> target model) -------- */
+
+/* Batching policy of sled_step; batch_size is the fixed size a STATIC batch waits for (<= max_batch; ignored by
+ * CONTINUOUS, the default).  Only while nothing is queued. */
+int sled_server_config(sled_engine* e, int32_t policy, int32_t batch_size);
+/* Queues one device's request and returns a ticket for it.  The draft tokens are copied; req->draft_probs is
+ * borrowed until the ticket's result has been polled.  Checked here: k, token ids, that the context is open. */
+int sled_submit(sled_engine* e, const sled_request* req, uint64_t* ticket);
+/* Lets the batch planner take the next batch out of the queue (arrival order; one request per context and step;
+ * at most max_batch requests and max_step_tokens tokens - the paper pads a batch to a common length, here it is
+ * ragged) and verifies it with sled_verify_batch.  STATIC: does nothing while fewer than batch_size requests wait,
+ * unless flush != 0.  *n_verified (may be NULL): requests verified by this call.  A request whose context has been
+ * released or cut back since it was queued gets its own error status and does not stop the others; if the step
+ * itself fails, every request of the batch is answered with that code, which is also returned. */
+int sled_step(sled_engine* e, uint64_t seed, int32_t flush, int32_t* n_verified);
+/* SLED_OK and the result if the ticket's request has been verified (the ticket is then forgotten), SLED_PENDING
+ * while it is queued, SLED_ERR_ARG for an unknown ticket. */
+int sled_poll(sled_engine* e, uint64_t ticket, sled_result* out);
+/* Requests waiting in the queue. */
+int32_t sled_queued(sled_engine* e);
+
+/* The queue and batch planner alone (host only, no device needed): what sled_submit / sled_step use. */
+sled_planner* sled_planner_create(int32_t policy, int32_t batch_size, int32_t max_batch, int32_t max_step_tokens);
+void sled_planner_destroy(sled_planner* p);
+int sled_planner_push(sled_planner* p, uint64_t ticket, uint64_t ctx_id, int32_t k);
+/* Next batch, whole or not at all: its tickets into tickets_out (cap entries); returns their number, 0 if no
+ * batch is due, SLED_ERR_BATCH_TOO_LARGE (queue unchanged) if cap is too small. */
+int32_t sled_planner_next_batch(sled_planner* p, int32_t flush, uint64_t* tickets_out, int32_t cap);
+int32_t sled_planner_queued(sled_planner* p);
 
 /* ---- stand-alone pieces of the step (device-resident operands) ---------------------- */
 
@@ -249,6 +301,16 @@ int sled_kvm_release(sled_kvm* m, uint64_t ctx_id);
 int sled_kvm_query(sled_kvm* m, uint64_t ctx_id, int64_t* n_kv, int32_t* pending, int32_t* n_pages,
                    int32_t* pages_out, int32_t cap);
 int32_t sled_kvm_free_pages(sled_kvm* m);
+/* As sled_kvm_reserve_batch, with request i continuing the first base_len[i] committed tokens of its context
+ * (0: its current end; see sled_request.base_len): the context is cut back first.  All or nothing. */
+int sled_kvm_reserve_batch_at(sled_kvm* m, const uint64_t* ctx_ids, const int32_t* extra, const int64_t* base_len,
+                              int32_t n);
+/* As sled_kvm_commit, recording the kept tokens: kept[0 .. n_keep-2] are the tokens behind the old pending one
+ * whose cache entries stay (the accepted drafts), then `pending`. */
+int sled_kvm_commit_tokens(sled_kvm* m, uint64_t ctx_id, int32_t n_keep, int32_t pending, const int32_t* kept);
+/* The known committed tokens of a context: they start at sequence index *hist_start, the last one is pending. */
+int sled_kvm_history(sled_kvm* m, uint64_t ctx_id, int64_t* hist_start, int32_t* n_tokens, int32_t* tokens_out,
+                     int32_t cap);
 /* Ragged packing of one step: for request i with k[i] drafts, writes token rows
  * cu_q[i] .. cu_q[i+1]-1 (row 0 = pending token, then the drafts): ids, owning request,
  * absolute position and physical cache slot (page * page_size + offset).  Pages must have

@@ -18,7 +18,10 @@ LIB_PATH = os.path.join(_HERE, "libsled.so")
 SLED_OK = 0
 SLED_ERR_ARG, SLED_ERR_UNKNOWN_CTX, SLED_ERR_DUP_CTX, SLED_ERR_K_RANGE, SLED_ERR_TOKEN_RANGE = -1, -2, -3, -4, -5
 SLED_ERR_NO_PAGES, SLED_ERR_BATCH_TOO_LARGE, SLED_ERR_NONFINITE, SLED_ERR_DEVICE, SLED_ERR_NO_DEVICE = -6, -7, -8, -9, -10
+SLED_ERR_BASE_LEN = -11
 SLED_F32, SLED_BF16 = 0, 1
+SLED_PENDING = 1
+SLED_BATCH_STATIC, SLED_BATCH_CONTINUOUS = 0, 1
 
 EXPORTS = (
     "sled_init", "sled_verify_batch", "sled_release", "sled_prefill", "sled_set_sampling", "sled_get_stats",
@@ -26,7 +29,10 @@ EXPORTS = (
     "sled_debug_load_kv", "sled_debug_read_kv", "sled_debug_copy_logits", "sled_debug_truncate", "sled_debug_truncate_batch",
     "sled_debug_set_commit", "sled_debug_set_timing", "sled_debug_query_ctx", "sled_debug_shuffle_pages",
     "sled_kvm_create", "sled_kvm_destroy", "sled_kvm_open", "sled_kvm_reserve_batch", "sled_kvm_commit",
-    "sled_kvm_release", "sled_kvm_query", "sled_kvm_free_pages", "sled_kvm_pack",
+    "sled_kvm_release", "sled_kvm_query", "sled_kvm_free_pages", "sled_kvm_pack", "sled_kvm_reserve_batch_at",
+    "sled_kvm_commit_tokens", "sled_kvm_history",
+    "sled_server_config", "sled_submit", "sled_step", "sled_poll", "sled_queued",
+    "sled_planner_create", "sled_planner_destroy", "sled_planner_push", "sled_planner_next_batch", "sled_planner_queued",
 )
 
 
@@ -36,7 +42,8 @@ class SledConfig(C.Structure):
         ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("weight_dtype", C.c_int32), ("kv_dtype", C.c_int32),
         ("page_size", C.c_int32), ("n_pages", C.c_int32), ("max_batch", C.c_int32), ("max_k", C.c_int32),
         ("max_step_tokens", C.c_int32), ("temperature", C.c_float), ("greedy", C.c_int32),
-        ("probs_on_device", C.c_int32), ("device_index", C.c_int32), ("stream", C.c_void_p)]
+        ("probs_on_device", C.c_int32), ("device_index", C.c_int32), ("stream", C.c_void_p),
+        ("draft_probs_dtype", C.c_int32)]
 
 
 class SledWeights(C.Structure):
@@ -46,7 +53,8 @@ class SledWeights(C.Structure):
 
 
 class SledRequest(C.Structure):
-    _fields_ = [("ctx_id", C.c_uint64), ("draft_tokens", C.c_void_p), ("draft_probs", C.c_void_p), ("k", C.c_int32)]
+    _fields_ = [("ctx_id", C.c_uint64), ("draft_tokens", C.c_void_p), ("draft_probs", C.c_void_p), ("k", C.c_int32),
+                ("base_len", C.c_int64)]
 
 
 class SledResult(C.Structure):
@@ -111,6 +119,19 @@ def lib():
             "sled_kvm_query": (C.c_int, [P, U64, C.POINTER(I64), C.POINTER(I32), C.POINTER(I32), P, I32]),
             "sled_kvm_free_pages": (I32, [P]),
             "sled_kvm_pack": (C.c_int, [P, P, P, P, I32, P, P, P, P, P]),
+            "sled_kvm_reserve_batch_at": (C.c_int, [P, P, P, P, I32]),
+            "sled_kvm_commit_tokens": (C.c_int, [P, U64, I32, I32, P]),
+            "sled_kvm_history": (C.c_int, [P, U64, C.POINTER(I64), C.POINTER(I32), P, I32]),
+            "sled_server_config": (C.c_int, [P, I32, I32]),
+            "sled_submit": (C.c_int, [P, C.POINTER(SledRequest), C.POINTER(U64)]),
+            "sled_step": (C.c_int, [P, U64, I32, C.POINTER(I32)]),
+            "sled_poll": (C.c_int, [P, U64, C.POINTER(SledResult)]),
+            "sled_queued": (I32, [P]),
+            "sled_planner_create": (P, [I32, I32, I32, I32]),
+            "sled_planner_destroy": (None, [P]),
+            "sled_planner_push": (C.c_int, [P, U64, U64, I32]),
+            "sled_planner_next_batch": (I32, [P, I32, P, I32]),
+            "sled_planner_queued": (I32, [P]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -154,12 +175,12 @@ class Engine:
 
     def __init__(self, shape, weights: dict, *, n_pages: int, max_batch: int, max_k: int, max_step_tokens: int,
                  temperature: float = 1.0, greedy: bool = False, probs_on_device: bool = False, device_index: int = 0,
-                 page_size: int = 16, stream: int | None = None):
+                 page_size: int = 16, stream: int | None = None, draft_probs_dtype: str = "fp32"):
         self.shape = shape
         cfg = SledConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                          shape.ffn_dim, shape.vocab, shape.rms_eps, shape.rope_theta, _DT[shape.weight_dtype],
                          _DT[shape.kv_dtype], page_size, n_pages, max_batch, max_k, max_step_tokens, temperature,
-                         int(greedy), int(probs_on_device), device_index, stream)
+                         int(greedy), int(probs_on_device), device_index, stream, _DT[draft_probs_dtype])
         w = SledWeights()
         w.tok_emb, w.final_norm, w.lm_head = _addr(weights["tok_emb"]), _addr(weights["final_norm"]), _addr(weights["lm_head"])
         keep = []
@@ -176,18 +197,22 @@ class Engine:
 
     # -- the three calls
     def verify_batch(self, requests, seed: int):
-        """requests: list of (ctx_id, draft_tokens int32 host array [k], draft_probs [k, V] fp32 or None).
+        """requests: list of (ctx_id, draft_tokens int32 host array [k], draft_probs [k, V] fp32 or None[, base_len]).
         Returns list of (n_accepted, next_token, status)."""
         n = len(requests)
         _settle(*[r[2] for r in requests])
         reqs = (SledRequest * max(n, 1))()
         keep = []
-        for i, (ctx, toks, probs) in enumerate(requests):
+        for i, r in enumerate(requests):
+            ctx, toks, probs = r[:3]
+            reqs[i].base_len = r[3] if len(r) > 3 else 0
             toks = np.ascontiguousarray(np.asarray(toks, dtype=np.int32).reshape(-1))
             keep.append(toks)
             if probs is not None and not isinstance(probs, torch.Tensor):
                 probs = np.ascontiguousarray(probs, dtype=np.float32)
                 keep.append(probs)
+            if isinstance(probs, torch.Tensor):
+                assert probs.dtype == (torch.bfloat16 if self.cfg.draft_probs_dtype == SLED_BF16 else torch.float32)
             reqs[i].ctx_id = ctx
             reqs[i].draft_tokens = toks.ctypes.data if toks.size else None
             reqs[i].draft_probs = _addr(probs) if probs is not None and toks.size else None
@@ -202,6 +227,37 @@ class Engine:
 
     def release(self, ctx_id: int) -> None:
         _check(lib().sled_release(self.h, ctx_id), "sled_release")
+
+    # -- the server loop
+    def server_config(self, policy: int, batch_size: int = 0) -> None:
+        _check(lib().sled_server_config(self.h, policy, batch_size), "sled_server_config")
+
+    def submit(self, ctx_id: int, draft_tokens, draft_probs=None, base_len: int = 0) -> int:
+        """Queues one request; returns its ticket.  draft_probs must stay alive until the ticket has been polled."""
+        toks = np.ascontiguousarray(np.asarray(draft_tokens, dtype=np.int32).reshape(-1))
+        _settle(draft_probs)
+        r = SledRequest(ctx_id, toks.ctypes.data if toks.size else None,
+                        _addr(draft_probs) if draft_probs is not None and toks.size else None, toks.size, base_len)
+        t = C.c_uint64()
+        _check(lib().sled_submit(self.h, C.byref(r), C.byref(t)), "sled_submit")
+        return t.value
+
+    def step(self, seed: int, flush: bool = False) -> int:
+        n = C.c_int32()
+        _check(lib().sled_step(self.h, seed, int(flush), C.byref(n)), "sled_step")
+        return n.value
+
+    def poll(self, ticket: int):
+        """(n_accepted, next_token, status) once verified, None while queued."""
+        r = SledResult()
+        rc = lib().sled_poll(self.h, ticket, C.byref(r))
+        if rc == SLED_PENDING:
+            return None
+        _check(rc, "sled_poll")
+        return (r.n_accepted, r.next_token, r.status)
+
+    def queued(self) -> int:
+        return lib().sled_queued(self.h)
 
     def prefill(self, ctx_id: int, tokens) -> None:
         t = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
@@ -329,13 +385,28 @@ class KvManager:
     def open(self, ctx: int, n_kv: int, pending: int) -> int:
         return lib().sled_kvm_open(self.h, ctx, n_kv, pending)
 
-    def reserve_batch(self, ctxs, extra) -> int:
+    def reserve_batch(self, ctxs, extra, base_len=None) -> int:
         c = np.ascontiguousarray(np.asarray(ctxs, dtype=np.uint64))
         x = np.ascontiguousarray(np.asarray(extra, dtype=np.int32))
-        return lib().sled_kvm_reserve_batch(self.h, c.ctypes.data, x.ctypes.data, c.size)
+        if base_len is None:
+            return lib().sled_kvm_reserve_batch(self.h, c.ctypes.data, x.ctypes.data, c.size)
+        b = np.ascontiguousarray(np.asarray(base_len, dtype=np.int64))
+        return lib().sled_kvm_reserve_batch_at(self.h, c.ctypes.data, x.ctypes.data, b.ctypes.data, c.size)
 
-    def commit(self, ctx: int, n_keep: int, pending: int) -> int:
-        return lib().sled_kvm_commit(self.h, ctx, n_keep, pending)
+    def commit(self, ctx: int, n_keep: int, pending: int, kept=None) -> int:
+        if kept is None:
+            return lib().sled_kvm_commit(self.h, ctx, n_keep, pending)
+        t = np.ascontiguousarray(np.asarray(kept, dtype=np.int32))
+        return lib().sled_kvm_commit_tokens(self.h, ctx, n_keep, pending, t.ctypes.data if t.size else None)
+
+    def history(self, ctx: int):
+        start, n = C.c_int64(), C.c_int32()
+        rc = lib().sled_kvm_history(self.h, ctx, C.byref(start), C.byref(n), None, 0)
+        if rc:
+            return rc, None
+        toks = np.zeros(max(n.value, 1), dtype=np.int32)
+        lib().sled_kvm_history(self.h, ctx, None, None, toks.ctypes.data, n.value)
+        return 0, (start.value, [int(x) for x in toks[:n.value]])
 
     def release(self, ctx: int) -> int:
         return lib().sled_kvm_release(self.h, ctx)
@@ -369,6 +440,36 @@ class KvManager:
         try:
             if self.h:
                 lib().sled_kvm_destroy(self.h)
+                self.h = None
+        except Exception:
+            pass
+
+
+class Planner:
+    """The request queue and batch planner alone (sled_planner_*): needs no device."""
+
+    def __init__(self, policy: int, batch_size: int, max_batch: int, max_step_tokens: int):
+        self.h = lib().sled_planner_create(policy, batch_size, max_batch, max_step_tokens)
+        if not self.h:
+            raise SledError(SLED_ERR_ARG, "sled_planner_create")
+        self.cap = max_batch
+
+    def push(self, ticket: int, ctx: int, k: int) -> int:
+        return lib().sled_planner_push(self.h, ticket, ctx, k)
+
+    def next_batch(self, flush: bool = False, cap: int | None = None):
+        cap = self.cap if cap is None else cap
+        out = np.zeros(max(cap, 1), dtype=np.uint64)
+        n = lib().sled_planner_next_batch(self.h, int(flush), out.ctypes.data, cap)
+        return n if n < 0 else [int(x) for x in out[:n]]
+
+    def queued(self) -> int:
+        return lib().sled_planner_queued(self.h)
+
+    def __del__(self):
+        try:
+            if self.h:
+                lib().sled_planner_destroy(self.h)
                 self.h = None
         except Exception:
             pass

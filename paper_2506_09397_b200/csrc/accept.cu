@@ -116,7 +116,11 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
   const int k = a.cu_q[req + 1] - row0 - 1;
   const int V = a.V;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const float* qbase = a.q_rows ? a.q_rows[req] : nullptr;
+  const void* qbase = a.q_rows ? a.q_rows[req] : nullptr;   // the request's [k][V] draft rows, fp32 or bf16
+  const bool q16 = a.q_bf16 != 0;
+  auto q_at = [&](int64_t idx) -> float {                     // a bf16 entry widens exactly
+    return q16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(qbase)[idx]) : static_cast<const float*>(qbase)[idx];
+  };
   int32_t* res = a.results + 3 * req;
   const int n_tiles = (V + kTile - 1) / kTile;
   const int tiles_per_rank = (n_tiles + C - 1) / C;
@@ -132,7 +136,7 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     int bad = 0;
     const bool vec = ((V & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
     // the draft rows are the caller's memory: any 4-byte aligned address is legal, 16-byte loads need more
-    const bool q_vec = vec && ((reinterpret_cast<uintptr_t>(qbase) & 15) == 0);
+    const bool q_vec = vec && ((reinterpret_cast<uintptr_t>(qbase) & (q16 ? 7 : 15)) == 0);   // four entries per load
     if (vec) {   // four consecutive entries per thread and step (16-byte loads), four steps in flight
       auto look = [&](int v, const float4& x4) {
         const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
@@ -236,7 +240,7 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
       xphase ^= 1;
     }
     // ---- the accept test of draft j+1, or fall through on the bonus row (same numbers in every block)
-    const float* qrow = nullptr;
+    int64_t q_off = -1;     // first entry of the deciding row's draft distribution, -1: none (bonus row)
     uint32_t u_smp = 0;
     if (threadIdx.x == 0) {
       uint32_t w[4];
@@ -246,7 +250,7 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
       if (j < k) {
         const int d = a.ids[row0 + 1 + j];
         const unsigned long long Ed = fixed_exp(__fsub_rn(__fmul_rn(z[d], a.inv_tau), m));
-        const float qd = qbase[static_cast<int64_t>(j) * V + d];
+        const float qd = q_at(static_cast<int64_t>(j) * V + d);
         const double lhs = __dmul_rn(__dmul_rn(static_cast<double>(w[0] >> 8), static_cast<double>(qd)),
                                      __ull2double_rn(Z));
         const double rhs = __dmul_rn(__ull2double_rn(Ed), 16777216.0);
@@ -258,11 +262,11 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     __syncthreads();
     if (sh.decision) continue;
     u_smp = static_cast<uint32_t>(sh.flag);
-    if (j < k) qrow = qbase + static_cast<int64_t>(j) * V;
+    if (j < k) q_off = static_cast<int64_t>(j) * V;
 
     // ---- deciding row: weights R_v = max(E_v - trunc(q_v * Z), 0) (or E_v), tile sums in vocabulary order
     const double Zd = __ull2double_rn(Z);
-    bool use_q = qrow != nullptr;
+    bool use_q = q_off >= 0;
     unsigned long long W = 0, before_me = 0;
     for (int attempt = 0; attempt < 2; ++attempt) {
       for (int tl = threadIdx.x; tl < n_tiles; tl += kThreads) sh.tile_sum[tl] = 0ull;
@@ -274,18 +278,22 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
         if (vec && v0 + kVec <= V) {
           const float4 z4 = *reinterpret_cast<const float4*>(z + v0);
           zs[0] = z4.x; zs[1] = z4.y; zs[2] = z4.z; zs[3] = z4.w;
-          if (use_q && q_vec) {
-            const float4 q4 = *reinterpret_cast<const float4*>(qrow + v0);
+          if (use_q && q_vec && !q16) {
+            const float4 q4 = *reinterpret_cast<const float4*>(static_cast<const float*>(qbase) + q_off + v0);
             qs[0] = q4.x; qs[1] = q4.y; qs[2] = q4.z; qs[3] = q4.w;
+          } else if (use_q && q_vec) {
+            const uint2 q4 = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(qbase) + q_off + v0);
+            qs[0] = __uint_as_float(q4.x << 16); qs[1] = __uint_as_float(q4.x & 0xffff0000u);
+            qs[2] = __uint_as_float(q4.y << 16); qs[3] = __uint_as_float(q4.y & 0xffff0000u);
           } else if (use_q) {
 #pragma unroll
-            for (int e = 0; e < kVec; ++e) qs[e] = qrow[v0 + e];
+            for (int e = 0; e < kVec; ++e) qs[e] = q_at(q_off + v0 + e);
           }
         } else {
 #pragma unroll
           for (int e = 0; e < kVec; ++e) {
             zs[e] = v0 + e < V ? z[v0 + e] : 0.f;
-            qs[e] = (use_q && v0 + e < V) ? qrow[v0 + e] : 0.f;
+            qs[e] = (use_q && v0 + e < V) ? q_at(q_off + v0 + e) : 0.f;
           }
         }
 #pragma unroll
@@ -346,7 +354,7 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
         if (v < V) {
           E = fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
           if (use_q) {
-            const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(qrow[v]), Zd));
+            const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(q_at(q_off + v)), Zd));
             E = E > Q ? E - Q : 0ull;
           }
         }

@@ -12,6 +12,9 @@
 #include "gemm_tc.h"
 #include "kernels.h"
 #include "kv_manager.h"
+#include "planner.h"
+
+#include <unordered_map>
 
 using namespace sled;
 
@@ -106,6 +109,17 @@ struct sled_engine {
   unsigned long long* h_stamps = nullptr;   // pinned mirror
   std::vector<int> stamp_kind;
   size_t stamp_cap = 0, stamp_used = 0;
+
+  // server loop (sled_submit / sled_step / sled_poll): queued requests with their own copy of the draft tokens,
+  // finished results by ticket
+  struct Waiting {
+    sled_request req;
+    std::vector<int32_t> drafts;
+  };
+  Planner* planner = nullptr;
+  std::unordered_map<uint64_t, Waiting> waiting;
+  std::unordered_map<uint64_t, sled_result> finished;
+  uint64_t next_ticket = 1;
 
   sled_stats st{};
   int64_t launches_step = 0;
@@ -568,6 +582,7 @@ void destroy(sled_engine* e) {
   if (e->copy_stream) cudaStreamDestroy(e->copy_stream);
   if (e->own_stream && e->stream) cudaStreamDestroy(e->stream);
   delete e->kvm;
+  delete e->planner;
   delete e;
 }
 
@@ -642,6 +657,7 @@ int check_cfg(const sled_config& c) {
   if (c.weight_dtype != SLED_F32 && c.weight_dtype != SLED_BF16) return SLED_ERR_ARG;
   if (c.kv_dtype != SLED_F32 && c.kv_dtype != SLED_BF16) return SLED_ERR_ARG;
   if (c.weight_dtype == SLED_BF16 && c.kv_dtype != SLED_BF16) return SLED_ERR_ARG;
+  if (c.draft_probs_dtype != SLED_F32 && c.draft_probs_dtype != SLED_BF16) return SLED_ERR_ARG;
   if (c.page_size <= 0 || c.n_pages <= 0 || c.max_batch <= 0 || c.max_k < 0 || c.max_step_tokens <= 0)
     return SLED_ERR_ARG;
   if (c.max_step_tokens < c.max_k + 1) return SLED_ERR_ARG;
@@ -667,6 +683,7 @@ const char* sled_strerror(int s) {
     case SLED_ERR_NONFINITE: return "non-finite logit";
     case SLED_ERR_DEVICE: return "device error";
     case SLED_ERR_NO_DEVICE: return "no CUDA device (this library has no CPU fallback)";
+    case SLED_ERR_BASE_LEN: return "base_len outside the context's known history";
     default: return "unknown status";
   }
 }
@@ -704,6 +721,7 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if (cudaEventCreateWithFlags(&e->ev_copy, cudaEventDisableTiming) != cudaSuccess) return fail(SLED_ERR_DEVICE);
   if (cudaEventCreate(&e->ev_a) != cudaSuccess || cudaEventCreate(&e->ev_b) != cudaSuccess) return fail(SLED_ERR_DEVICE);
   e->kvm = new KvManager(c.n_pages, c.page_size);
+  e->planner = new Planner(kBatchContinuous, 0, c.max_batch, c.max_step_tokens);
 
   const size_t es = dtype_size(c.weight_dtype);
   const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kd = c.n_kv_heads * c.head_dim, F = c.ffn_dim;
@@ -757,7 +775,7 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->part_acc), static_cast<size_t>(e->part_rows_cap) * qd * 4))) return fail(rc);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->part_ml), static_cast<size_t>(e->part_rows_cap) * c.n_q_heads * 8))) return fail(rc);
   if (!c.probs_on_device && !c.greedy)
-    if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->q_stage), maxT * c.vocab * 4))) return fail(rc);
+    if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->q_stage), maxT * c.vocab * dtype_size(c.draft_probs_dtype)))) return fail(rc);
   // results block: [0] error word (+3 words of padding), then 3 words per request
   if (cudaMallocHost(reinterpret_cast<void**>(&e->h_results), sizeof(int32_t) * (kResultsHead + 3 * c.max_batch)) != cudaSuccess)
     return fail(SLED_ERR_DEVICE);
@@ -799,7 +817,8 @@ int sled_set_sampling(sled_engine* e, float temperature, int32_t greedy) {
   if (!e || !(temperature > 0.f)) return SLED_ERR_ARG;
   if (!greedy && !e->cfg.probs_on_device && !e->q_stage) {
     cudaSetDevice(e->cfg.device_index);
-    int rc = dmalloc(e, reinterpret_cast<void**>(&e->q_stage), static_cast<size_t>(e->cfg.max_step_tokens) * e->cfg.vocab * 4);
+    int rc = dmalloc(e, reinterpret_cast<void**>(&e->q_stage),
+                     static_cast<size_t>(e->cfg.max_step_tokens) * e->cfg.vocab * dtype_size(e->cfg.draft_probs_dtype));
     if (rc) return rc;
   }
   e->cfg.temperature = temperature;
@@ -851,7 +870,7 @@ int sled_prefill(sled_engine* e, uint64_t ctx_id, const int32_t* tokens, int32_t
       e->kvm->release(ctx_id);
       return rc;
     }
-    e->kvm->commit(ctx_id, chunk, tokens[done + chunk]);
+    e->kvm->commit(ctx_id, chunk, tokens[done + chunk], tokens + done + 1);
     done += chunk;
   }
   e->kvm->truncate(ctx_id, n_kv, tokens[n - 1]);
@@ -870,6 +889,7 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
     if (r.k < 0 || r.k > c.max_k) return SLED_ERR_K_RANGE;
     if (r.k > 0 && !r.draft_tokens) return SLED_ERR_ARG;
     if (r.k > 0 && !c.greedy && !r.draft_probs) return SLED_ERR_ARG;
+    if (r.base_len < 0) return SLED_ERR_ARG;
     for (int j = 0; j < r.k; ++j)
       if (r.draft_tokens[j] < 0 || r.draft_tokens[j] >= c.vocab) return SLED_ERR_TOKEN_RANGE;
     T += r.k + 1;
@@ -877,8 +897,11 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   if (T > c.max_step_tokens) return SLED_ERR_BATCH_TOO_LARGE;
   std::vector<uint64_t> ctxs(n_reqs);
   std::vector<int32_t> extra(n_reqs);
-  for (int i = 0; i < n_reqs; ++i) { ctxs[i] = reqs[i].ctx_id; extra[i] = reqs[i].k + 1; }
-  int rc = e->kvm->reserve_batch(ctxs.data(), extra.data(), n_reqs);  // unknown / duplicate / no pages: atomic
+  std::vector<int64_t> base(n_reqs);
+  for (int i = 0; i < n_reqs; ++i) { ctxs[i] = reqs[i].ctx_id; extra[i] = reqs[i].k + 1; base[i] = reqs[i].base_len; }
+  // unknown / duplicate context, base_len out of range, no pages: nothing has changed.  Otherwise contexts whose
+  // request names a base_len are cut back to it here, and stay there whatever happens later in the call.
+  int rc = e->kvm->reserve_batch(ctxs.data(), extra.data(), n_reqs, base.data());
   if (rc) return rc;
   std::vector<int32_t> old_pending(n_reqs);
   for (int i = 0; i < n_reqs; ++i) old_pending[i] = e->kvm->find(ctxs[i])->pending;
@@ -909,13 +932,14 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   Packed pk;
   if ((rc = pack_step(e, plan, false, &pk))) return rollback(rc);
   uint32_t *d_lo = nullptr, *d_hi = nullptr;
-  const float** d_qptr = nullptr;
+  const void** d_qptr = nullptr;
   uint32_t* h_lo = e->meta_alloc<uint32_t>(n_reqs, &d_lo);
   uint32_t* h_hi = e->meta_alloc<uint32_t>(n_reqs, &d_hi);
-  const float** h_qptr = e->meta_alloc<const float*>(n_reqs, &d_qptr);
+  const void** h_qptr = e->meta_alloc<const void*>(n_reqs, &d_qptr);
   if (!h_lo || !h_hi || !h_qptr) return rollback(SLED_ERR_BATCH_TOO_LARGE);
   bool staged = false;
-  struct QCopy { float* dst; const float* src; size_t bytes; };
+  struct QCopy { char* dst; const void* src; size_t bytes; };
+  const size_t qsize = dtype_size(c.draft_probs_dtype);
   std::vector<QCopy> copies;
   {
     size_t row = 0;
@@ -933,8 +957,8 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
         else if (!e->q_stage) return rollback(SLED_ERR_ARG);  // engine was created for device-resident rows only
         else {
           // draft distributions travel on the copy stream while the forward pass runs
-          float* dst = e->q_stage + row * c.vocab;
-          copies.push_back({dst, reqs[i].draft_probs, static_cast<size_t>(reqs[i].k) * c.vocab * 4});
+          char* dst = reinterpret_cast<char*>(e->q_stage) + row * c.vocab * qsize;
+          copies.push_back({dst, reqs[i].draft_probs, static_cast<size_t>(reqs[i].k) * c.vocab * qsize});
           h_qptr[i] = dst;
           row += reqs[i].k;
           staged = true;
@@ -959,6 +983,7 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   aa.cu_q = pk.cu_q;
   aa.ids = pk.ids;
   aa.q_rows = c.greedy ? nullptr : d_qptr;
+  aa.q_bf16 = c.draft_probs_dtype == SLED_BF16;
   aa.ctx_lo = d_lo;
   aa.ctx_hi = d_hi;
   aa.pos0 = pk.kv_base;
@@ -1005,7 +1030,7 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
     results[i].next_token = r[1];
     results[i].status = r[2];
     if (results[i].status == SLED_OK && e->commit) {
-      e->kvm->commit(ctxs[i], results[i].n_accepted + 1, results[i].next_token);
+      e->kvm->commit(ctxs[i], results[i].n_accepted + 1, results[i].next_token, reqs[i].draft_tokens);
       e->st.drafts_accepted += results[i].n_accepted;
       e->st.tokens_committed += results[i].n_accepted + 1;
     } else {
@@ -1014,6 +1039,85 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   }
   return SLED_OK;
 }
+
+// ------------------------------------------------------------------- server loop --
+int sled_server_config(sled_engine* e, int32_t policy, int32_t batch_size) {
+  if (!e) return SLED_ERR_ARG;
+  if (!e->waiting.empty()) return SLED_ERR_ARG;   // the policy changes only while nothing is queued
+  Planner* p = new Planner(policy, batch_size, e->cfg.max_batch, e->cfg.max_step_tokens);
+  if (!p->valid()) {
+    delete p;
+    return SLED_ERR_ARG;
+  }
+  delete e->planner;
+  e->planner = p;
+  return SLED_OK;
+}
+
+int sled_submit(sled_engine* e, const sled_request* req, uint64_t* ticket) {
+  if (!e || !req || !ticket) return SLED_ERR_ARG;
+  const sled_config& c = e->cfg;
+  if (req->k < 0 || req->k > c.max_k) return SLED_ERR_K_RANGE;
+  if (req->k > 0 && (!req->draft_tokens || (!c.greedy && !req->draft_probs))) return SLED_ERR_ARG;
+  if (req->base_len < 0) return SLED_ERR_ARG;
+  for (int j = 0; j < req->k; ++j)
+    if (req->draft_tokens[j] < 0 || req->draft_tokens[j] >= c.vocab) return SLED_ERR_TOKEN_RANGE;
+  if (!e->kvm->find(req->ctx_id)) return SLED_ERR_UNKNOWN_CTX;
+  const uint64_t t = e->next_ticket++;
+  int rc = e->planner->push(t, req->ctx_id, req->k);
+  if (rc) return rc;
+  sled_engine::Waiting& w = e->waiting[t];
+  w.req = *req;
+  w.drafts.assign(req->draft_tokens, req->draft_tokens + req->k);
+  *ticket = t;
+  return SLED_OK;
+}
+
+int sled_step(sled_engine* e, uint64_t seed, int32_t flush, int32_t* n_verified) {
+  if (!e) return SLED_ERR_ARG;
+  if (n_verified) *n_verified = 0;
+  const std::vector<uint64_t> batch = e->planner->next_batch(flush != 0);
+  if (batch.empty()) return SLED_OK;
+  // Requests were checked when they came in, but their context may have been released, or cut back, since: those
+  // are answered with their own error; the rest of the batch runs.
+  std::vector<sled_request> reqs;
+  std::vector<uint64_t> tickets;
+  for (uint64_t t : batch) {
+    sled_engine::Waiting& w = e->waiting[t];
+    w.req.draft_tokens = w.drafts.data();
+    const CtxState* cs = e->kvm->find(w.req.ctx_id);
+    int bad = SLED_OK;
+    if (!cs) bad = SLED_ERR_UNKNOWN_CTX;
+    else if (w.req.base_len != 0 && (w.req.base_len < cs->hist_start + 1 || w.req.base_len > cs->n_kv + 1)) bad = SLED_ERR_BASE_LEN;
+    if (bad) {
+      e->finished[t] = sled_result{0, -1, bad};
+      e->waiting.erase(t);
+      continue;
+    }
+    reqs.push_back(w.req);
+    tickets.push_back(t);
+  }
+  if (reqs.empty()) return SLED_OK;
+  std::vector<sled_result> res(reqs.size());
+  const int rc = sled_verify_batch(e, reqs.data(), static_cast<int32_t>(reqs.size()), seed, res.data());
+  for (size_t i = 0; i < tickets.size(); ++i) {
+    e->finished[tickets[i]] = rc == SLED_OK ? res[i] : sled_result{0, -1, rc};   // a failed step answers every request with its code
+    e->waiting.erase(tickets[i]);
+  }
+  if (rc == SLED_OK && n_verified) *n_verified = static_cast<int32_t>(tickets.size());
+  return rc;
+}
+
+int sled_poll(sled_engine* e, uint64_t ticket, sled_result* out) {
+  if (!e || !out) return SLED_ERR_ARG;
+  auto it = e->finished.find(ticket);
+  if (it == e->finished.end()) return e->waiting.count(ticket) ? SLED_PENDING : SLED_ERR_ARG;
+  *out = it->second;
+  e->finished.erase(it);
+  return SLED_OK;
+}
+
+int32_t sled_queued(sled_engine* e) { return e ? e->planner->queued() : SLED_ERR_ARG; }
 
 // ------------------------------------------------------------ stand-alone pieces --
 int sled_accept_rows(const float* logits, const int32_t* cu_rows, const int32_t* drafts, const float* q_rows,
@@ -1032,7 +1136,7 @@ int sled_accept_rows(const float* logits, const int32_t* cu_rows, const int32_t*
   // small per-call device arrays
   std::vector<int32_t> ids(rows, 0), p0(n_reqs);
   std::vector<uint32_t> lo(n_reqs), hi(n_reqs);
-  std::vector<const float*> qp(n_reqs, nullptr);
+  std::vector<const void*> qp(n_reqs, nullptr);
   int64_t drow = 0;
   for (int i = 0; i < n_reqs; ++i) {
     const int k = cu_rows[i + 1] - cu_rows[i] - 1;
@@ -1070,7 +1174,7 @@ int sled_accept_rows(const float* logits, const int32_t* cu_rows, const int32_t*
   aa.logits = logits;
   aa.cu_q = reinterpret_cast<int32_t*>(dev + o_cu);
   aa.ids = reinterpret_cast<int32_t*>(dev + o_ids);
-  aa.q_rows = greedy ? nullptr : reinterpret_cast<const float* const*>(dev + o_qp);
+  aa.q_rows = greedy ? nullptr : reinterpret_cast<const void* const*>(dev + o_qp);
   aa.ctx_lo = reinterpret_cast<uint32_t*>(dev + o_lo);
   aa.ctx_hi = reinterpret_cast<uint32_t*>(dev + o_hi);
   aa.pos0 = reinterpret_cast<int32_t*>(dev + o_p0);

@@ -75,7 +75,8 @@ struct AcceptArgs {
   const float* logits;        // [rows][V]
   const int32_t* cu_q;        // [B+1] first row of each request
   const int32_t* ids;         // [rows] fed tokens: drafts of request i are ids[cu_q[i]+1 ..]
-  const float* const* q_rows; // [B] device pointer to the request's [k][V] draft distributions (may hold null)
+  const void* const* q_rows;  // [B] device pointer to the request's [k][V] draft distributions (may hold null)
+  int q_bf16;                 // 1: the rows are bf16, 0: fp32
   const uint32_t* ctx_lo;     // [B]
   const uint32_t* ctx_hi;     // [B]
   const int32_t* pos0;        // [B] absolute index of the pending token

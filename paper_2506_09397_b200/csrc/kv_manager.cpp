@@ -33,6 +33,8 @@ int KvManager::open(uint64_t ctx, int64_t n_kv, int32_t pending) {
   CtxState c;
   c.n_kv = n_kv;
   c.pending = pending;
+  c.hist_start = n_kv;
+  c.hist.assign(1, pending);
   for (int64_t i = 0; i < need; ++i) {
     c.pages.push_back(free_.back());
     free_.pop_back();
@@ -41,7 +43,7 @@ int KvManager::open(uint64_t ctx, int64_t n_kv, int32_t pending) {
   return SLED_OK;
 }
 
-int KvManager::reserve_batch(const uint64_t* ctxs, const int32_t* extra, int32_t n) {
+int KvManager::reserve_batch(const uint64_t* ctxs, const int32_t* extra, int32_t n, const int64_t* base_len) {
   // first pass: everything that can fail, without touching any state
   std::unordered_set<uint64_t> seen;
   int64_t need = 0;
@@ -51,9 +53,24 @@ int KvManager::reserve_batch(const uint64_t* ctxs, const int32_t* extra, int32_t
     auto it = ctx_.find(ctxs[i]);
     if (it == ctx_.end()) return SLED_ERR_UNKNOWN_CTX;
     const CtxState& c = it->second;
-    need += pages_for(c.n_kv + extra[i]) - static_cast<int64_t>(c.pages.size());
+    int64_t n_kv = c.n_kv;
+    if (base_len && base_len[i] != 0) {
+      // only as far back as the tokens are known, and never beyond the current end
+      if (base_len[i] < c.hist_start + 1 || base_len[i] > c.n_kv + 1) return SLED_ERR_BASE_LEN;
+      n_kv = base_len[i] - 1;
+    }
+    need += pages_for(n_kv + extra[i]) - static_cast<int64_t>(c.pages.size());   // negative: pages come back
   }
   if (need > static_cast<int64_t>(free_.size())) return SLED_ERR_NO_PAGES;
+  if (base_len)   // contexts that shrink first, so that their pages are there for the ones that grow
+    for (int32_t i = 0; i < n; ++i) {
+      if (base_len[i] == 0) continue;
+      CtxState& c = ctx_.find(ctxs[i])->second;
+      c.n_kv = base_len[i] - 1;
+      c.hist.resize(static_cast<size_t>(base_len[i] - c.hist_start));
+      c.pending = c.hist.back();
+      shrink_to(c, c.n_kv + extra[i]);
+    }
   for (int32_t i = 0; i < n; ++i) {
     CtxState& c = ctx_.find(ctxs[i])->second;
     const int64_t want = pages_for(c.n_kv + extra[i]);
@@ -66,7 +83,7 @@ int KvManager::reserve_batch(const uint64_t* ctxs, const int32_t* extra, int32_t
   return SLED_OK;
 }
 
-int KvManager::commit(uint64_t ctx, int32_t n_keep, int32_t pending) {
+int KvManager::commit(uint64_t ctx, int32_t n_keep, int32_t pending, const int32_t* kept) {
   auto it = ctx_.find(ctx);
   if (it == ctx_.end()) return SLED_ERR_UNKNOWN_CTX;
   CtxState& c = it->second;
@@ -74,6 +91,15 @@ int KvManager::commit(uint64_t ctx, int32_t n_keep, int32_t pending) {
   c.n_kv += n_keep;
   c.n_reserved = 0;
   c.pending = pending;
+  if (n_keep == 0) {
+    c.hist.back() = pending;   // nothing kept: the pending token stays (callers pass the old one back)
+  } else if (kept || n_keep == 1) {
+    for (int32_t j = 0; j + 1 < n_keep; ++j) c.hist.push_back(kept[j]);
+    c.hist.push_back(pending);
+  } else {                     // tokens not given: what is known restarts at the new pending token
+    c.hist_start = c.n_kv;
+    c.hist.assign(1, pending);
+  }
   shrink_to(c, c.n_kv);
   return SLED_OK;
 }
@@ -86,6 +112,12 @@ int KvManager::truncate(uint64_t ctx, int64_t n_kv, int32_t pending) {
   c.n_kv = n_kv;
   c.n_reserved = 0;
   c.pending = pending;
+  if (n_kv >= c.hist_start && c.hist[static_cast<size_t>(n_kv - c.hist_start)] == pending) {
+    c.hist.resize(static_cast<size_t>(n_kv - c.hist_start) + 1);   // a cut inside the known history
+  } else {
+    c.hist_start = n_kv;
+    c.hist.assign(1, pending);
+  }
   shrink_to(c, c.n_kv);
   return SLED_OK;
 }
@@ -137,6 +169,32 @@ int sled_kvm_reserve_batch(sled_kvm* m, const uint64_t* ctx_ids, const int32_t* 
 
 int sled_kvm_commit(sled_kvm* m, uint64_t ctx_id, int32_t n_keep, int32_t pending) {
   return m ? m->m.commit(ctx_id, n_keep, pending) : SLED_ERR_ARG;
+}
+
+int sled_kvm_reserve_batch_at(sled_kvm* m, const uint64_t* ctx_ids, const int32_t* extra, const int64_t* base_len,
+                              int32_t n) {
+  if (!m || n < 0 || (n > 0 && (!ctx_ids || !extra))) return SLED_ERR_ARG;
+  if (base_len)
+    for (int32_t i = 0; i < n; ++i)
+      if (base_len[i] < 0) return SLED_ERR_ARG;
+  return m->m.reserve_batch(ctx_ids, extra, n, base_len);
+}
+
+int sled_kvm_commit_tokens(sled_kvm* m, uint64_t ctx_id, int32_t n_keep, int32_t pending, const int32_t* kept) {
+  if (!m || (n_keep > 1 && !kept)) return SLED_ERR_ARG;
+  return m->m.commit(ctx_id, n_keep, pending, kept);
+}
+
+int sled_kvm_history(sled_kvm* m, uint64_t ctx_id, int64_t* hist_start, int32_t* n_tokens, int32_t* tokens_out,
+                     int32_t cap) {
+  if (!m) return SLED_ERR_ARG;
+  const sled::CtxState* c = m->m.find(ctx_id);
+  if (!c) return SLED_ERR_UNKNOWN_CTX;
+  if (hist_start) *hist_start = c->hist_start;
+  if (n_tokens) *n_tokens = static_cast<int32_t>(c->hist.size());
+  if (tokens_out)
+    for (int32_t i = 0; i < cap && i < static_cast<int32_t>(c->hist.size()); ++i) tokens_out[i] = c->hist[i];
+  return SLED_OK;
 }
 
 int sled_kvm_release(sled_kvm* m, uint64_t ctx_id) { return m ? m->m.release(ctx_id) : SLED_ERR_ARG; }

@@ -14,14 +14,22 @@ struct CtxState {
   int64_t n_reserved = 0;  // slots reserved behind them for the step in flight
   int32_t pending = 0;     // last committed token; its KV is written by the next step
   std::vector<int32_t> pages;
+  // committed tokens from sequence index hist_start on (the last one is `pending`): what a request's base_len can go
+  // back to.  A context opened from cache content alone knows its history from the pending token on.
+  std::vector<int32_t> hist;
+  int64_t hist_start = 0;
 };
 
 class KvManager {
  public:
   KvManager(int32_t n_pages, int32_t page_size);
   int open(uint64_t ctx, int64_t n_kv, int32_t pending);
-  int reserve_batch(const uint64_t* ctxs, const int32_t* extra, int32_t n);
-  int commit(uint64_t ctx, int32_t n_keep, int32_t pending);
+  // base_len (may be null; entries of 0 mean "continue at the end"): request i continues the first base_len[i]
+  // committed tokens of its context, which is cut back to that length before slots are reserved
+  int reserve_batch(const uint64_t* ctxs, const int32_t* extra, int32_t n, const int64_t* base_len = nullptr);
+  // kept: the n_keep - 1 tokens behind the old pending one whose cache entries stay (null: unknown, the history
+  // restarts at the new pending token)
+  int commit(uint64_t ctx, int32_t n_keep, int32_t pending, const int32_t* kept = nullptr);
   int truncate(uint64_t ctx, int64_t n_kv, int32_t pending);
   int release(uint64_t ctx);
   void shuffle_free(uint64_t seed);  // seeded permutation of the free list

@@ -26,7 +26,7 @@ struct alignas(256) StaticBlock {
   uint32_t lo[kMaxReqs];          // context id, low / high word
   uint32_t hi[kMaxReqs];
   int32_t pos0[kMaxReqs];         // index of the pending token
-  const float* qptr[kMaxReqs];    // device address of each request's draft rows
+  const void* qptr[kMaxReqs];     // device address of each request's draft rows
   int32_t results[3 * kMaxReqs];  // n_accepted, next_token, status
 };
 

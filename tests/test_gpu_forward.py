@@ -336,3 +336,88 @@ def test_step_between_128_and_160_tokens():
             assert (n2, x2, 0) == g
         row += k + 1
     eng.shutdown()
+
+
+def test_resent_request_goes_back_to_base_len():
+    # a device's answer is lost; it sends its drafts again, extended, naming the length it still believes in
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=9)
+    eng = _engine(shape, w)
+    orc = O.OracleModel(shape, oracle_weights(w))
+    lens = {31: 23, 32: 40, 33: 17}
+    for c, n in lens.items():
+        p = I.make_prompt(shape.vocab, n, 9, c)
+        eng.prefill(c, p)
+        orc.prefill(c, p)
+    reqs = [(c,) + tuple(I.make_drafts(shape.vocab, 4, 9, c)) for c in lens]
+    explain = []
+    _verify_both(eng, orc, reqs, seed=1, tau=1.0, greedy=False, tol=2e-2, explain=explain)
+    grown = {c: eng.query_ctx(c)[0] for c in lens}
+    assert all(grown[c] >= lens[c] for c in lens)
+    # context 31 resends from its old length with more drafts, 32 continues normally, 33 names its current length (no-op)
+    d31, q31 = I.make_drafts(shape.vocab, 7, 9, 31, step=1)
+    d32, q32 = I.make_drafts(shape.vocab, 3, 9, 32, step=1)
+    d33, q33 = I.make_drafts(shape.vocab, 2, 9, 33, step=1)
+    base = {31: lens[31], 32: 0, 33: grown[33] + 1}
+    batch = [(31, d31, q31), (32, d32, q32), (33, d33, q33)]
+    got = eng.verify_batch([(c, d.numpy(), q.numpy(), base[c]) for c, d, q in batch], 2)
+    glog = eng.logits(sum(len(d) + 1 for _, d, _ in batch))
+    row = 0
+    for (c, d, q), g in zip(batch, got):
+        k = len(d)
+        if base[c]:
+            orc.rebase(c, base[c])
+        pos0 = orc.ctx[c].n_kv
+        if c == 31:
+            assert pos0 == lens[31] - 1
+        st, n_acc, nxt, ol, mg = orc.verify(c, d.numpy(), q.numpy(), 2, commit=False)
+        mine = glog[row:row + k + 1]
+        row += k + 1
+        assert np.max(np.abs(mine - ol)) <= 2e-2
+        st2, n2, x2, _ = O.accept(mine, q.numpy(), d.numpy(), 1.0, False, 2, c, pos0)
+        assert (n2, x2, 0) == g
+        assert eng.query_ctx(c)[:2] == (pos0 + g[0] + 1, g[1])
+    # out-of-range base_len: refused, nothing changes (context 32 in the same batch included)
+    before = [str(eng.query_ctx(c)) for c in lens]
+    for bad in (eng.query_ctx(31)[0] + 2, 10**6):
+        with pytest.raises(B.SledError) as ei:
+            eng.verify_batch([(32, d32.numpy(), q32.numpy(), 0), (31, d31.numpy(), q31.numpy(), bad)], 3)
+        assert ei.value.code == B.SLED_ERR_BASE_LEN
+    assert before == [str(eng.query_ctx(c)) for c in lens]
+    # a context opened from cache content alone cannot go back before the point where its tokens are known
+    K, V = I.make_kv(shape, 20, 9, 40)
+    eng.load_kv(40, (K * 0.3).contiguous(), (V * 0.3).contiguous(), pending=5)
+    with pytest.raises(B.SledError) as ei:
+        eng.verify_batch([(40, d33.numpy(), q33.numpy(), 20)], 3)
+    assert ei.value.code == B.SLED_ERR_BASE_LEN
+    assert eng.verify_batch([(40, d33.numpy(), q33.numpy(), 21)], 3)[0][2] == 0
+    eng.shutdown()
+
+
+@pytest.mark.parametrize("where", ["host", "device"])
+def test_draft_rows_in_bf16(where):
+    # rows sent in 16 bits (half the request bytes): the decision must be the oracle's rule applied to the GPU's
+    # logits and to the rows as sent (a bf16 value widens to fp32 exactly)
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=10)
+    eng = _engine(shape, w, draft_probs_dtype="bf16")
+    ctxs = [51, 52, 53, 54]
+    for c in ctxs:
+        eng.prefill(c, I.make_prompt(shape.vocab, 12 + c % 7, 10, c))
+    eng.set_commit(False)
+    reqs, rows = [], []
+    for c, k in zip(ctxs, [5, 0, 8, 3]):
+        d, q = I.make_drafts(shape.vocab, k, 10, c)
+        q16 = q.to(torch.bfloat16).contiguous()
+        rows.append(q16.float().numpy())
+        reqs.append((c, d.numpy(), q16.cuda() if where == "device" else q16))
+    got = eng.verify_batch(reqs, 4)
+    glog = eng.logits(sum(len(r[1]) + 1 for r in reqs))
+    row = 0
+    for (c, d, _), qf, g in zip(reqs, rows, got):
+        k = len(d)
+        st2, n2, x2, _ = O.accept(glog[row:row + k + 1], qf if k else None, d, 1.0, False, 4, c, eng.query_ctx(c)[0])
+        assert (n2, x2, 0) == g
+        row += k + 1
+    assert any(g[0] < len(r[1]) for r, g in zip(reqs, got))      # a rejection happened: the residual read a 16-bit row
+    eng.shutdown()

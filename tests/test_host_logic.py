@@ -20,7 +20,7 @@ def built():
 
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "sled.h")).read()
-    declared = set(re.findall(r"^(?:int|void|void\*|const char\*|int32_t|sled_kvm\*)\s+(sled_[a-z_0-9]+)\(", header, re.M))
+    declared = set(re.findall(r"^(?:int|void|void\*|const char\*|int32_t|sled_kvm\*|sled_planner\*)\s+(sled_[a-z_0-9]+)\(", header, re.M))
     assert len(declared) > 20
     assert declared == set(B.EXPORTS)
     raw = C.CDLL(B.LIB_PATH)
@@ -125,3 +125,74 @@ def test_page_manager_errors():
     assert m.commit(1, 6, 3) == 0
     assert m.query(1)[1][:2] == (16, 3)
     assert m.free_pages() == 3                              # 16 tokens fit one page: the second went back
+
+
+def test_page_manager_goes_back_to_a_base_length():
+    # Random walk with requests that continue an earlier length of their context (a resent draft): the manager is
+    # compared, after every operation, with plain Python lists holding each context's token history.
+    rng = np.random.default_rng(7)
+    n_pages, ps = 48, 16
+    m = B.KvManager(n_pages, ps)
+    hist = {}                                               # ctx -> (hist_start, [tokens from there on]); last = pending
+    nxt = 1
+    n_back = 0
+    for step in range(3000):
+        op = rng.integers(0, 10)
+        if op < 2 and len(hist) < 6:
+            n_kv = int(rng.integers(0, 60))
+            if m.open(nxt, n_kv, 7) == 0:
+                hist[nxt] = (n_kv, [7])
+            nxt += 1
+        elif op < 9 and hist:
+            ids = [int(x) for x in rng.choice(list(hist), size=min(len(hist), int(rng.integers(1, 4))), replace=False)]
+            ks = [int(rng.integers(0, 9)) for _ in ids]
+            base = []
+            for ctx in ids:
+                start, toks = hist[ctx]
+                n = start + len(toks)                       # committed tokens
+                r = rng.integers(0, 4)
+                base.append(0 if r == 0 else int(rng.integers(start + 1, n + 1)) if r < 3 else
+                            int(rng.choice([start, n + 1])))   # the last two are out of range
+            free_before = m.free_pages()
+            before = {ctx: m.query(ctx)[1] for ctx in ids}
+            rc = m.reserve_batch(ids, [k + 1 for k in ks], base)
+            bad = any(b != 0 and not (hist[c][0] + 1 <= b <= hist[c][0] + len(hist[c][1])) for c, b in zip(ids, base))
+            if bad:
+                assert rc == B.SLED_ERR_BASE_LEN
+            if rc != 0:
+                assert rc in (B.SLED_ERR_BASE_LEN, B.SLED_ERR_NO_PAGES) and m.free_pages() == free_before
+                for ctx in ids:                             # a refused batch changed nothing
+                    q = m.query(ctx)[1]
+                    assert q[:2] == before[ctx][:2] and list(q[2]) == list(before[ctx][2])
+                    assert m.history(ctx)[1] == (hist[ctx][0], hist[ctx][1])
+                continue
+            for ctx, b in zip(ids, base):
+                if b:
+                    start, toks = hist[ctx]
+                    n_back += b < start + len(toks)
+                    hist[ctx] = (start, toks[:b - start])
+            for ctx, k in zip(ids, ks):
+                start, toks = hist[ctx]
+                n_kv, pending = start + len(toks) - 1, toks[-1]
+                q = m.query(ctx)[1]
+                assert q[:2] == (n_kv, pending) and len(q[2]) == (n_kv + k + 1 + ps - 1) // ps
+                drafts = [int(x) for x in rng.integers(100, 200, k)]
+                n_acc = int(rng.integers(0, k + 1))
+                new = int(rng.integers(200, 300))
+                assert m.commit(ctx, n_acc + 1, new, drafts) == 0
+                hist[ctx] = (start, toks + drafts[:n_acc] + [new])
+        elif hist:
+            ctx = int(rng.choice(list(hist)))
+            assert m.release(ctx) == 0
+            del hist[ctx]
+        live = {c: (s + len(t) - 1, t[-1]) for c, (s, t) in hist.items()}
+        _check_invariants(m, live, n_pages, ps)
+        for c, (s, t) in hist.items():
+            assert m.history(c)[1] == (s, t)
+    assert n_back > 100                                      # the walk did go back many times
+    # a commit that does not say which tokens were kept restarts the known history at the new pending token
+    m2 = B.KvManager(8, 16)
+    assert m2.open(1, 3, 9) == 0 and m2.reserve_batch([1], [4]) == 0
+    assert m2.commit(1, 3, 5) == 0
+    assert m2.history(1)[1] == (6, [5])
+    assert m2.reserve_batch([1], [1], [6]) == B.SLED_ERR_BASE_LEN and m2.reserve_batch([1], [1], [7]) == 0

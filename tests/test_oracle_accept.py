@@ -254,3 +254,45 @@ def test_chi_square_detects_a_planted_mistake():
         counts[draws[i] if n_acc >= 1 else nxt] += 1
     chi2 = ((counts - n * p) ** 2 / (n * p)).sum()
     assert chi2 > stats.chi2.ppf(1 - 1e-3, V - 1)
+
+
+# ------------------------------------------------ draft rows sent in 16 bits: how far from lossless --
+def _law_with_reported_q(p, q_true, q_sent):
+    """Distribution of the first committed token when the device draws d ~ q_true but the server applies Eq. 1 and
+    the residual with q_sent (all exact fp64): sum_d q_true(d) [a_d 1{x=d} + (1 - a_d) res(x)], a_d = min(1, p_d /
+    q_sent_d), res = norm(max(p - q_sent, 0))."""
+    a = np.minimum(1.0, p / q_sent)
+    res = np.maximum(p - q_sent, 0.0)
+    res = res / res.sum()
+    return q_true * a + (q_true * (1.0 - a)).sum() * res
+
+
+def test_bf16_draft_rows_deviate_by_their_rounding_and_no_more():
+    import torch
+    rng = np.random.default_rng(8)
+    worst = 0.0
+    for trial in range(200):
+        V = int(rng.integers(8, 400))
+        p = _softmax64((rng.standard_normal(V) * 2).astype(np.float32))
+        q = _softmax64((0.8 * np.log(p) + 0.6 * rng.standard_normal(V) * 2).astype(np.float32))
+        q16 = torch.from_numpy(q.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+        exact = _law_with_reported_q(p, q, q)
+        assert np.abs(exact - p).sum() < 1e-12                # with the true q the rule is lossless (Section 3.1)
+        tv = 0.5 * np.abs(_law_with_reported_q(p, q, q16) - p).sum()
+        assert 0.0 < tv <= 2.0 ** -8                          # rounded q: off by at most the relative rounding step
+        worst = max(worst, tv)
+    assert worst > 2.0 ** -14                                  # the bound is not vacuous: the deviation is real
+    # the oracle applied to 16-bit rows follows that law, not p: the chi-square test against the predicted law passes
+    V, n = 24, 120000
+    z = (rng.standard_normal((2, V)) * 1.5).astype(np.float32)
+    p = _softmax64(z[0])
+    q64 = _softmax64((rng.standard_normal(V) * 1.5).astype(np.float32))
+    q16 = torch.from_numpy(q64.astype(np.float32)).to(torch.bfloat16).to(torch.float32).numpy()
+    law = _law_with_reported_q(p, q64, q16.astype(np.float64))
+    draws = rng.choice(V, size=n, p=q64)
+    counts = np.zeros(V)
+    for i in range(n):
+        st, n_acc, nxt, _ = O.accept(z, q16[None, :], np.array([draws[i]], np.int32), 1.0, False, 31, i, 3)
+        counts[draws[i] if n_acc >= 1 else nxt] += 1
+    chi2 = ((counts - n * law) ** 2 / (n * law)).sum()
+    assert chi2 < stats.chi2.ppf(1 - 1e-3, V - 1), chi2
