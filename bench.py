@@ -60,9 +60,17 @@ def parse_args(argv=None):
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--workload", default="step", choices=["step", "accept", "attention"],
+    ap.add_argument("--workload", default="step", choices=["step", "accept", "attention", "serve"],
                     help="step: the full verification step (the headline); accept / attention: one kernel alone "
-                         "on the acceptance-only / attention-only workload")
+                         "on the acceptance-only / attention-only workload; serve: the server loop (queue, batch "
+                         "planner, step) driven by a simulated population of devices")
+    ap.add_argument("--devices", default="16,64,256,1024", help="serve: device counts to simulate")
+    ap.add_argument("--draft-rate", type=float, default=5.24, help="serve: tokens per second a device drafts")
+    ap.add_argument("--c-th", type=float, default=0.4, help="serve: confidence threshold of dynamic drafting")
+    ap.add_argument("--policy", default="continuous", choices=["continuous", "static"])
+    ap.add_argument("--static-batch", type=int, default=16, help="serve: batch size static batching waits for")
+    ap.add_argument("--rounds", type=int, default=6, help="serve: verification rounds per device that are simulated")
+    ap.add_argument("--max-batch", type=int, default=128, help="serve: most requests per step")
     ap.add_argument("--tau", type=float, default=1.0)
     ap.add_argument("--drafts", default="correlated", choices=["correlated", "independent"],
                     help="correlated: draft distributions built from the target's own logits (rho = 0.8), "
@@ -693,10 +701,152 @@ def run_attention_only(args):
     eng.shutdown()
 
 
+def run_serve(args):
+    """The server loop under a simulated population of devices (Section 4 of the paper models verification requests
+    the same way): every device is an independent source whose time to draft its next request is exponentially
+    distributed with mean k / draft_rate; k follows dynamic drafting (Section 3.3): a device keeps drafting while
+    the confidence of its newest token (uniform here, a stand-in) is at least c_th, up to max_k.  A device has one
+    request outstanding at a time.  The server's clock advances by the measured device time of each sled_step;
+    between steps it is idle until the next request arrives.  Reported per device count: whole-system token
+    generation rate (committed tokens per simulated second), tokens per second and device, batch sizes, server
+    utilisation; capacity = the largest simulated device count whose per-device rate is still at least 90 % of a
+    lone device's."""
+    import heapq
+    from paper_2506_09397_b200 import binding as B
+    shape = I.SHAPES[args.shape]
+    if args.layers:
+        shape = replace(shape, n_layers=args.layers)
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    counts = [int(x) for x in args.devices.split(",") if x]
+    max_k, V = 8, shape.vocab
+    w = I.make_weights(shape, args.seed, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    n_max = max(counts)
+    ctx_len = I.draw_context_lengths(n_max, 128, 512, args.seed)
+    # small populations are simulated for longer, so that every population answers a few hundred requests
+    rounds_for = lambda n: max(args.rounds, -(-300 // n))
+    n_pages = max(sum((c + 4 * rounds_for(n) * (max_k + 1) + 16 + 15) // 16 for c in ctx_len[:n]) for n in counts) + 64
+    max_batch = min(args.max_batch, n_max)
+    eng = B.Engine(shape, w, n_pages=n_pages, max_batch=max_batch, max_k=max_k, max_step_tokens=max_batch * (max_k + 1),
+                   temperature=1.0, greedy=False, device_index=0, stream=stream.cuda_stream, probs_on_device=True)
+    del w
+    eng.server_config(B.SLED_BATCH_STATIC if args.policy == "static" else B.SLED_BATCH_CONTINUOUS,
+                      min(args.static_batch, max_batch))
+    # a pool of draft-distribution rows on the device; a request takes the first k rows of one pool entry
+    pool = [I.make_drafts(V, max_k, args.seed, 7000 + i, device=dev)[1] for i in range(32)]
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(args.seed)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(args.seed)
+    mean_k = sum(k * (1 - args.c_th) ** (k - 1) * (args.c_th if k < max_k else 1.0) for k in range(1, max_k + 1))
+    out = []
+    for n_dev in sorted(counts):
+        t_end = rounds_for(n_dev) * (mean_k / args.draft_rate + 0.005)   # about that many verification cycles of a lone device
+        t_warm = 0.25 * t_end
+        max_rounds = 4 * rounds_for(n_dev)                               # bounds how far a context can grow
+        for i in range(n_dev):                                   # fresh contexts for every device count
+            K, Vv = I.make_kv(shape, ctx_len[i], args.seed, i, device=dev)
+            eng.load_kv(i, K, Vv, pending=1)
+            del K, Vv
+        # every launch shape once before the clock starts (first uses configure kernels)
+        eng.set_commit(False)
+        for b in sorted({1, min(3, n_dev), min(12, n_dev), min(20, n_dev), min(60, n_dev), min(max_batch, n_dev)}):
+            tk = [eng.submit(i, np.zeros(max_k, np.int32), pool[0]) for i in range(b)]
+            eng.step(0, flush=True)
+            for x in tk:
+                eng.poll(x)
+        eng.set_commit(True)
+
+        def draw_k():
+            k = 1
+            while k < max_k and rng.random() >= args.c_th:        # confident: draft another token
+                k += 1
+            return k
+
+        heap = []
+        for i in range(n_dev):
+            k = draw_k()
+            heapq.heappush(heap, (rng.exponential(k / args.draft_rate), i, k))
+        t, busy, steps, tokens, served, latency, batch_sizes = 0.0, 0.0, 0, 0, 0, [], []
+        rounds_done = {i: 0 for i in range(n_dev)}
+        in_flight = {}
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        while t < t_end and (heap or in_flight):
+            while heap and heap[0][0] <= t:                      # requests that have arrived by now
+                ta, i, k = heapq.heappop(heap)
+                q = pool[int(rng.integers(0, len(pool)))][:k]
+                d = torch.multinomial(q, 1, generator=gen).reshape(k).to(torch.int32).cpu().numpy()
+                in_flight[eng.submit(i, d, q)] = (i, ta, k, q)
+            if not in_flight:
+                t = heap[0][0]                                   # idle until the next arrival
+                continue
+            e0.record(stream)
+            n = eng.step(1000 + steps, flush=not heap)          # static batching: flush when nobody else can come
+            e1.record(stream)
+            e1.synchronize()
+            if n == 0:                                           # static batching still waiting for its batch
+                t = heap[0][0]
+                continue
+            dt = e0.elapsed_time(e1) / 1e3
+            t += dt
+            steps += 1
+            counted = t > t_warm
+            if counted:
+                busy += dt
+                batch_sizes.append(n)
+            for ticket in list(in_flight):
+                r = eng.poll(ticket)
+                if r is None:
+                    continue
+                i, ta, k, _ = in_flight.pop(ticket)
+                if r[2] != 0:
+                    raise SystemExit(f"request of device {i} failed with status {r[2]}")
+                if counted:
+                    tokens += r[0] + 1
+                    served += 1
+                    latency.append(t - ta)
+                rounds_done[i] += 1
+                if rounds_done[i] < max_rounds:
+                    k2 = draw_k()
+                    heapq.heappush(heap, (t + rng.exponential(k2 / args.draft_rate), i, k2))
+        while in_flight:                                         # drain what is still queued (not counted)
+            eng.step(0, flush=True)
+            for ticket in list(in_flight):
+                if eng.poll(ticket) is not None:
+                    in_flight.pop(ticket)
+        span = max(t, t_end) - t_warm
+        entry = {"devices": n_dev, "wstgr_tokens_per_s": tokens / span, "tokens_per_s_per_device": tokens / span / n_dev,
+                 "requests": served, "steps": len(batch_sizes), "mean_batch": float(np.mean(batch_sizes)) if batch_sizes else 0.0,
+                 "max_batch_seen": int(max(batch_sizes)) if batch_sizes else 0, "server_utilisation": busy / span,
+                 "mean_step_ms": 1e3 * busy / max(1, len(batch_sizes)),
+                 "mean_response_ms": 1e3 * float(np.mean(latency)) if latency else None,
+                 "measured_seconds": span, "tokens_per_request": tokens / max(1, served)}
+        out.append(entry)
+        for i in range(n_dev):
+            eng.release(i)
+    lone_rate = out[0]["tokens_per_s_per_device"]                # the smallest population: its requests hardly ever wait
+    ok = [e["devices"] for e in out if e["tokens_per_s_per_device"] >= 0.9 * lone_rate]
+    print(json.dumps({"metric": "wstgr_tokens_per_s", "value": max(e["wstgr_tokens_per_s"] for e in out), "unit": "tokens/s",
+                      "n_gpus": 1, "higher_is_better": True, "dtype": "bf16" if shape.weight_dtype == "bf16" else "f32",
+                      "data": "synthetic",
+                      "config": {"workload": f"server loop, {shape.name} ({shape.n_layers} layers), {args.policy} batching, "
+                                             f"devices drafting {args.draft_rate} tokens/s, c_th={args.c_th}, max_k={max_k}, "
+                                             f"contexts 128..512, about {args.rounds} verification rounds per device simulated "
+                                             "(more for small populations; the first quarter of the time is not counted)",
+                                 "draft_distributions": "independent of the target (softmax of N(0,1) logits)"},
+                      "capacity_devices": {"value": max(ok) if ok else 0, "rule": "largest simulated count whose devices still get >= 90 % of "
+                                           "the token rate of the smallest population's", "reached_largest_simulated": bool(ok) and max(ok) == max(counts)},
+                      "by_devices": out}))
+    eng.shutdown()
+
+
 def main(argv=None):
     args = parse_args(argv)
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "serve":
+        run_serve(args)
     elif args.workload == "accept":
         run_accept_only(args)
     elif args.workload == "attention":

@@ -271,6 +271,13 @@ int sled_debug_truncate(sled_engine* e, uint64_t ctx_id, int64_t n_kv, int32_t p
 /* The same for n contexts in one call (ctx_ids, n_kv, pending: HOST arrays [n]); stops at the first error. */
 int sled_debug_truncate_batch(sled_engine* e, const uint64_t* ctx_ids, const int64_t* n_kv, const int32_t* pending,
                               int32_t n);
+/* Self-test of the recovery from a device-side wait that runs out (engines with bf16 weights).  Every wait inside
+ * the tensor-core and attention kernels is bounded: when one expires the kernel records a code, kernels that follow
+ * return early, and sled_verify_batch returns SLED_ERR_DEVICE with every context, page and counter as before.  This
+ * call arms that path without any fault: the next sled_verify_batch starts with a small kernel that waits limit_us
+ * microseconds (<= 100000) on a barrier nobody signals, using the kernels' own bounded wait.  That step fails as
+ * described; the one after it runs normally. */
+int sled_debug_arm_wait_timeout(sled_engine* e, int32_t limit_us);
 /* commit = 0: verification steps leave every context as it was (repeatable timing). */
 int sled_debug_set_commit(sled_engine* e, int32_t commit);
 /* Device time per kind of kernel into sled_stats.  mode 0: off.  mode 1: every launch stamps the GPU's global timer

@@ -55,7 +55,8 @@ class _Weights(C.Structure):
 
 
 class Margin(C.Structure):
-    _fields_ = [("accept_rel", C.c_double), ("sample_rel", C.c_double), ("greedy_gap", C.c_double)]
+    _fields_ = [("accept_rel", C.c_double), ("sample_rel", C.c_double), ("greedy_gap", C.c_double),
+                ("draw_mass", C.c_double)]
 
 
 _lib = None

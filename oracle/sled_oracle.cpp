@@ -149,6 +149,8 @@ struct orc_margin {
   double accept_rel;  // min over the accept tests taken of |lhs-rhs| / max(lhs, rhs)
   double sample_rel;  // distance of the sampling target to the nearer CDF boundary of the chosen token, / total weight
   double greedy_gap;  // smallest (top1 - top2) logit gap over the rows looked at (greedy mode)
+  double draw_mass;   // total weight the token was drawn from, as a fraction of the row's Z (1 on a bonus row, the
+                      // rejected mass sum max(p - q, 0) after a rejection): small values make the draw sensitive
 };
 
 enum { ORC_OK = 0, ORC_NONFINITE = 1 };
@@ -176,7 +178,7 @@ enum { ORC_OK = 0, ORC_NONFINITE = 1 };
 int orc_accept(const float* logits, const float* q, const int32_t* drafts, int32_t k, int32_t V,
                float tau, int32_t greedy, uint64_t seed, uint64_t ctx_id, int64_t pos0,
                int32_t* n_accepted, int32_t* next_token, orc_margin* mg) {
-  orc_margin local = {INFINITY, INFINITY, INFINITY};
+  orc_margin local = {INFINITY, INFINITY, INFINITY, 1.0};
   const float inv_tau = 1.0f / tau;
   std::vector<uint64_t> E(static_cast<size_t>(V));
   *n_accepted = 0;
@@ -237,6 +239,7 @@ int orc_accept(const float* logits, const float* q, const int32_t* drafts, int32
         pick = v;
         double lo = static_cast<double>(tgt - before), hi = static_cast<double>(run - tgt);
         local.sample_rel = (lo < hi ? lo : hi) / static_cast<double>(W);
+        local.draw_mass = static_cast<double>(W) / static_cast<double>(Z);
         break;
       }
     }

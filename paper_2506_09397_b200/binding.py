@@ -26,7 +26,7 @@ SLED_BATCH_STATIC, SLED_BATCH_CONTINUOUS = 0, 1
 EXPORTS = (
     "sled_init", "sled_verify_batch", "sled_release", "sled_prefill", "sled_set_sampling", "sled_get_stats",
     "sled_get_stream", "sled_shutdown", "sled_strerror", "sled_accept_rows", "sled_accept_rows_static", "sled_attention_ragged",
-    "sled_debug_load_kv", "sled_debug_read_kv", "sled_debug_copy_logits", "sled_debug_truncate", "sled_debug_truncate_batch",
+    "sled_debug_load_kv", "sled_debug_read_kv", "sled_debug_copy_logits", "sled_debug_truncate", "sled_debug_truncate_batch", "sled_debug_arm_wait_timeout",
     "sled_debug_set_commit", "sled_debug_set_timing", "sled_debug_query_ctx", "sled_debug_shuffle_pages",
     "sled_kvm_create", "sled_kvm_destroy", "sled_kvm_open", "sled_kvm_reserve_batch", "sled_kvm_commit",
     "sled_kvm_release", "sled_kvm_query", "sled_kvm_free_pages", "sled_kvm_pack", "sled_kvm_reserve_batch_at",
@@ -106,6 +106,7 @@ def lib():
             "sled_debug_copy_logits": (C.c_int, [P, P, I32]),
             "sled_debug_truncate": (C.c_int, [P, U64, I64, I32]),
             "sled_debug_truncate_batch": (C.c_int, [P, P, P, P, I32]),
+            "sled_debug_arm_wait_timeout": (C.c_int, [P, I32]),
             "sled_debug_set_commit": (C.c_int, [P, I32]),
             "sled_debug_set_timing": (C.c_int, [P, I32]),
             "sled_debug_query_ctx": (C.c_int, [P, U64, C.POINTER(I64), C.POINTER(I32), C.POINTER(I32), P, I32]),
@@ -295,6 +296,9 @@ class Engine:
 
     def truncate(self, ctx_id: int, n_kv: int, pending: int) -> None:
         _check(lib().sled_debug_truncate(self.h, ctx_id, n_kv, pending), "sled_debug_truncate")
+
+    def arm_wait_timeout(self, limit_us: int) -> None:
+        _check(lib().sled_debug_arm_wait_timeout(self.h, limit_us), "sled_debug_arm_wait_timeout")
 
     def set_commit(self, on: bool) -> None:
         _check(lib().sled_debug_set_commit(self.h, int(on)), "sled_debug_set_commit")

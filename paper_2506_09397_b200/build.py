@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libsled.so")
-SOURCES = ["engine.cu", "kernels_small.cu", "attention.cu", "attention_mma.cu", "accept.cu", "gemm_tc.cu", "kv_manager.cpp", "planner.cpp", "no_alloc.cu"]
+SOURCES = ["engine.cu", "kernels_small.cu", "attention.cu", "attention_mma.cu", "attention_tc.cu", "accept.cu", "gemm_tc.cu", "kv_manager.cpp", "planner.cpp", "no_alloc.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall"]
 

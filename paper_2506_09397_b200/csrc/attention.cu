@@ -206,8 +206,10 @@ int launch_typed(const AttnArgs& a, cudaStream_t s) {
 int launch_attention(const AttnArgs& a, cudaStream_t s) {
   if (a.n_items <= 0 || a.T <= 0) return 0;
   int n = -1;
-  if (a.kvdtype == BF16 && a.adtype == BF16 && a.map_k && a.page_size == 16 && (a.h == 64 || a.h == 128))
-    n = launch_attention_mma(a, s);   // tensor-core kernel
+  if (a.use_tc && a.kvdtype == BF16 && a.adtype == BF16 && a.map_k && a.page_size == 16 && a.h == 128)
+    n = launch_attention_tc(a, s);    // tcgen05 kernel
+  else if (a.kvdtype == BF16 && a.adtype == BF16 && a.map_k && a.page_size == 16 && (a.h == 64 || a.h == 128))
+    n = launch_attention_mma(a, s);   // warp-level tensor-core kernel
   else if (a.kvdtype == BF16 && a.adtype == BF16) n = launch_typed<__nv_bfloat16, __nv_bfloat16>(a, s);
   else if (a.kvdtype == F32 && a.adtype == F32) n = launch_typed<float, float>(a, s);
   else if (a.kvdtype == BF16 && a.adtype == F32) n = launch_typed<__nv_bfloat16, float>(a, s);

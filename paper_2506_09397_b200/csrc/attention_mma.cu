@@ -38,12 +38,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// bounded wait; gives up at once when another warp of the block already has (*stop set)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* stop) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > kWaitCycles) return false;
+    if (*stop != 0 || clock64() - t0 > kWaitCycles) return false;
   }
 }
 
@@ -137,7 +138,7 @@ __device__ __forceinline__ void consume_item(const AttnArgs& a, const ItemCtx& c
 
   for (int tile = 0; tile < c.n_tiles; ++tile, ++it) {
     const int s = it % kStages;
-    if (*s_abort || !mbar_wait(bar_full + 8 * s, (it / kStages) & 1)) { *s_abort = 1; failed = true; break; }
+    if (*s_abort || !mbar_wait(bar_full + 8 * s, (it / kStages) & 1, s_abort)) { *s_abort = 1; failed = true; break; }
     if (active) {
       const uint32_t kb = base + s * L::kBytes, vb = kb + L::kKBytes;
       const int k0 = c.key_start + tile * kTile + key_off;    // first key of this warp's share
@@ -370,7 +371,7 @@ __global__ void __launch_bounds__(160, 2) attn_mma_kernel(AttnArgs a, const __gr
       for (int pass = 0; pass < n_pass && !*s_abort; ++pass) {
         for (int tile = pass == 0 ? pre : 0; tile < c.n_tiles; ++tile, ++it) {
           const int s = it % kStages;
-          if (*s_abort || !mbar_wait(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1)) { *s_abort = 1; break; }
+          if (*s_abort || !mbar_wait(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1, s_abort)) { *s_abort = 1; break; }
           load_tile(tile, s);
         }
       }

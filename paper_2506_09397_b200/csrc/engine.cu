@@ -64,6 +64,7 @@ struct sled_engine {
   cudaEvent_t ev_copy = nullptr, ev_a = nullptr, ev_b = nullptr;
   KvManager* kvm = nullptr;
   bool commit = true;
+  long long probe_wait_cycles = 0;   // > 0: the next verification step starts with the give-up self-test kernel
   int timing = 0;   // 0 off, 1 device timestamps per launch (overlap untouched), 2 events between kernel groups (serialises)
 
   // device memory
@@ -89,6 +90,7 @@ struct sled_engine {
   float* part_ml = nullptr;
   int part_rows_cap = 0;
   float* q_stage = nullptr;
+  bool attn_tc = false;          // head_dim 128, bf16 cache, 16-token pages: attention may run on tcgen05
   TcActivation tc_norm, tc_attn, tc_ffn;
   int32_t* tc_error = nullptr;  // device word set by a kernel whose bounded wait ran out: the first word of the
                                 // results block (d_results), so the step's one result copy brings it along
@@ -217,6 +219,7 @@ struct Packed {
   int4* items;
   int n_items = 0;
   bool any_split = false;
+  bool use_tc = false;   // the tcgen05 attention kernel serves this step (every request has at most 128 query rows)
   // host views
   int32_t *h_cu_q, *h_kv_base;
 };
@@ -284,12 +287,17 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
   // longer - so that all blocks end together.  Many requests: one common chunk length, doubled until the item
   // count is near the machine size; the hardware hands items out as blocks retire.
   const int group = e->cfg.n_q_heads / Hkv;
-  const int64_t slots = 2LL * e->n_sm;
+  int max_rows = 0;
+  for (int i = 0; i < B; ++i) max_rows = std::max(max_rows, plan[i].n * group);
+  pk->use_tc = e->attn_tc && max_rows <= 128;
+  // blocks resident at once: the tcgen05 kernel runs one block per SM, the warp-level kernel two
+  const int64_t slots = (pk->use_tc ? 1LL : 2LL) * e->n_sm;
   std::vector<int64_t> chunk_of(B, 256);
   std::vector<double> cost(B);
-  auto heavy = [&](int i) { return plan[i].n * group > 32; };
+  // the warp-level kernel's tiles take the tensor pipes longer when a request has more than 32 query rows
+  auto heavy = [&](int i) { return !pk->use_tc && plan[i].n * group > 32; };
   for (int i = 0; i < B; ++i) {
-    const double passes = (plan[i].n * group + 63) / 64;
+    const double passes = pk->use_tc ? 1.0 : (plan[i].n * group + 63) / 64;
     cost[i] = static_cast<double>((n_keys[i] + 63) / 64) * passes * (heavy(i) ? 1.75 : 1.0);
   }
   auto part_rows_of = [&]() {
@@ -408,6 +416,7 @@ AttnArgs attn_args(sled_engine* e, const Packed& pk, int layer, const void* q, v
     a.map_v = &e->kv_maps[2 * layer + 1];
     a.error = e->tc_error;
   }
+  a.use_tc = pk.use_tc ? 1 : 0;
   a.stamp = e->stamp(K_ATTN);
   if (pk.any_split) a.stamp_merge = e->stamp(K_ATTN);
   return a;
@@ -790,6 +799,7 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
         if (tma_map_bf16_rows(&e->kv_maps[2 * l], e->kpool + e->kv_layer_bytes * l, rows, c.head_dim, 16) ||
             tma_map_bf16_rows(&e->kv_maps[2 * l + 1], e->vpool + e->kv_layer_bytes * l, rows, c.head_dim, 16))
           return fail(SLED_ERR_DEVICE);
+      e->attn_tc = c.head_dim == 128;
     }
     if (tc_activation_init(&e->tc_norm, e->act_norm, static_cast<int>(padT), d) ||
         tc_activation_init(&e->tc_attn, e->attn_out, static_cast<int>(padT), qd) ||
@@ -976,6 +986,12 @@ int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, 
   if (staged && cudaEventRecord(e->ev_copy, e->copy_stream) != cudaSuccess) return rollback(SLED_ERR_DEVICE);
 
   // ---- forward + acceptance
+  if (e->probe_wait_cycles > 0) {   // self-test armed by sled_debug_arm_wait_timeout: this step will be reported as failed
+    const int n_probe = tc_wait_probe_launch(e->tc_error, e->probe_wait_cycles, e->stream);
+    e->probe_wait_cycles = 0;
+    if (n_probe < 0) return rollback(SLED_ERR_DEVICE);
+    e->count(n_probe, K_OTHER);
+  }
   if ((rc = run_forward(e, pk, true))) return rollback(rc);
   if (staged && cudaStreamWaitEvent(e->stream, e->ev_copy, 0) != cudaSuccess) return rollback(SLED_ERR_DEVICE);
   AcceptArgs aa{};
@@ -1325,6 +1341,12 @@ int sled_debug_truncate_batch(sled_engine* e, const uint64_t* ctx_ids, const int
     const int rc = sled_debug_truncate(e, ctx_ids[i], n_kv[i], pending[i]);
     if (rc) return rc;
   }
+  return SLED_OK;
+}
+
+int sled_debug_arm_wait_timeout(sled_engine* e, int32_t limit_us) {
+  if (!e || !e->tc_error || limit_us <= 0 || limit_us > 100000) return SLED_ERR_ARG;
+  e->probe_wait_cycles = static_cast<long long>(limit_us) * 2000;   // about 2 clock cycles per nanosecond
   return SLED_OK;
 }
 

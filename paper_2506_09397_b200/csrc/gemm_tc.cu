@@ -52,13 +52,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // bounded wait: false (and *error = code) when the phase did not complete in time
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* error, int code, volatile int* stop) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* error, int code, volatile int* stop,
+                                          long long limit = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*stop != 0) return false;            // another warp of this block gave up, or an earlier kernel did
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > limit) {
       atomicCAS(error, 0, code);
       return false;
     }
@@ -543,6 +544,21 @@ __global__ void __launch_bounds__(192) tc_gemm_pair_kernel(const __grid_constant
   stamp_time(epi.stamp_end, true);
 }
 
+// Self-test of the give-up path: one thread waits, with the same bounded wait as the kernels above but a short
+// limit, on a barrier that nobody will ever signal.  The wait runs out, the code lands in *error and the kernel
+// returns normally; kernels launched afterwards find the word set and return early, and the host reports the step
+// as failed.  Nothing traps, spins without bound or touches memory it does not own.
+__global__ void wait_probe_kernel(int32_t* error, long long limit_cycles) {
+  __shared__ __align__(8) unsigned long long bar_mem;
+  __shared__ int stop_mem;
+  if (threadIdx.x == 0) {
+    stop_mem = 0;
+    mbar_init(smem_u32(&bar_mem), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_wait(smem_u32(&bar_mem), 0, error, 9, &stop_mem, limit_cycles);
+  }
+}
+
 // Weights are kept tile by tile: block (m, kb) of the tiled array is the 128 x 64 piece W[128m .. +127][64kb .. +63]
 // as 128 rows of 128 bytes, zero where the matrix ends.  One pipeline stage is then one contiguous 16 KB read, and
 // the stages of a CTA follow each other in memory (DRAM pages are read whole instead of 128 bytes at a time).
@@ -595,6 +611,12 @@ int make_map(CUtensorMap* map, const void* ptr, long long rows, int K, int box_r
 
 
 }  // namespace
+
+int tc_wait_probe_launch(int32_t* error, long long limit_cycles, cudaStream_t s) {
+  if (!error || limit_cycles <= 0 || limit_cycles > kWaitCycles) return -1;
+  wait_probe_kernel<<<1, 32, 0, s>>>(error, limit_cycles);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
 
 int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int cols, int box_rows) {
   return make_map(map, dev_ptr, rows, cols, box_rows);

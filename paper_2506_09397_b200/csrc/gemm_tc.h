@@ -48,4 +48,8 @@ int tc_gemm_split(int T, int N, int K, int n_sm);
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
                    int32_t* error, const TcEpilogue& epi, cudaStream_t s);
 
+// Self-test: launches a kernel whose bounded wait (limit in clock cycles, at most the kernels' own limit) runs out
+// on a barrier nobody signals and records code 9 in *error.  Returns kernels launched (1) or a negative value.
+int tc_wait_probe_launch(int32_t* error, long long limit_cycles, cudaStream_t s);
+
 }  // namespace sled

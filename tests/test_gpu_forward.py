@@ -37,7 +37,11 @@ def _verify_both(eng, orc, reqs, seed, tau, greedy, tol, explain):
         st2, n2, x2, _ = O.accept(mine, None if greedy or k == 0 else q.numpy(), d.numpy(), tau, greedy, seed, c, pos0)
         assert (n2, x2) == g[:2] and g[2] == 0
         if (n_acc, nxt) != g[:2]:
-            assert rel_margin_ok(mg, tol), (c, (n_acc, nxt), g, mg.accept_rel, mg.sample_rel, mg.greedy_gap)
+            # the two sides may differ only where the logit deviation measured on the rows either side looked at can
+            # move the deciding comparison
+            upto = max(n_acc, g[0]) + 1
+            eps = float(np.max(np.abs(mine[:upto] - ologits[:upto])))
+            assert rel_margin_ok(mg, eps), (c, (n_acc, nxt), g, eps, mg.accept_rel, mg.sample_rel, mg.greedy_gap, mg.draw_mass)
             explain.append(c)
         # the oracle follows the GPU's decision so that both sides keep the same history
         oc = orc.ctx[c]
@@ -421,3 +425,35 @@ def test_draft_rows_in_bf16(where):
         row += k + 1
     assert any(g[0] < len(r[1]) for r, g in zip(reqs, got))      # a rejection happened: the residual read a 16-bit row
     eng.shutdown()
+
+
+def test_a_wait_that_runs_out_fails_the_step_and_nothing_else():
+    # every device-side wait is bounded; this arms the give-up path on purpose (a kernel waits 2 ms on a barrier
+    # nobody signals and returns with its error code): the step must come back as a device error with every
+    # context untouched, and the next step on the same engine must be an ordinary, correct one
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=12)
+    eng = _engine(shape, w)
+    orc = O.OracleModel(shape, oracle_weights(w))
+    ctxs = [71, 72, 73]
+    for c in ctxs:
+        p = I.make_prompt(shape.vocab, 15 + c % 5, 12, c)
+        eng.prefill(c, p)
+        orc.prefill(c, p)
+    reqs = [(c,) + tuple(I.make_drafts(shape.vocab, 5, 12, c)) for c in ctxs]
+    explain = []
+    _verify_both(eng, orc, reqs, seed=1, tau=1.0, greedy=False, tol=2e-2, explain=explain)
+    before = [str(eng.query_ctx(c)) for c in ctxs] + [eng.stats().pages_free, eng.stats().steps]
+    reqs = [(c,) + tuple(I.make_drafts(shape.vocab, 4, 12, c, step=1)) for c in ctxs]
+    eng.arm_wait_timeout(2000)
+    with pytest.raises(B.SledError) as ei:
+        eng.verify_batch([(c, d.numpy(), q.numpy()) for c, d, q in reqs], 2)
+    assert ei.value.code == B.SLED_ERR_DEVICE
+    assert before == [str(eng.query_ctx(c)) for c in ctxs] + [eng.stats().pages_free, eng.stats().steps]
+    _verify_both(eng, orc, reqs, seed=2, tau=1.0, greedy=False, tol=2e-2, explain=explain)   # the same requests, now served
+    eng.shutdown()
+    # the fp32 configuration has no such waits: arming is refused
+    eng32 = _engine(I.TINY, I.make_weights(I.TINY, seed=0))
+    with pytest.raises(B.SledError):
+        eng32.arm_wait_timeout(1000)
+    eng32.shutdown()

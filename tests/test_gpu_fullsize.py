@@ -12,15 +12,25 @@ from util import oracle_weights
 pytestmark = pytest.mark.gpu
 
 
-def _full_step(shape, batch, ks, ctx, seed, check):
-    """One verification step of `shape` with synthetic cache content; requests in `check` are recomputed
-    by the oracle (logit deviation no larger than what bf16 rounding of the activations explains,
-    decisions bit-exact on the GPU's logits)."""
+def _full_step(shape, batch, ks, ctx, seed, check, greedy=False, gpu_vs_rounded=None):
+    """One verification step of `shape` with synthetic cache content; the requests in `check` are recomputed by the
+    oracle in both of its evaluation modes.  Asserted per checked request:
+      * against the exact oracle: the GPU's logits deviate by what rounding the inputs of the matrix products to
+        bf16 produces, and no more (at most 1.15 of the rounded oracle's own deviation; measured 1.01-1.06);
+      * against the rounded oracle (which rounds at the same points): the two are two realisations of the same
+        rounding noise, at most as far apart as independent ones would be (factor sqrt 2; measured 0.9-1.2, bound
+        1.3).  They are not closer than that, even in a two-layer model (measured 0.93): fp32 accumulation puts the
+        GPU's value a few 1e-6 away from the oracle's ahead of a rounding, which flips one rounding in a thousand;
+        each flip is a full rounding step, so ahead of the next rounding the two differ by 1e-4, which flips one in
+        forty there, and after three or four rounding points the two round independently;
+      * decisions bit-exact on the GPU's own logits."""
+    if gpu_vs_rounded is None:
+        gpu_vs_rounded = FULL_DEPTH
     dev = "cuda"
     w = I.make_weights(shape, seed, device=dev)
     T = sum(k + 1 for k in ks)
     n_pages = sum((c + k + 1 + 15) // 16 for c, k in zip(ctx, ks)) + 8
-    eng = B.Engine(shape, w, n_pages=n_pages, max_batch=batch, max_k=max(ks), max_step_tokens=T)
+    eng = B.Engine(shape, w, n_pages=n_pages, max_batch=batch, max_k=max(ks), max_step_tokens=T, greedy=greedy)
     eng.shuffle_pages(seed)
     kv_host = {}
     reqs = []
@@ -31,36 +41,37 @@ def _full_step(shape, batch, ks, ctx, seed, check):
             kv_host[i] = (K.float().cpu().numpy(), V.float().cpu().numpy())
         del K, V
         d, q = I.make_drafts(shape.vocab, ks[i], seed, i, device=dev)
-        reqs.append((i, d.cpu().numpy(), q))
+        reqs.append((i, d.cpu().numpy(), None if greedy else q))
+        if i in check and not greedy:
+            kv_host[i] += (q.cpu().numpy(),)
     got = eng.verify_batch(reqs, seed=5)
     logits = eng.logits(T)
     w_host = oracle_weights(I.weights_to(w, "cpu"))
     del w
-    # two oracle evaluations: the reference one, and the separately reported mode that rounds the inputs of the
-    # matrix products to bf16 at the points a 16-bit implementation must (it measures how much of the difference
-    # is rounding of activations, which grows with the square root of the depth)
     orc = O.OracleModel(shape, w_host)
     orc_r = O.OracleModel(shape, w_host, round_acts=True)
+    rms = lambda a: float(np.sqrt(np.mean(a.astype(np.float64) ** 2)))
     row = 0
     for i in range(batch):
         k = ks[i]
         if i in check:
-            qh = reqs[i][2].cpu().numpy()
             orc.load_kv(i, kv_host[i][0], kv_host[i][1], pending=7 + i)
             orc_r.load_kv(i, kv_host[i][0], kv_host[i][1], pending=7 + i)
             ol = orc.score(i, reqs[i][1])
             ol_r = orc_r.score(i, reqs[i][1])
+            orc.release(i)
+            orc_r.release(i)
             mine = logits[row:row + k + 1]
-            rms = lambda a: float(np.sqrt(np.mean(a.astype(np.float64) ** 2)))
-            e_gpu, e_round = rms(mine - ol), rms(ol_r - ol)
-            m_gpu, m_round = float(np.max(np.abs(mine - ol))), float(np.max(np.abs(ol_r - ol)))
-            print(f"{shape.name} request {i}: gpu-vs-oracle rms {e_gpu:.4f} max {m_gpu:.4f}; rounding alone rms {e_round:.4f} max {m_round:.4f}")
-            # the GPU's deviation is no larger than what the documented rounding points produce by themselves
-            assert e_gpu <= 1.5 * e_round + 1e-3, (e_gpu, e_round)
+            e_gpu, e_round, e_gr = rms(mine - ol), rms(ol_r - ol), rms(mine - ol_r)
+            m_gpu, m_round, m_gr = (float(np.max(np.abs(x))) for x in (mine - ol, ol_r - ol, mine - ol_r))
+            print(f"{shape.name} B={batch} request {i} (k={k}, context {ctx[i]}): gpu-exact rms {e_gpu:.4f} max {m_gpu:.4f}; "
+                  f"rounded-exact rms {e_round:.4f} max {m_round:.4f}; gpu-rounded rms {e_gr:.4f} max {m_gr:.4f}")
+            assert e_gr <= gpu_vs_rounded * e_round + 1e-3, (e_gr, e_round)
+            assert e_gpu <= 1.15 * e_round + 1e-3, (e_gpu, e_round)
             assert m_gpu <= 1.5 * m_round + 5e-3, (m_gpu, m_round)
             assert e_gpu <= 0.012 * shape.n_layers ** 0.5 * max(1.0, float(ol.std()))
             # bit-exact decision on identical logits
-            st2, n2, x2, _ = O.accept(mine, qh, reqs[i][1], 1.0, False, 5, i, ctx[i])
+            st2, n2, x2, _ = O.accept(mine, None if greedy else kv_host[i][2], reqs[i][1], 1.0, greedy, 5, i, ctx[i])
             assert st2 == 0 and (n2, x2, 0) == got[i]
         row += k + 1
     assert np.isfinite(logits).all() and np.abs(logits).max() > 0.5
@@ -71,28 +82,69 @@ def _full_step(shape, batch, ks, ctx, seed, check):
     torch.cuda.empty_cache()
 
 
+# bound on rms(gpu - rounded oracle) / rms(rounded oracle - exact oracle), see _full_step
+FULL_DEPTH = 1.3
+
+
+def _pick(ks, ctx, n=3):
+    """Requests to recompute: the cheapest one, the one with the longest context, and one with the most drafts."""
+    cheap = int(np.argmin([c + 100 * k for c, k in zip(ctx, ks)]))
+    longest = int(np.argmax(ctx))
+    most = int(np.argmax([k * 10000 - c for c, k in zip(ctx, ks)]))
+    return set([cheap, longest, most][:n])
+
+
+def test_llama8b_shapes_two_layers():
+    # the full-size matrices, vocabulary and batches with only two layers (more requests recomputed per second of oracle)
+    from dataclasses import replace
+    shape = replace(I.LLAMA_8B, n_layers=2)
+    ks = I.draw_k(16, [3, 5, 8], 0)
+    ctx = I.draw_context_lengths(16, 512, 4096, 0)
+    _full_step(shape, 16, ks, ctx, 0, check=_pick(ks, ctx) | {0, 5})
+    ks = I.draw_k(64, [3, 5, 8], 1)
+    ctx = I.draw_context_lengths(64, 512, 4096, 1)
+    _full_step(shape, 64, ks, ctx, 1, check=_pick(ks, ctx))
+
+
 def test_llama8b_step_batch16():
     shape = I.LLAMA_8B
     ks = I.draw_k(16, [3, 5, 8], 0)
     ctx = I.draw_context_lengths(16, 512, 4096, 0)
-    smallest = int(np.argmin([c + 100 * k for c, k in zip(ctx, ks)]))
-    _full_step(shape, 16, ks, ctx, 0, check={smallest})
+    _full_step(shape, 16, ks, ctx, 0, check=_pick(ks, ctx))
+
+
+def test_llama8b_step_batch16_greedy():
+    shape = I.LLAMA_8B
+    ks = I.draw_k(16, [3, 5, 8], 3)
+    ctx = I.draw_context_lengths(16, 512, 4096, 3)
+    _full_step(shape, 16, ks, ctx, 3, check=_pick(ks, ctx, 2), greedy=True)
+
+
+def test_llama8b_step_batch1():
+    shape = I.LLAMA_8B
+    _full_step(shape, 1, [5], [3000], 4, check={0})
 
 
 def test_llama8b_step_batch64_sampled():
-    # several token tiles per weight tile (the tensor-bound regime); one request checked
+    # several token tiles per weight tile (the tensor-bound regime)
     shape = I.LLAMA_8B
     ks = I.draw_k(64, [3, 5, 8], 1)
     ctx = I.draw_context_lengths(64, 512, 4096, 1)
-    smallest = int(np.argmin([c + 100 * k for c, k in zip(ctx, ks)]))
-    _full_step(shape, 64, ks, ctx, 1, check={smallest})
+    _full_step(shape, 64, ks, ctx, 1, check=_pick(ks, ctx))
+
+
+def test_llama8b_step_batch128_sampled():
+    shape = I.LLAMA_8B
+    ks = I.draw_k(128, [3, 5, 8], 2)
+    ctx = I.draw_context_lengths(128, 512, 4096, 2)
+    _full_step(shape, 128, ks, ctx, 2, check=_pick(ks, ctx, 2))
 
 
 def test_llama1b_step_batch16():
     shape = I.LLAMA_1B
     ks = I.draw_k(16, [2, 3, 4, 5, 6, 7, 8], 0)
     ctx = I.draw_context_lengths(16, 256, 2048, 0)
-    _full_step(shape, 16, ks, ctx, 0, check={0, 5, 11})
+    _full_step(shape, 16, ks, ctx, 0, check={0, 5, 11, int(np.argmax(ctx))})
 
 
 @pytest.mark.parametrize("tau,greedy", [(0.7, False), (1.0, False), (1.0, True)])
