@@ -80,6 +80,10 @@ typedef struct sled_config {
                              rounded to 16 bits by the device, half the bytes per request (Section 3.2 wants requests
                              small).  Eq. 1 is then applied with the rounded q: the output follows the target's
                              distribution up to the rounding of q (relative 2^-9 per entry), no longer exactly. */
+  int32_t attention_impl; /* 0: the library's choice (the warp-level tensor-core kernel).  1: the tcgen05 kernel where it
+                             applies (bf16 cache, 16-token pages, head_dim 128, requests of at most 48 query rows, i.e.
+                             (k + 1) * n_q_heads / n_kv_heads <= 48); other steps fall back to 0.  Same results within
+                             the attention tolerance; measured slower than 0 on the workloads here. */
 } sled_config;
 
 /* Target weights, row-major [out][in], all of type weight_dtype.  HOST or DEVICE

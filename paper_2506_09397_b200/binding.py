@@ -43,7 +43,7 @@ class SledConfig(C.Structure):
         ("page_size", C.c_int32), ("n_pages", C.c_int32), ("max_batch", C.c_int32), ("max_k", C.c_int32),
         ("max_step_tokens", C.c_int32), ("temperature", C.c_float), ("greedy", C.c_int32),
         ("probs_on_device", C.c_int32), ("device_index", C.c_int32), ("stream", C.c_void_p),
-        ("draft_probs_dtype", C.c_int32)]
+        ("draft_probs_dtype", C.c_int32), ("attention_impl", C.c_int32)]
 
 
 class SledWeights(C.Structure):
@@ -176,12 +176,13 @@ class Engine:
 
     def __init__(self, shape, weights: dict, *, n_pages: int, max_batch: int, max_k: int, max_step_tokens: int,
                  temperature: float = 1.0, greedy: bool = False, probs_on_device: bool = False, device_index: int = 0,
-                 page_size: int = 16, stream: int | None = None, draft_probs_dtype: str = "fp32"):
+                 page_size: int = 16, stream: int | None = None, draft_probs_dtype: str = "fp32",
+                 attention_impl: int = 0):
         self.shape = shape
         cfg = SledConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                          shape.ffn_dim, shape.vocab, shape.rms_eps, shape.rope_theta, _DT[shape.weight_dtype],
                          _DT[shape.kv_dtype], page_size, n_pages, max_batch, max_k, max_step_tokens, temperature,
-                         int(greedy), int(probs_on_device), device_index, stream, _DT[draft_probs_dtype])
+                         int(greedy), int(probs_on_device), device_index, stream, _DT[draft_probs_dtype], attention_impl)
         w = SledWeights()
         w.tok_emb, w.final_norm, w.lm_head = _addr(weights["tok_emb"]), _addr(weights["final_norm"]), _addr(weights["lm_head"])
         keep = []

@@ -65,12 +65,12 @@ struct AttnArgs {
   const CUtensorMap* map_v = nullptr;
   int32_t* error = nullptr;
   Stamp stamp, stamp_merge;   // of the attention kernel and of the merge kernel that may follow it
-  int use_tc = 0;             // 1: every item has at most 128 query rows and head_dim is 128: the tcgen05 kernel runs
+  int use_tc = 0;             // 1: every item has at most 48 query rows and head_dim is 128: the tcgen05 kernel runs
 };
 int launch_attention(const AttnArgs& a, cudaStream_t s);
 // warp-level tensor-core kernel alone (attention_mma.cu); returns 1 or a negative value
 int launch_attention_mma(const AttnArgs& a, cudaStream_t s);
-// tcgen05 kernel alone (attention_tc.cu): head_dim 128, at most 128 query rows per item; returns 1 or a negative value
+// tcgen05 kernel alone (attention_tc.cu): head_dim 128, at most 48 query rows per item; returns 1 or a negative value
 int launch_attention_tc(const AttnArgs& a, cudaStream_t s);
 
 // ---- fused vocabulary softmax + acceptance + corrective / bonus draw (accept.cu)

@@ -15,14 +15,16 @@ def _attn_shape(h, hq, hkv, kv="bf16"):
     return I.ModelShape("attn_only", 1, 64, hq, hkv, h, 64, 64, 5e5, "bf16" if kv == "bf16" else "fp32", kv)
 
 
-@pytest.mark.parametrize("h,hq,hkv,kv", [(128, 32, 8, "bf16"), (64, 32, 8, "bf16"), (64, 4, 4, "fp32")])
-def test_ragged_attention_matches_oracle(h, hq, hkv, kv):
+@pytest.mark.parametrize("h,hq,hkv,kv,impl", [(128, 32, 8, "bf16", 0), (128, 32, 8, "bf16", 1), (64, 32, 8, "bf16", 0),
+                                              (64, 4, 4, "fp32", 0)])
+def test_ragged_attention_matches_oracle(h, hq, hkv, kv, impl):
+    # impl 1: the tcgen05 kernel (head_dim 128, at most 48 query rows per request); 0: the warp-level kernels
     shape = _attn_shape(h, hq, hkv, kv)
     w = I.make_weights(shape, 0)
     lens = [128, 131, 700, 2048, 5000, 9, 16, 17, 1023, 3000]     # total cached tokens incl. the new ones
     qlens = [2, 9, 5, 3, 8, 9, 4, 1, 7, 6]
     n_pages = sum((n + 15) // 16 for n in lens) + 4
-    eng = B.Engine(shape, w, n_pages=n_pages, max_batch=16, max_k=8, max_step_tokens=128)
+    eng = B.Engine(shape, w, n_pages=n_pages, max_batch=16, max_k=8, max_step_tokens=128, attention_impl=impl)
     eng.shuffle_pages(1)
     Ks, Vs = {}, {}
     for i, n in enumerate(lens):

@@ -138,11 +138,13 @@ def test_batch_composition_does_not_change_a_request():
     eng.shutdown()
 
 
-def test_synthetic_cache_and_long_context_split():
+@pytest.mark.parametrize("attention_impl", [0, 1])
+def test_synthetic_cache_and_long_context_split(attention_impl):
     # cache content loaded directly; one context long enough that its keys are split over several blocks
+    # (attention_impl 1: the same step with the tcgen05 attention kernel)
     shape = I.SMALL_GQA
     w = I.make_weights(shape, seed=2)
-    eng = _engine(shape, w, n_pages=400)
+    eng = _engine(shape, w, n_pages=400, attention_impl=attention_impl)
     eng.shuffle_pages(5)
     orc = O.OracleModel(shape, oracle_weights(w))
     lens = {21: 1500, 22: 300, 23: 17}
