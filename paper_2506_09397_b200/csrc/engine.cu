@@ -92,7 +92,6 @@ struct sled_engine {
   float* q_stage = nullptr;
   bool attn_tc = false;          // head_dim 128, bf16 cache, 16-token pages: attention may run on tcgen05
   TcActivation tc_norm, tc_attn, tc_ffn;
-  unsigned int* fuse_counters = nullptr;   // one per normalisation that runs inside the linear layer consuming it; zero at step begin
   int32_t* tc_error = nullptr;  // device word set by a kernel whose bounded wait ran out: the first word of the
                                 // results block (d_results), so the step's one result copy brings it along
 
@@ -192,7 +191,7 @@ int linear_split(const sled_engine* e, int T, const Linear& L) {
 
 // out partial sums [split][T][N] into e->partial (or into `dst` when given, then split must be 1)
 int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Linear& L, int T, float* dst, int* split_out,
-               const TcEpilogue& epi = TcEpilogue(), const TcPrologue& pro = TcPrologue()) {
+               const TcEpilogue& epi = TcEpilogue()) {
   int split = dst ? 1 : linear_split(e, T, L);
   float* out = dst ? dst : e->partial;
   const int64_t stride = static_cast<int64_t>(T) * L.N;
@@ -204,7 +203,7 @@ int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Lin
     TcEpilogue ep = epi;
     ep.stamp_begin = st.begin;
     ep.stamp_end = st.end;
-    n = tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_error, ep, e->stream, pro);
+    n = tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_error, ep, e->stream);
   } else {
     n = launch_gemm_simt(A, e->adtype(), L.w, e->cfg.weight_dtype, T, L.N, L.K, split, out, stride, e->stream, st);
   }
@@ -435,39 +434,15 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
   e->count(n, K_OTHER);
   int split = 0;           // split count of the partial sums waiting to be added to x
   int64_t stride = 0;
-  // A normalisation runs inside the linear layer that consumes it when all blocks of that launch are resident at
-  // once (the step's tokens fit one token tile): one kernel boundary less.  The previous layer's K slices live in
-  // e->partial, which the fused layer itself overwrites - but only in its epilogue, after every block has passed the
-  // counter, i.e. after all slices have been added to x.
-  const bool tc = c.weight_dtype == SLED_BF16;
-  if (tc) cudaMemsetAsync(e->fuse_counters, 0, sizeof(unsigned int) * (2 * c.n_layers + 2), e->stream);
-  auto prologue = [&](const void* gain, int which) {
-    TcPrologue p;
-    p.x = e->x;
-    p.partial = split > 0 ? e->partial : nullptr;
-    p.n_split = split;
-    p.split_stride = stride;
-    p.gain = static_cast<const __nv_bfloat16*>(gain);
-    p.eps = c.rms_eps;
-    p.d = d;
-    p.act = static_cast<__nv_bfloat16*>(e->act_norm);
-    p.counter = e->fuse_counters + which;
-    return p;
-  };
   for (int l = 0; l < c.n_layers; ++l) {
     Layer& L = e->layers[l];
+    e->mark(K_OTHER);
+    n = launch_add_rmsnorm(e->x, e->partial, split, stride, L.attn_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm,
+                           ad, e->stream, e->stamp(K_OTHER));
+    if (n < 0) return SLED_ERR_DEVICE;
+    e->count(n, K_OTHER);
     int s_qkv;
-    int rc;
-    if (tc && tc_gemm_can_fuse_prologue(T, L.qkv.N, L.qkv.K, linear_split(e, T, L.qkv), e->n_sm)) {
-      rc = run_linear(e, e->act_norm, &e->tc_norm, L.qkv, T, nullptr, &s_qkv, TcEpilogue(), prologue(L.attn_norm, 2 * l));
-    } else {
-      e->mark(K_OTHER);
-      n = launch_add_rmsnorm(e->x, e->partial, split, stride, L.attn_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm,
-                             ad, e->stream, e->stamp(K_OTHER));
-      if (n < 0) return SLED_ERR_DEVICE;
-      e->count(n, K_OTHER);
-      rc = run_linear(e, e->act_norm, &e->tc_norm, L.qkv, T, nullptr, &s_qkv);
-    }
+    int rc = run_linear(e, e->act_norm, &e->tc_norm, L.qkv, T, nullptr, &s_qkv);
     if (rc) return rc;
     e->mark(K_OTHER);
     n = launch_rope_kv(e->partial, s_qkv, static_cast<int64_t>(T) * L.qkv.N, e->rope_cs, pk.tok_slot, T, c.n_q_heads,
@@ -482,14 +457,10 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
     rc = run_linear(e, e->attn_out, &e->tc_attn, L.o, T, nullptr, &split);
     if (rc) return rc;
     stride = static_cast<int64_t>(T) * L.o.N;
-    const bool fuse_ffn_norm = tc && tc_gemm_can_fuse_prologue(T, L.gate_up.N, L.gate_up.K, linear_split(e, T, L.gate_up), e->n_sm);
-    if (!fuse_ffn_norm) {
-      e->mark(K_OTHER);
-      n = launch_add_rmsnorm(e->x, e->partial, split, stride, L.ffn_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm, ad,
-                             e->stream, e->stamp(K_OTHER));
-      e->count(n, K_OTHER);
-    }
-    const TcPrologue ffn_pro = fuse_ffn_norm ? prologue(L.ffn_norm, 2 * l + 1) : TcPrologue();
+    e->mark(K_OTHER);
+    n = launch_add_rmsnorm(e->x, e->partial, split, stride, L.ffn_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm, ad,
+                           e->stream, e->stamp(K_OTHER));
+    e->count(n, K_OTHER);
     int s_gu;
     if (c.weight_dtype == SLED_BF16 && linear_split(e, T, L.gate_up) == 1) {
       // the whole sum is formed in one place: SwiGLU is applied there, act_ffn comes straight out of the GEMM
@@ -497,15 +468,8 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
       epi.mode = kEpiSwiglu;
       epi.act_out = static_cast<__nv_bfloat16*>(e->act_ffn);
       epi.act_ld = c.ffn_dim;
-      rc = run_linear(e, e->act_norm, &e->tc_norm, L.gate_up, T, nullptr, &s_gu, epi, ffn_pro);
+      rc = run_linear(e, e->act_norm, &e->tc_norm, L.gate_up, T, nullptr, &s_gu, epi);
       if (rc) return rc;
-    } else if (fuse_ffn_norm) {
-      rc = run_linear(e, e->act_norm, &e->tc_norm, L.gate_up, T, nullptr, &s_gu, TcEpilogue(), ffn_pro);
-      if (rc) return rc;
-      e->mark(K_OTHER);
-      n = launch_swiglu(e->partial, s_gu, static_cast<int64_t>(T) * L.gate_up.N, T, c.ffn_dim, e->act_ffn, ad, e->stream,
-                        e->stamp(K_OTHER));
-      e->count(n, K_OTHER);
     } else {
       rc = run_linear(e, e->act_norm, &e->tc_norm, L.gate_up, T, nullptr, &s_gu);
       if (rc) return rc;
@@ -808,7 +772,6 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   if ((cudaMemset(e->act_ffn, 0, padT * F * as)) != cudaSuccess) return fail(SLED_ERR_DEVICE);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->logits), maxT * c.vocab * 4))) return fail(rc);
   if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->rope_cs), maxT * (c.head_dim / 2) * sizeof(float2)))) return fail(rc);
-  if ((rc = dmalloc(e, reinterpret_cast<void**>(&e->fuse_counters), sizeof(unsigned int) * (2 * c.n_layers + 2)))) return fail(rc);
   {
     size_t need = 0;
     const Linear* shapes[4] = {&e->layers[0].qkv, &e->layers[0].o, &e->layers[0].gate_up, &e->layers[0].down};

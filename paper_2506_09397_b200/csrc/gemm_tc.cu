@@ -152,8 +152,7 @@ template <int TN_MAX, int STAGES>
 __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constant__ CUtensorMap map_w,
                                                        const __grid_constant__ CUtensorMap map_a, int T, int N,
                                                        int kb_total, int kb_per_split, float* __restrict__ out,
-                                                       long long split_stride, int32_t* error, TcEpilogue epi,
-                                                       TcPrologue pro) {
+                                                       long long split_stride, int32_t* error, TcEpilogue epi) {
   using L = SplitSmemLayout<TN_MAX, STAGES>;
   constexpr int kTmemCols = TN_MAX <= 32 ? 32 : TN_MAX <= 64 ? 64 : TN_MAX <= 128 ? 128 : 256;   // a power of two
   extern __shared__ __align__(1024) uint8_t smem_raw[];    // swizzled tiles need 1024-byte alignment
@@ -211,27 +210,9 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
         tma_load_2d(base + kb * L::kStageBytes, &map_w, 0, (m_tile * kb_total + kb0 + kb) * kBlockM, full, pol_first);
       }
       pdl_wait_here();
-      if (pro.x != nullptr) {
-        // the activations are being produced by this launch's own blocks: wait until all of them are through
-        const unsigned int n_blocks = gridDim.x * gridDim.y * gridDim.z;
-        const long long t_start = clock64();
-        for (;;) {
-          unsigned int seen;
-          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(pro.counter) : "memory");
-          if (seen >= n_blocks) break;
-          if (*abort_slot != 0 || clock64() - t_start > kWaitCycles) {
-            atomicCAS(error, 0, 10);
-            *abort_slot = 1;
-            ok = false;
-            break;
-          }
-          __nanosleep(64);
-        }
-        asm volatile("fence.proxy.async.global;" ::: "memory");   // generic-proxy writes of other blocks before this thread's TMA reads
-      }
-      for (int kb = 0; ok && kb < pre; ++kb)
+      for (int kb = 0; kb < pre; ++kb)
         tma_load_2d(base + kb * L::kStageBytes + kWStageBytes, &map_a, (kb0 + kb) * kBlockK, t0, bars + 8 * kb, pol_last);
-      for (int kb = pre; ok && kb < nkb; ++kb) {
+      for (int kb = pre; kb < nkb; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
         if (!mbar_wait(bars + 8 * (STAGES + s), ph ^ 1, error, 1, abort_slot)) { ok = false; break; }
@@ -263,47 +244,6 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
     }
   } else {
     const int quad = warp & 3;                      // a warp may only touch tensor-memory lanes 32*(warp%4)..+31
-    if (pro.x != nullptr) {
-      // ---- first phase: residual add + RMSNorm of this block's tokens (the four epilogue warps, 128 threads)
-      pdl_wait_here();                              // the previous linear layer's K slices are complete
-      const int tid = threadIdx.x - 64;
-      const unsigned int n_blocks = gridDim.x * gridDim.y * gridDim.z;
-      const unsigned int block_id = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
-      float* red = reinterpret_cast<float*>(base_ptr + L::kTiles + 128);   // 4 floats behind the barriers
-      for (int t = block_id; t < T; t += n_blocks) {
-        const long long row = static_cast<long long>(t) * pro.d;
-        float ss = 0.f;
-        for (int i = tid * 4; i < pro.d; i += 128 * 4) {
-          float4 v = *reinterpret_cast<const float4*>(pro.x + row + i);
-          for (int sp = 0; sp < pro.n_split; ++sp) {
-            const float4 p = __ldcg(reinterpret_cast<const float4*>(pro.partial + sp * pro.split_stride + row + i));
-            v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
-          }
-          if (pro.n_split > 0) *reinterpret_cast<float4*>(pro.x + row + i) = v;
-          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        asm volatile("bar.sync 1, 128;" ::: "memory");          // the scratch of the previous token has been read
-        if (lane == 0) red[quad] = ss;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        const float scale = rsqrtf((red[0] + red[1] + red[2] + red[3]) / static_cast<float>(pro.d) + pro.eps);
-        for (int i = tid * 4; i < pro.d; i += 128 * 4) {          // each thread re-reads what it wrote itself
-          const float4 v = *reinterpret_cast<const float4*>(pro.x + row + i);
-          const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * scale * __bfloat162float(pro.gain[i]),
-                                                          v.y * scale * __bfloat162float(pro.gain[i + 1]));
-          const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * scale * __bfloat162float(pro.gain[i + 2]),
-                                                          v.w * scale * __bfloat162float(pro.gain[i + 3]));
-          uint2 pk;
-          pk.x = *reinterpret_cast<const uint32_t*>(&lo);
-          pk.y = *reinterpret_cast<const uint32_t*>(&hi);
-          *reinterpret_cast<uint2*>(pro.act + row + i) = pk;
-        }
-      }
-      __threadfence();                                           // this block's activations before its count
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (tid == 0) atomicAdd(pro.counter, 1u);
-    }
     if (nkb > 0) ok = mbar_wait(bars + 8 * (2 * STAGES), 0, error, 3, abort_slot);
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     if (ok) {
@@ -744,7 +684,7 @@ int tc_gemm_split(int T, int N, int K, int n_sm) {
 
 template <int TN_MAX, int STAGES>
 static int launch_split(const CUtensorMap& mw, const CUtensorMap& ma, int T, int N, int K, int n_split, float* out,
-                        int64_t split_stride, int32_t* error, const TcEpilogue& epi, cudaStream_t s, const TcPrologue& pro) {
+                        int64_t split_stride, int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
   using L = SplitSmemLayout<TN_MAX, STAGES>;
   static bool configured = false;
   if (!configured) {
@@ -765,7 +705,7 @@ static int launch_split(const CUtensorMap& mw, const CUtensorMap& ma, int T, int
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   const long long stride = split_stride;
-  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_split_kernel<TN_MAX, STAGES>, mw, ma, T, N, kb_total, kb_per, out, stride, error, epi, pro);
+  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_split_kernel<TN_MAX, STAGES>, mw, ma, T, N, kb_total, kb_per, out, stride, error, epi);
   return err == cudaSuccess ? 1 : -1;
 }
 
@@ -806,33 +746,16 @@ static int launch_pair(const CUtensorMap& mw, const CUtensorMap& ma, int T, int 
   return err == cudaSuccess ? 1 : -1;
 }
 
-bool tc_gemm_can_fuse_prologue(int T, int N, int K, int n_split, int n_sm) {
-  // the single-CTA kernel with one token tile, every block resident at once (two per SM), a row of d = K floats
-  // that 128 threads walk in float4 steps
-  const int n_mtiles = (N + kBlockM - 1) / kBlockM;
-  return T > 0 && T <= kSingleTileMax && n_split >= 1 && n_mtiles * n_split <= 2 * n_sm && K % 4 == 0;
-}
-
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
-                   int32_t* error, const TcEpilogue& epi, cudaStream_t s, const TcPrologue& pro) {
+                   int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
   if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
   if (epi.mode != kEpiStore && n_split != 1) return -1;   // a fused epilogue needs the complete sum
-  if (pro.x != nullptr) {
-    static int n_sm_pro = 0;
-    if (n_sm_pro == 0) {
-      int dev = 0;
-      cudaDeviceProp prop;
-      if (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess) n_sm_pro = prop.multiProcessorCount;
-    }
-    if (!tc_gemm_can_fuse_prologue(T, w.N, w.K, n_split, n_sm_pro) || pro.d != w.K || !pro.counter || !pro.act || !pro.gain)
-      return -1;
-  }
   // token tile = the smallest box that holds the step; what the narrower activation stage saves goes into ring depth
-  if (T <= 32) return launch_split<32, 5>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, epi, s, pro);
-  if (T <= 64) return launch_split<64, 4>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s, pro);
-  if (T <= 96) return launch_split<96, 4>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, epi, s, pro);
-  if (T <= 128) return launch_split<128, 3>(w.map, a.map[3], T, w.N, w.K, n_split, out, split_stride, error, epi, s, pro);
-  if (T <= kSingleTileMax) return launch_split<160, 3>(w.map, a.map[4], T, w.N, w.K, n_split, out, split_stride, error, epi, s, pro);
+  if (T <= 32) return launch_split<32, 5>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (T <= 64) return launch_split<64, 4>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (T <= 96) return launch_split<96, 4>(w.map, a.map[2], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (T <= 128) return launch_split<128, 3>(w.map, a.map[3], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
+  if (T <= kSingleTileMax) return launch_split<160, 3>(w.map, a.map[4], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (pair_kernel_applies(T, w.N)) {
     static int n_sm = 0;
     if (n_sm == 0) {
@@ -843,7 +766,7 @@ int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split,
     if (n_sm >= 2)   // weight tiles pair up: persistent CTA pairs, half of the token tile staged by each CTA
       return launch_pair(w.map, a.map[3], T, w.N, w.K, n_split, out, split_stride, error, epi, n_sm, s);
   }
-  return launch_split<256, 2>(w.map, a.map[5], T, w.N, w.K, n_split, out, split_stride, error, epi, s, pro);
+  return launch_split<256, 2>(w.map, a.map[5], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
 }
 
 }  // namespace sled

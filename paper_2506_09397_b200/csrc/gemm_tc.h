@@ -32,27 +32,6 @@ struct TcEpilogue {       // what happens to the finished sums (see emit16 in ge
   unsigned long long* stamp_end = nullptr;
 };
 
-// Optional first phase of a linear layer: the residual add + RMSNorm that produces its input.  When `x` is set, the
-// blocks of the launch first compute, one token per block,
-//     x[t] += sum_s partial[s][t]   (the previous linear layer's K slices, in slice order)
-//     a[t]  = bf16( x[t] * rsqrt(mean(x[t]^2) + eps) * gain )
-// into the layer's activation buffer, meet at a counter in global memory, and only then load activations.  This
-// removes one kernel boundary per normalisation.  It requires every block of the launch to be resident at once
-// (checked by the launcher: at most two blocks per SM, single-CTA kernel only).
-struct TcPrologue {
-  float* x = nullptr;              // [T][d] fp32 residual stream, updated in place
-  const float* partial = nullptr;  // [n_split][T][d] or null
-  int n_split = 0;
-  long long split_stride = 0;
-  const __nv_bfloat16* gain = nullptr;   // [d]
-  float eps = 0.f;
-  int d = 0;
-  __nv_bfloat16* act = nullptr;    // [T][d] the layer's input (the buffer behind the TcActivation)
-  unsigned int* counter = nullptr; // zero before the launch; counts the blocks that are through with their tokens
-};
-// true if a launch of this shape can carry a prologue (all its blocks resident at once)
-bool tc_gemm_can_fuse_prologue(int T, int N, int K, int n_split, int n_sm);
-
 // 2D bf16 tensor map over a row-major [rows][cols] array: boxes of 64 columns x box_rows rows, 128-byte swizzle
 int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int cols, int box_rows);
 // Bytes of the tiled copy of an [N][K] matrix, and its construction from the row-major matrix (both in
@@ -67,7 +46,7 @@ int tc_gemm_split(int T, int N, int K, int n_sm);
 // out[slice][T][N] = A[T][K slice] . W[N][K slice]^T; returns kernels launched (1) or a negative value;
 // `error` is a device word set if a bounded wait ran out
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
-                   int32_t* error, const TcEpilogue& epi, cudaStream_t s, const TcPrologue& pro = TcPrologue());
+                   int32_t* error, const TcEpilogue& epi, cudaStream_t s);
 
 // Self-test: launches a kernel whose bounded wait (limit in clock cycles, at most the kernels' own limit) runs out
 // on a barrier nobody signals and records code 9 in *error.  Returns kernels launched (1) or a negative value.
