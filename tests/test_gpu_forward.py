@@ -314,6 +314,45 @@ def test_errors_leave_everything_unchanged():
     eng.shutdown()
 
 
+@pytest.mark.parametrize("T_want", [163, 190, 225, 262, 300, 389, 520, 1030])
+def test_wide_steps_on_cta_pairs(T_want):
+    # more than 160 tokens: every linear layer of this shape (even numbers of weight tiles) runs on the persistent
+    # CTA pairs; the step sizes give one to five token tiles with ragged last tiles of different widths, K-slice
+    # counts that change with the step size, and fewer units than pairs (most pairs leave without work)
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=12)
+    n_req = (T_want + 8) // 9
+    eng = _engine(shape, w, n_pages=4 * n_req + 8, max_batch=n_req, max_k=8, max_step_tokens=T_want + 8)
+    orc = O.OracleModel(shape, oracle_weights(w))
+    checked = {0, n_req // 2, n_req - 1}
+    n_kv = {}
+    for c in range(n_req):
+        p = I.make_prompt(shape.vocab, 3 + (7 * c) % 29, 12, c)
+        eng.prefill(c, p)
+        n_kv[c] = len(p) - 1                                               # the prompt's last token waits as "pending"
+        if c in checked:
+            orc.prefill(c, p)
+    ks = [8] * n_req
+    ks[-1] = T_want - 9 * (n_req - 1) - 1                                  # the last request fills the step to T_want exactly
+    assert 0 <= ks[-1] <= 8
+    reqs = [(c,) + tuple(I.make_drafts(shape.vocab, ks[c], 12, c)) for c in range(n_req)]
+    T = sum(len(d) + 1 for _, d, _ in reqs)
+    assert T == T_want
+    eng.set_commit(False)
+    got = eng.verify_batch([(c, d.numpy(), q.numpy()) for c, d, q in reqs], 4)
+    glog = eng.logits(T)
+    row = 0
+    for (c, d, q), g in zip(reqs, got):
+        k = len(d)
+        if c in checked:
+            st, n_acc, nxt, ol, mg = orc.verify(c, d.numpy(), q.numpy(), 4, commit=False)
+            assert np.max(np.abs(glog[row:row + k + 1] - ol)) <= 2e-2
+        st2, n2, x2, _ = O.accept(glog[row:row + k + 1], q.numpy(), d.numpy(), 1.0, False, 4, c, n_kv[c])
+        assert (n2, x2, 0) == g
+        row += k + 1
+    eng.shutdown()
+
+
 def test_step_between_128_and_160_tokens():
     # 129..160 tokens: the widest single token tile of the linear layers (160 columns, partly filled)
     shape = I.SMALL_GQA
