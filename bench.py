@@ -37,11 +37,11 @@ import torch
 from paper_2506_09397_b200 import inputs as I
 
 # DRAM traffic of the linear-layer kernel per launch (ncu: dram__bytes_read.sum + dram__bytes_write.sum, summed over
-# the 129 launches of a step; profiles/ncu_linear_and_attention_kernels_llama8b_2layer_b{16,64}.txt), keyed by
+# the 129 launches of a step; profiles/ncu_linear_layer_kernel_llama8b_2layer_b{16,64}.txt), keyed by
 # (shape, layers, batch).  Only valid for the kernel source it was taken from: reported as null when that file has
 # changed since.
-TRAFFIC_LINEAR = {"bytes_per_launch": {("llama8b", 32, 16): 119.4e6, ("llama8b", 32, 64): 127.7e6},
-                  "source_sha1": "34e4a651329b36d0406bc42b191d7a0961ff9274"}
+TRAFFIC_LINEAR = {"bytes_per_launch": {("llama8b", 32, 16): 119.5e6, ("llama8b", 32, 64): 127.0e6},
+                  "source_sha1": "fc5587e8a039e73b10e13f625c55ab2648de0908"}
 
 METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
@@ -75,6 +75,8 @@ def parse_args(argv=None):
     ap.add_argument("--drafts", default="correlated", choices=["correlated", "independent"],
                     help="correlated: draft distributions built from the target's own logits (rho = 0.8), "
                          "independent: softmax of N(0,1) logits")
+    ap.add_argument("--attention-impl", type=int, default=0, choices=[0, 1],
+                    help="0: warp-level tensor-core attention kernel (default), 1: the tcgen05 kernel (head_dim 128)")
     ap.add_argument("--sweep", default="1,64,128", help="other batch sizes measured after the headline one")
     ap.add_argument("--no-sweep", action="store_true")
     return ap.parse_args(argv)
@@ -311,7 +313,7 @@ class Point:
         n_pages = sum((c + k + 1 + 15) // 16 for c, k in zip(self.ctx, self.ks)) + 64
         self.eng = B.Engine(shape, w_dev, n_pages=n_pages, max_batch=batch, max_k=max(self.ks),
                             max_step_tokens=max(self.T, 16), temperature=1.0, greedy=args.greedy,
-                            device_index=local_rank, stream=stream.cuda_stream)
+                            device_index=local_rank, stream=stream.cuda_stream, attention_impl=args.attention_impl)
         self.eng.shuffle_pages(self.seed)
         for i in range(batch):
             K, V = I.make_kv(shape, self.ctx[i], self.seed, i, device=self.dev)
@@ -463,7 +465,7 @@ class Point:
         torch.cuda.empty_cache()
         self.eng = B.Engine(self.shape, w_dev, n_pages=n_pages, max_batch=self.Bn, max_k=max(self.ks),
                             max_step_tokens=max(self.T, 16), temperature=1.0, greedy=False, device_index=local_rank,
-                            stream=stream.cuda_stream, draft_probs_dtype="bf16")
+                            stream=stream.cuda_stream, draft_probs_dtype="bf16", attention_impl=args.attention_impl)
         self.eng.shuffle_pages(self.seed)
         for i in range(self.Bn):
             K, V = I.make_kv(self.shape, self.ctx[i], self.seed, i, device=self.dev)
@@ -544,6 +546,7 @@ def run_sled(args):
             "ms_per_step": ms_all / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if shape.weight_dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": pt.name, "tokens_scored_per_step": T,
+                       "attention_kernel": "tcgen05" if args.attention_impl == 1 else "warp-level mma",
                        "l2": "inputs larger than L2 (a step streams %.2f GB of weights)" % (2e-9 * shape.streamed_params()),
                        "draft_distributions": ("target-correlated: draft logits = 0.8 z + 0.6 std(z) noise, z the target's "
                                                "own logits at that position (untimed passes), q = softmax, d ~ q"
@@ -669,7 +672,7 @@ def run_attention_only(args):
     lens = I.draw_lognormal_kv_lengths(nreq, 2048, 1.0, 128, 16384, args.seed + 1)
     w = I.make_weights(shape, 0)
     eng = B.Engine(shape, w, n_pages=sum((n + 15) // 16 for n in lens) + 8, max_batch=nreq, max_k=8,
-                   max_step_tokens=sum(qlens))
+                   max_step_tokens=sum(qlens), attention_impl=args.attention_impl)
     eng.shuffle_pages(2)
     for i, n in enumerate(lens):
         K, V = I.make_kv(shape, n, 6, i, device="cuda")
