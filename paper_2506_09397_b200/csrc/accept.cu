@@ -56,6 +56,80 @@ __device__ __forceinline__ unsigned long long fixed_exp(float x) {
   return __float2ull_rz(scaled);
 }
 
+// Two fp32 lanes per instruction (add / mul / fma .f32x2): each lane is rounded to nearest exactly like the scalar
+// operation, so the packed form of fixed_exp below returns the same integers with about half the instructions.
+__device__ __forceinline__ unsigned long long pack2(float a, float b) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+
+// fixed_exp(z0 * inv_tau - m) and fixed_exp(z1 * inv_tau - m): the same operations in the same order, two lanes at
+// a time.  The integer part n of x * log2(e) is read off the low mantissa bits of t = x * log2(e) + 1.5 * 2^23
+// (t keeps the exponent of the shift constant, so its bit pattern minus the constant's is n).
+struct Exp2Consts {
+  unsigned long long inv_tau, neg_m, log2e, shift, neg_shift, ln2_hi, ln2_lo, c6, c5, c4, c3, half, one;
+};
+__device__ __forceinline__ Exp2Consts exp2_consts(float inv_tau, float m) {
+  Exp2Consts c;
+  c.inv_tau = pack2(inv_tau, inv_tau);
+  c.neg_m = pack2(-m, -m);
+  c.log2e = pack2(0x1.715476p+0f, 0x1.715476p+0f);
+  c.shift = pack2(12582912.0f, 12582912.0f);
+  c.neg_shift = pack2(-12582912.0f, -12582912.0f);
+  c.ln2_hi = pack2(-0x1.62e4p-1f, -0x1.62e4p-1f);
+  c.ln2_lo = pack2(-0x1.7f7d1cp-20f, -0x1.7f7d1cp-20f);
+  c.c6 = pack2(0x1.6c16c2p-10f, 0x1.6c16c2p-10f);
+  c.c5 = pack2(0x1.111112p-7f, 0x1.111112p-7f);
+  c.c4 = pack2(0x1.555556p-5f, 0x1.555556p-5f);
+  c.c3 = pack2(0x1.555556p-3f, 0x1.555556p-3f);
+  c.half = pack2(0.5f, 0.5f);
+  c.one = pack2(1.0f, 1.0f);
+  return c;
+}
+__device__ __forceinline__ void fixed_exp_pair(float z0, float z1, const Exp2Consts& c, unsigned long long& e0,
+                                               unsigned long long& e1) {
+  const unsigned long long x = add2(mul2(pack2(z0, z1), c.inv_tau), c.neg_m);   // a - m == a + (-m), rounded once
+  const unsigned long long t = fma2(x, c.log2e, c.shift);
+  const unsigned long long nf = add2(t, c.neg_shift);
+  unsigned long long r = fma2(nf, c.ln2_hi, x);
+  r = fma2(nf, c.ln2_lo, r);
+  unsigned long long p = fma2(c.c6, r, c.c5);
+  p = fma2(p, r, c.c4);
+  p = fma2(p, r, c.c3);
+  p = fma2(p, r, c.half);
+  p = fma2(p, r, c.one);
+  p = fma2(p, r, c.one);
+  float x0, x1, t0, t1, p0, p1;
+  unpack2(x, x0, x1);
+  unpack2(t, t0, t1);
+  unpack2(p, p0, p1);
+  // bits(t) - bits(1.5 * 2^23) = n; scaled = p * 2^(n + 40) by adding (n + 40) to p's exponent field
+  const uint32_t base = 0x4B400000u - 40u;
+  const float s0 = __uint_as_float(__float_as_uint(p0) + ((__float_as_uint(t0) - base) << 23));
+  const float s1 = __uint_as_float(__float_as_uint(p1) + ((__float_as_uint(t1) - base) << 23));
+  e0 = __float2ull_rz(x0 >= -30.0f ? s0 : 0.0f);
+  e1 = __float2ull_rz(x1 >= -30.0f ? s1 : 0.0f);
+}
+
 __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -137,7 +211,33 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     const bool vec = ((V & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
     // the draft rows are the caller's memory: any 4-byte aligned address is legal, 16-byte loads need more
     const bool q_vec = vec && ((reinterpret_cast<uintptr_t>(qbase) & (q16 ? 7 : 15)) == 0);   // four entries per load
-    if (vec) {   // four consecutive entries per thread and step (16-byte loads), four steps in flight
+    if (vec && !a.greedy) {
+      // sampling needs the maximum only, and rounding is monotone: max(z * inv_tau) = max(z) * inv_tau.  A NaN or an
+      // infinity anywhere turns the running sum of z * 0 into a NaN.
+      float mx = -INFINITY;
+      unsigned long long nan2 = pack2(0.f, 0.f);
+      const unsigned long long zero2 = pack2(0.f, 0.f);
+      auto look = [&](const float4& x4) {
+        mx = fmaxf(fmaxf(mx, fmaxf(x4.x, x4.y)), fmaxf(x4.z, x4.w));
+        nan2 = fma2(pack2(x4.x, x4.y), zero2, nan2);
+        nan2 = fma2(pack2(x4.z, x4.w), zero2, nan2);
+      };
+      constexpr int kStep = kThreads * 4;
+      int v = v_lo + threadIdx.x * 4;
+      for (; v + 3 * kStep < v_hi; v += 4 * kStep) {
+        const float4 x0 = *reinterpret_cast<const float4*>(z + v);
+        const float4 x1 = *reinterpret_cast<const float4*>(z + v + kStep);
+        const float4 x2 = *reinterpret_cast<const float4*>(z + v + 2 * kStep);
+        const float4 x3 = *reinterpret_cast<const float4*>(z + v + 3 * kStep);
+        look(x0); look(x1); look(x2); look(x3);
+      }
+      for (; v < v_hi; v += kStep) look(*reinterpret_cast<const float4*>(z + v));
+      float n0, n1;
+      unpack2(nan2, n0, n1);
+      bad = !(n0 == 0.f) || !(n1 == 0.f);
+      best = __fmul_rn(mx, a.inv_tau);   // -inf when this thread saw no entry
+      best_i = 0;                        // not used when sampling
+    } else if (vec) {   // four consecutive entries per thread and step (16-byte loads), four steps in flight
       auto look = [&](int v, const float4& x4) {
         const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
 #pragma unroll
@@ -212,10 +312,13 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     const float m = best;
     // ---- pass 2: Z = sum of the integer numerators
     unsigned long long zsum = 0;
+    const Exp2Consts ec = exp2_consts(a.inv_tau, m);
     if (vec) {
       auto add4 = [&](const float4& x4) {
-        zsum += fixed_exp(__fsub_rn(__fmul_rn(x4.x, a.inv_tau), m)) + fixed_exp(__fsub_rn(__fmul_rn(x4.y, a.inv_tau), m)) +
-                fixed_exp(__fsub_rn(__fmul_rn(x4.z, a.inv_tau), m)) + fixed_exp(__fsub_rn(__fmul_rn(x4.w, a.inv_tau), m));
+        unsigned long long e0, e1, e2, e3;
+        fixed_exp_pair(x4.x, x4.y, ec, e0, e1);
+        fixed_exp_pair(x4.z, x4.w, ec, e2, e3);
+        zsum += (e0 + e1) + (e2 + e3);
       };
       constexpr int kStep = kThreads * 4;
       int v = v_lo + threadIdx.x * 4;
@@ -296,10 +399,13 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
             qs[e] = (use_q && v0 + e < V) ? q_at(q_off + v0 + e) : 0.f;
           }
         }
+        unsigned long long Es[kVec];
+#pragma unroll
+        for (int e = 0; e < kVec; e += 2) fixed_exp_pair(zs[e], zs[e + 1], ec, Es[e], Es[e + 1]);
 #pragma unroll
         for (int e = 0; e < kVec; ++e) {
           if (v0 + e < V) {
-            unsigned long long E = fixed_exp(__fsub_rn(__fmul_rn(zs[e], a.inv_tau), m));
+            unsigned long long E = Es[e];
             if (use_q) {
               const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(qs[e]), Zd));
               E = E > Q ? E - Q : 0ull;
