@@ -75,6 +75,8 @@ def parse_args(argv=None):
     ap.add_argument("--drafts", default="correlated", choices=["correlated", "independent"],
                     help="correlated: draft distributions built from the target's own logits (rho = 0.8), "
                          "independent: softmax of N(0,1) logits")
+    ap.add_argument("--weight-bits", type=int, default=16, choices=[16, 8],
+                    help="8: the linear layers' weights as e4m3 bytes with one scale per output row (step workload)")
     ap.add_argument("--attention-impl", type=int, default=0, choices=[0, 1],
                     help="0: warp-level tensor-core attention kernel (default), 1: the tcgen05 kernel (head_dim 128)")
     ap.add_argument("--sweep", default="1,64,128", help="other batch sizes measured after the headline one")
@@ -196,10 +198,15 @@ def linear_shapes(shape):
     return per_layer * s.n_layers + [(s.vocab, s.d_model)]
 
 
+WEIGHT_BITS = 16   # --weight-bits 8: e4m3 bytes + one fp32 scale per output row
+
+
 def linear_bytes(shape, T: int) -> float:
-    """Bytes the linear layers must move in one step: every weight once (bf16), their bf16 inputs,
-    their fp32 outputs."""
+    """Bytes the linear layers must move in one step: every weight once (bf16, or a byte and the rows' scales),
+    their bf16 inputs, their fp32 outputs."""
     es = 2 if shape.weight_dtype == "bf16" else 4
+    if WEIGHT_BITS == 8:
+        return float(sum(n * k + n * 4 + T * k * es + T * n * 4 for n, k in linear_shapes(shape)))
     return float(sum(n * k * es + T * k * es + T * n * 4 for n, k in linear_shapes(shape)))
 
 
@@ -313,7 +320,8 @@ class Point:
         n_pages = sum((c + k + 1 + 15) // 16 for c, k in zip(self.ctx, self.ks)) + 64
         self.eng = B.Engine(shape, w_dev, n_pages=n_pages, max_batch=batch, max_k=max(self.ks),
                             max_step_tokens=max(self.T, 16), temperature=1.0, greedy=args.greedy,
-                            device_index=local_rank, stream=stream.cuda_stream, attention_impl=args.attention_impl)
+                            device_index=local_rank, stream=stream.cuda_stream, attention_impl=args.attention_impl,
+                            linear_weight_bits=args.weight_bits)
         self.eng.shuffle_pages(self.seed)
         for i in range(batch):
             K, V = I.make_kv(shape, self.ctx[i], self.seed, i, device=self.dev)
@@ -465,7 +473,8 @@ class Point:
         torch.cuda.empty_cache()
         self.eng = B.Engine(self.shape, w_dev, n_pages=n_pages, max_batch=self.Bn, max_k=max(self.ks),
                             max_step_tokens=max(self.T, 16), temperature=1.0, greedy=False, device_index=local_rank,
-                            stream=stream.cuda_stream, draft_probs_dtype="bf16", attention_impl=args.attention_impl)
+                            stream=stream.cuda_stream, draft_probs_dtype="bf16", attention_impl=args.attention_impl,
+                            linear_weight_bits=args.weight_bits)
         self.eng.shuffle_pages(self.seed)
         for i in range(self.Bn):
             K, V = I.make_kv(self.shape, self.ctx[i], self.seed, i, device=self.dev)
@@ -498,6 +507,12 @@ def run_sled(args):
     dev = f"cuda:{local_rank}"
     peaks, peak_src = load_peaks()
     w = I.make_weights(shape, seed, device=dev)
+    if args.weight_bits == 8:
+        global WEIGHT_BITS
+        WEIGHT_BITS = 8
+        args.no_cpu_baseline = True          # the oracle arm is timed on the 16-bit workload
+        w, _ = I.quantize_linear_weights(w, dequantised=False)
+        torch.cuda.empty_cache()
     need_host_w = (rank == 0 and world == 1 and not args.no_cpu_baseline)
     w_host = I.weights_to(w, "cpu") if need_host_w else None
     stream = torch.cuda.Stream(device=dev)
@@ -544,10 +559,12 @@ def run_sled(args):
     step_s = ms_all / args.steps / 1e3
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_all / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if shape.weight_dtype == "bf16" else "f32", "data": "synthetic",
+            "dtype": ("bf16 (e4m3 weights)" if args.weight_bits == 8 else "bf16") if shape.weight_dtype == "bf16" else "f32",
+            "data": "synthetic",
             "config": {"workload": pt.name, "tokens_scored_per_step": T,
                        "attention_kernel": "tcgen05" if args.attention_impl == 1 else "warp-level mma",
-                       "l2": "inputs larger than L2 (a step streams %.2f GB of weights)" % (2e-9 * shape.streamed_params()),
+                       "linear_weight_bits": args.weight_bits,
+                       "l2": "inputs larger than L2 (a step streams %.2f GB of weights)" % ((1e-9 if args.weight_bits == 8 else 2e-9) * shape.streamed_params()),
                        "draft_distributions": ("target-correlated: draft logits = 0.8 z + 0.6 std(z) noise, z the target's "
                                                "own logits at that position (untimed passes), q = softmax, d ~ q"
                                                if correlated else "independent of the target (softmax of N(0,1) logits)"),

@@ -84,6 +84,12 @@ typedef struct sled_config {
                              applies (bf16 cache, 16-token pages, head_dim 128, requests of at most 48 query rows, i.e.
                              (k + 1) * n_q_heads / n_kv_heads <= 48); other steps fall back to 0.  Same results within
                              the attention tolerance; measured slower than 0 on the workloads here. */
+  int32_t linear_weight_bits; /* 0 or 16: the linear layers' matrices are of weight_dtype.  8 (needs weight_dtype =
+                             SLED_BF16): wq, wk, wv, wo, w_gate, w_up, w_down and lm_head are e4m3 bytes (1 sign, 4
+                             exponent bits with bias 7, 3 mantissa bits, subnormals, no infinities; the patterns 0x7f and
+                             0xff must not occur) and every output row has an fp32 scale: W[n][k] = scale[n] *
+                             e4m3(byte[n][k]).  Half the weight bytes per step (the paper sweeps 16-, 8- and 4-bit
+                             precision, Section 4); activations, embedding and norms stay bf16, sums fp32. */
 } sled_config;
 
 /* Target weights, row-major [out][in], all of type weight_dtype.  HOST or DEVICE
@@ -102,6 +108,15 @@ typedef struct sled_weights {
   const void* const* w_gate;      /* [ffn_dim][d_model] */
   const void* const* w_up;        /* [ffn_dim][d_model] */
   const void* const* w_down;      /* [d_model][ffn_dim] */
+  /* linear_weight_bits = 8 only (ignored otherwise): fp32 scales, one per output row of the matrix of the same name */
+  const float* lm_head_scale;         /* [vocab] */
+  const float* const* wq_scale;       /* [n_q_heads*head_dim] */
+  const float* const* wk_scale;       /* [n_kv_heads*head_dim] */
+  const float* const* wv_scale;       /* [n_kv_heads*head_dim] */
+  const float* const* wo_scale;       /* [d_model] */
+  const float* const* w_gate_scale;   /* [ffn_dim] */
+  const float* const* w_up_scale;     /* [ffn_dim] */
+  const float* const* w_down_scale;   /* [d_model] */
 } sled_weights;
 
 /* One device's verification request (Section 3.2: the draft tokens it sends;

@@ -43,13 +43,15 @@ class SledConfig(C.Structure):
         ("page_size", C.c_int32), ("n_pages", C.c_int32), ("max_batch", C.c_int32), ("max_k", C.c_int32),
         ("max_step_tokens", C.c_int32), ("temperature", C.c_float), ("greedy", C.c_int32),
         ("probs_on_device", C.c_int32), ("device_index", C.c_int32), ("stream", C.c_void_p),
-        ("draft_probs_dtype", C.c_int32), ("attention_impl", C.c_int32)]
+        ("draft_probs_dtype", C.c_int32), ("attention_impl", C.c_int32), ("linear_weight_bits", C.c_int32)]
 
 
 class SledWeights(C.Structure):
     _fields_ = [("tok_emb", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p)] + [
         (n, C.POINTER(C.c_void_p)) for n in
-        ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")]
+        ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")] + [
+        ("lm_head_scale", C.c_void_p)] + [
+        (n + "_scale", C.POINTER(C.c_void_p)) for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")]
 
 
 class SledRequest(C.Structure):
@@ -177,12 +179,15 @@ class Engine:
     def __init__(self, shape, weights: dict, *, n_pages: int, max_batch: int, max_k: int, max_step_tokens: int,
                  temperature: float = 1.0, greedy: bool = False, probs_on_device: bool = False, device_index: int = 0,
                  page_size: int = 16, stream: int | None = None, draft_probs_dtype: str = "fp32",
-                 attention_impl: int = 0):
+                 attention_impl: int = 0, linear_weight_bits: int = 16):
+        """linear_weight_bits = 8: weights["wq"] .. ["w_down"] and ["lm_head"] are uint8 tensors of e4m3 bytes and
+        weights["wq_scale"] .. / ["lm_head_scale"] fp32 tensors with one scale per output row."""
         self.shape = shape
         cfg = SledConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                          shape.ffn_dim, shape.vocab, shape.rms_eps, shape.rope_theta, _DT[shape.weight_dtype],
                          _DT[shape.kv_dtype], page_size, n_pages, max_batch, max_k, max_step_tokens, temperature,
-                         int(greedy), int(probs_on_device), device_index, stream, _DT[draft_probs_dtype], attention_impl)
+                         int(greedy), int(probs_on_device), device_index, stream, _DT[draft_probs_dtype], attention_impl,
+                         linear_weight_bits)
         w = SledWeights()
         w.tok_emb, w.final_norm, w.lm_head = _addr(weights["tok_emb"]), _addr(weights["final_norm"]), _addr(weights["lm_head"])
         keep = []
@@ -190,6 +195,12 @@ class Engine:
             arr = (C.c_void_p * shape.n_layers)(*[_addr(t) for t in weights[name]])
             keep.append(arr)
             setattr(w, name, C.cast(arr, C.POINTER(C.c_void_p)))
+        if linear_weight_bits == 8:
+            w.lm_head_scale = _addr(weights["lm_head_scale"])
+            for name in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down"):
+                arr = (C.c_void_p * shape.n_layers)(*[_addr(t) for t in weights[name + "_scale"]])
+                keep.append(arr)
+                setattr(w, name + "_scale", C.cast(arr, C.POINTER(C.c_void_p)))
         h = C.c_void_p()
         _settle(weights["tok_emb"])
         _check(lib().sled_init(C.byref(w), C.byref(cfg), C.byref(h)), "sled_init")

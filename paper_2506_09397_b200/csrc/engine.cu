@@ -34,8 +34,9 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Linear {      // one weight matrix [N][K] in device memory
   void* w = nullptr;
+  float* scale = nullptr;   // 8-bit weights: one scale per output row
   int N = 0, K = 0;
-  TcWeight tc;       // tensor-core operand description (bf16 weights only)
+  TcWeight tc;       // tensor-core operand description (bf16 and 8-bit weights)
 };
 
 struct Layer {
@@ -185,6 +186,7 @@ int simt_split(int T, int N, int K, int n_sm) {
 }
 
 int linear_split(const sled_engine* e, int T, const Linear& L) {
+  if (L.tc.w8) return tc_gemm_split_w8(T, L.N, L.K, e->n_sm);
   if (e->cfg.weight_dtype == SLED_BF16) return tc_gemm_split(T, L.N, L.K, e->n_sm);
   return simt_split(T, L.N, L.K, e->n_sm);
 }
@@ -605,9 +607,21 @@ int upload(sled_engine* e, const void* src, size_t bytes, void** dst) {
 }
 
 // bf16 weights: replaces the row-major matrix `rowmajor` (a plain cudaMalloc that this call frees) by its tiled copy
-int finish_linear(sled_engine* e, Linear* L, void* rowmajor, int N, int K) {
+bool w8(const sled_engine* e) { return e->cfg.linear_weight_bits == 8; }
+size_t weight_elem_size(const sled_engine* e) { return w8(e) ? 1 : dtype_size(e->cfg.weight_dtype); }
+
+// takes over `rowmajor` (device, cudaMalloc'ed) and, for 8-bit weights, `scale` (device, [N], kept)
+int finish_linear(sled_engine* e, Linear* L, void* rowmajor, float* scale, int N, int K) {
   L->N = N;
   L->K = K;
+  if (w8(e)) {
+    L->scale = scale;
+    e->allocs.push_back(scale);
+    int rc = dmalloc(e, &L->w, tc_weight_w8_tiled_bytes(N, K));
+    if (!rc && tc_weight_init_w8(&L->tc, rowmajor, L->w, scale, N, K) != 0) rc = SLED_ERR_ARG;
+    cudaFree(rowmajor);
+    return rc;
+  }
   if (e->cfg.weight_dtype != SLED_BF16) {
     L->w = rowmajor;
     e->allocs.push_back(rowmajor);
@@ -619,41 +633,59 @@ int finish_linear(sled_engine* e, Linear* L, void* rowmajor, int N, int K) {
   return rc;
 }
 
-int make_linear(sled_engine* e, Linear* L, std::initializer_list<std::pair<const void*, int>> parts, int K) {
-  // concatenates the row blocks of `parts` into one [N][K] matrix
-  const size_t es = dtype_size(e->cfg.weight_dtype);
+struct Part { const void* w; const float* scale; int rows; };
+
+int make_linear(sled_engine* e, Linear* L, std::initializer_list<Part> parts, int K) {
+  // concatenates the row blocks of `parts` (and, for 8-bit weights, their scales) into one [N][K] matrix
+  const size_t es = weight_elem_size(e);
   int N = 0;
   for (auto& p : parts) {
-    if (!p.first) return SLED_ERR_ARG;
-    N += p.second;
+    if (!p.w || (w8(e) && !p.scale)) return SLED_ERR_ARG;
+    N += p.rows;
   }
   void* tmp = nullptr;
+  float* scale = nullptr;
   CU_TRY(cudaMalloc(&tmp, static_cast<size_t>(N) * K * es));
-  size_t off = 0;
+  if (w8(e) && cudaMalloc(reinterpret_cast<void**>(&scale), sizeof(float) * N) != cudaSuccess) {
+    cudaFree(tmp);
+    return SLED_ERR_DEVICE;
+  }
+  size_t off = 0, row = 0;
   for (auto& p : parts) {
-    const size_t bytes = static_cast<size_t>(p.second) * K * es;
-    if (cudaMemcpy(static_cast<char*>(tmp) + off, p.first, bytes, cudaMemcpyDefault) != cudaSuccess) {
+    const size_t bytes = static_cast<size_t>(p.rows) * K * es;
+    if (cudaMemcpy(static_cast<char*>(tmp) + off, p.w, bytes, cudaMemcpyDefault) != cudaSuccess ||
+        (scale && cudaMemcpy(scale + row, p.scale, sizeof(float) * p.rows, cudaMemcpyDefault) != cudaSuccess)) {
       cudaFree(tmp);
+      if (scale) cudaFree(scale);
       return SLED_ERR_DEVICE;
     }
     off += bytes;
+    row += p.rows;
   }
-  return finish_linear(e, L, tmp, N, K);
+  return finish_linear(e, L, tmp, scale, N, K);
 }
 
 // gate and up projections as one matrix with their rows interleaved (row 2f = gate f, row 2f+1 = up f),
 // so that a pair sits in neighbouring rows of an output tile and SwiGLU can be applied where the sums end up
-int make_gate_up(sled_engine* e, Linear* L, const void* gate, const void* up, int F, int K) {
-  if (!gate || !up) return SLED_ERR_ARG;
-  const size_t row = static_cast<size_t>(K) * dtype_size(e->cfg.weight_dtype);
+int make_gate_up(sled_engine* e, Linear* L, const Part& gate, const Part& up, int F, int K) {
+  if (!gate.w || !up.w || (w8(e) && (!gate.scale || !up.scale))) return SLED_ERR_ARG;
+  const size_t row = static_cast<size_t>(K) * weight_elem_size(e);
   void* tmp = nullptr;
+  float* scale = nullptr;
   CU_TRY(cudaMalloc(&tmp, 2 * static_cast<size_t>(F) * row));
-  if (cudaMemcpy2D(tmp, 2 * row, gate, row, row, F, cudaMemcpyDefault) != cudaSuccess ||
-      cudaMemcpy2D(static_cast<char*>(tmp) + row, 2 * row, up, row, row, F, cudaMemcpyDefault) != cudaSuccess) {
+  bool bad = cudaMemcpy2D(tmp, 2 * row, gate.w, row, row, F, cudaMemcpyDefault) != cudaSuccess ||
+             cudaMemcpy2D(static_cast<char*>(tmp) + row, 2 * row, up.w, row, row, F, cudaMemcpyDefault) != cudaSuccess;
+  if (!bad && w8(e)) {
+    bad = cudaMalloc(reinterpret_cast<void**>(&scale), sizeof(float) * 2 * F) != cudaSuccess ||
+          cudaMemcpy2D(scale, 2 * sizeof(float), gate.scale, sizeof(float), sizeof(float), F, cudaMemcpyDefault) != cudaSuccess ||
+          cudaMemcpy2D(scale + 1, 2 * sizeof(float), up.scale, sizeof(float), sizeof(float), F, cudaMemcpyDefault) != cudaSuccess;
+  }
+  if (bad) {
     cudaFree(tmp);
+    if (scale) cudaFree(scale);
     return SLED_ERR_DEVICE;
   }
-  return finish_linear(e, L, tmp, 2 * F, K);
+  return finish_linear(e, L, tmp, scale, 2 * F, K);
 }
 
 int check_cfg(const sled_config& c) {
@@ -668,6 +700,8 @@ int check_cfg(const sled_config& c) {
   if (c.weight_dtype == SLED_BF16 && c.kv_dtype != SLED_BF16) return SLED_ERR_ARG;
   if (c.draft_probs_dtype != SLED_F32 && c.draft_probs_dtype != SLED_BF16) return SLED_ERR_ARG;
   if (c.attention_impl != 0 && c.attention_impl != 1) return SLED_ERR_ARG;
+  if (c.linear_weight_bits != 0 && c.linear_weight_bits != 16 && c.linear_weight_bits != 8) return SLED_ERR_ARG;
+  if (c.linear_weight_bits == 8 && c.weight_dtype != SLED_BF16) return SLED_ERR_ARG;
   if (c.page_size <= 0 || c.n_pages <= 0 || c.max_batch <= 0 || c.max_k < 0 || c.max_step_tokens <= 0)
     return SLED_ERR_ARG;
   if (c.max_step_tokens < c.max_k + 1) return SLED_ERR_ARG;
@@ -737,7 +771,12 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kd = c.n_kv_heads * c.head_dim, F = c.ffn_dim;
   if ((rc = upload(e, w->tok_emb, static_cast<size_t>(c.vocab) * d * es, &e->tok_emb))) return fail(rc);
   if ((rc = upload(e, w->final_norm, d * es, &e->final_norm))) return fail(rc);
-  if ((rc = make_linear(e, &e->lm_head, {{w->lm_head, c.vocab}}, d))) return fail(rc);
+  const bool q8 = c.linear_weight_bits == 8;
+  if (q8 && (!w->wq_scale || !w->wk_scale || !w->wv_scale || !w->wo_scale || !w->w_gate_scale || !w->w_up_scale ||
+             !w->w_down_scale))
+    return fail(SLED_ERR_ARG);
+  auto sc = [&](const float* const* arr, int l) { return q8 ? arr[l] : nullptr; };
+  if ((rc = make_linear(e, &e->lm_head, {{w->lm_head, q8 ? w->lm_head_scale : nullptr, c.vocab}}, d))) return fail(rc);
   if (!w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo || !w->ffn_norm || !w->w_gate || !w->w_up || !w->w_down)
     return fail(SLED_ERR_ARG);
   e->layers.resize(c.n_layers);
@@ -745,10 +784,13 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
     Layer& L = e->layers[l];
     if ((rc = upload(e, w->attn_norm[l], d * es, &L.attn_norm))) return fail(rc);
     if ((rc = upload(e, w->ffn_norm[l], d * es, &L.ffn_norm))) return fail(rc);
-    if ((rc = make_linear(e, &L.qkv, {{w->wq[l], qd}, {w->wk[l], kd}, {w->wv[l], kd}}, d))) return fail(rc);
-    if ((rc = make_linear(e, &L.o, {{w->wo[l], d}}, qd))) return fail(rc);
-    if ((rc = make_gate_up(e, &L.gate_up, w->w_gate[l], w->w_up[l], F, d))) return fail(rc);
-    if ((rc = make_linear(e, &L.down, {{w->w_down[l], d}}, F))) return fail(rc);
+    if ((rc = make_linear(e, &L.qkv, {{w->wq[l], sc(w->wq_scale, l), qd}, {w->wk[l], sc(w->wk_scale, l), kd},
+                                      {w->wv[l], sc(w->wv_scale, l), kd}}, d)))
+      return fail(rc);
+    if ((rc = make_linear(e, &L.o, {{w->wo[l], sc(w->wo_scale, l), d}}, qd))) return fail(rc);
+    if ((rc = make_gate_up(e, &L.gate_up, {w->w_gate[l], sc(w->w_gate_scale, l), F}, {w->w_up[l], sc(w->w_up_scale, l), F}, F, d)))
+      return fail(rc);
+    if ((rc = make_linear(e, &L.down, {{w->w_down[l], sc(w->w_down_scale, l), d}}, F))) return fail(rc);
   }
 
   // KV pool: per layer [page][Hkv][page_size][h]

@@ -288,6 +288,260 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
 }
 
 // ------------------------------------------------------------------------------------------------
+// Linear layer with 8-bit weights (e4m3 bytes, one fp32 scale per output row; activations stay bf16).
+//
+// The weight bytes are what a narrow step streams, so they cross DRAM and L2 as bytes: a tile (128 rows x 64 k) is
+// 8 KB, stored as four groups [128 rows][16 bytes] (group c = bytes 16c .. 16c+15 of every row) and fetched with one
+// bulk copy into a deep ring (10-14 stages, 80-112 KB in flight per SM).  Warps 2-5 - idle until the epilogue in the
+// bf16 kernel - turn raw stages into the 128-byte-swizzled bf16 tiles the MMA reads: a lane takes the 16 bytes of a
+// row's group (consecutive lanes read consecutive 16-byte pieces: no bank conflicts), widens every byte
+// s.eeee.mmm to the bf16 pattern s.0000eeee.mmm0000 - the same number times 2^-120, subnormals included - and
+// multiplies by 2^120 (an exact bf16 x bf16 product), then stores two 16-byte chunks at their swizzled places.
+// The MMAs run exactly as in the bf16 kernel; the row's scale multiplies the fp32 sums in the epilogue.
+// One CTA per SM (224 KB of shared memory): rings of 10-14 raw stages, 4 bf16 weight stages, 4 activation stages.
+//   warp 0    : bulk copies of raw weight tiles (before the wait on the previous kernel) and TMA loads of activations
+//   warp 1    : tensor memory, MMAs; commits a slab to the "bf16 stage free" and "activation stage free" barriers
+//   warps 2-17: conversion; warps 2-5 then run the epilogue
+// All waits are bounded as above.
+constexpr int kW8StageBytes = kBlockM * kBlockK;   // 8 KB
+constexpr int kW8MmaStages = 4;
+constexpr int kW8ConvWarps = 16;                   // warps 2..17 convert: four per bf16 stage, 32 rows each
+constexpr int kW8Threads = 64 + 32 * kW8ConvWarps;
+static_assert(kW8ConvWarps == 4 * kW8MmaStages, "four conversion warps per bf16 weight stage");
+template <int TN_MAX>
+struct W8SmemLayout {
+  // every ring has to cover its own latency at the pace DRAM delivers a slab (about 350 cycles): raw tiles come
+  // from DRAM, activation tiles from L2, and a bf16 stage is busy from the start of its conversion to the end of its MMAs
+  static constexpr int kActStages = TN_MAX <= 96 ? 8 : TN_MAX <= 128 ? 6 : 4;
+  static constexpr int kRawStages = TN_MAX <= 32 ? 16 : TN_MAX <= 64 ? 12 : TN_MAX <= 128 ? 8 : 10;
+  static constexpr int kAStageBytes = TN_MAX * kBlockK * 2;
+  static constexpr int kWOff = 0;                                          // bf16 weight stages (1024-byte aligned)
+  static constexpr int kAOff = kW8MmaStages * kWStageBytes;                // activation stages (multiples of 1 KB)
+  static constexpr int kRawOff = kAOff + kActStages * kAStageBytes;         // raw weight stages
+  static constexpr int kTiles = kRawOff + kRawStages * kW8StageBytes;
+  static constexpr int kBars = 2 * kRawStages + 2 * kW8MmaStages + 2 * kActStages + 1;
+  static constexpr int kTotal = kTiles + 8 * kBars + 16;
+};
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// four e4m3 bytes -> four bf16 (two packed pairs), exact
+__device__ __forceinline__ void e4m3x4_to_bf16(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  const uint32_t y0 = __byte_perm(w, 0u, 0x1404);   // bytes 0 and 1 into the high byte of each 16-bit half
+  const uint32_t y1 = __byte_perm(w, 0u, 0x3424);   // bytes 2 and 3
+  const uint32_t v0 = (y0 & 0x80008000u) | ((y0 >> 4) & 0x07f007f0u);
+  const uint32_t v1 = (y1 & 0x80008000u) | ((y1 >> 4) & 0x07f007f0u);
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(lo) : "r"(v0), "r"(0x7B807B80u));   // x 2^120
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(hi) : "r"(v1), "r"(0x7B807B80u));
+}
+
+template <int TN_MAX>
+__global__ void __launch_bounds__(kW8Threads) tc_gemm_w8_kernel(const uint8_t* __restrict__ w8, const float* __restrict__ scale,
+                                                         const __grid_constant__ CUtensorMap map_a, int T, int N,
+                                                         int kb_total, int kb_per_split, float* __restrict__ out,
+                                                         long long split_stride, int32_t* error, TcEpilogue epi) {
+  using L = W8SmemLayout<TN_MAX>;
+  constexpr int R = L::kRawStages, SW = kW8MmaStages, SA = L::kActStages;
+  static_assert(L::kTotal <= 227 * 1024, "one CTA's shared memory");
+  constexpr int kTmemCols = TN_MAX <= 32 ? 32 : TN_MAX <= 64 ? 64 : TN_MAX <= 128 ? 128 : 256;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t base = smem_u32(smem_raw);
+  uint8_t* base_ptr = smem_raw;
+  const uint32_t bars = base + L::kTiles;
+  const uint32_t bar_raw_full = bars, bar_raw_empty = bars + 8 * R, bar_w_full = bars + 16 * R,
+                 bar_w_empty = bar_w_full + 8 * SW, bar_a_full = bar_w_empty + 8 * SW, bar_a_empty = bar_a_full + 8 * SA,
+                 bar_acc = bar_a_empty + 8 * SA;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kTiles + 8 * L::kBars);
+  volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * L::kBars + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  stamp_time(epi.stamp_begin, false);
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int t_tile = blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
+  const int kb0 = split * kb_per_split;
+  const int nkb = min(kb_per_split, kb_total - kb0);
+  const int t0 = t_tile * TN_MAX;
+  const int tn = min(TN_MAX, ((T - t0) + 15) & ~15);
+
+  if (threadIdx.x == 0) {
+    if (base & 1023u) atomicCAS(error, 0, 5);
+    *abort_slot = (base & 1023u) ? 1 : 0;
+  }
+  if (warp == 0 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    for (int i = 0; i < R; ++i) { mbar_init(bar_raw_full + 8 * i, 1); mbar_init(bar_raw_empty + 8 * i, 4); }
+    for (int i = 0; i < SW; ++i) { mbar_init(bar_w_full + 8 * i, 4); mbar_init(bar_w_empty + 8 * i, 1); }
+    for (int i = 0; i < SA; ++i) { mbar_init(bar_a_full + 8 * i, 1); mbar_init(bar_a_empty + 8 * i, 1); }
+    mbar_init(bar_acc, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))),
+                 "r"(static_cast<uint32_t>(kTmemCols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  bool ok = true;
+  if (threadIdx.x == 32 && *reinterpret_cast<volatile int32_t*>(error) != 0) *abort_slot = 1;
+
+  if (warp == 0) {
+    if (lane == 0 && *abort_slot == 0) {
+      uint64_t pol_first, pol_last;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_last));
+      const uint8_t* w_mine = w8 + (static_cast<long long>(m_tile) * kb_total + kb0) * kW8StageBytes;
+      const int pre_raw = min(R, nkb);
+      for (int kb = 0; kb < pre_raw; ++kb) {   // weights do not depend on the previous kernel
+        mbar_expect_tx(bar_raw_full + 8 * kb, kW8StageBytes);
+        bulk_load(base + L::kRawOff + kb * kW8StageBytes, w_mine + static_cast<long long>(kb) * kW8StageBytes, kW8StageBytes,
+                  bar_raw_full + 8 * kb, pol_first);
+      }
+      pdl_wait_here();
+      const int pre_a = min(SA, nkb);
+      for (int kb = 0; kb < pre_a; ++kb) {
+        mbar_expect_tx(bar_a_full + 8 * kb, L::kAStageBytes);
+        tma_load_2d(base + L::kAOff + kb * L::kAStageBytes, &map_a, (kb0 + kb) * kBlockK, t0, bar_a_full + 8 * kb, pol_last);
+      }
+      for (int kb = 0; ok && kb < nkb; ++kb) {
+        const int kr = kb + R;     // the raw stage of slab kb is free once it has been converted
+        if (kr < nkb) {
+          const int rs = kr % R;
+          if (!mbar_wait(bar_raw_empty + 8 * rs, ((kr / R) & 1) ^ 1, error, 1, abort_slot)) { ok = false; break; }
+          mbar_expect_tx(bar_raw_full + 8 * rs, kW8StageBytes);
+          bulk_load(base + L::kRawOff + rs * kW8StageBytes, w_mine + static_cast<long long>(kr) * kW8StageBytes, kW8StageBytes,
+                    bar_raw_full + 8 * rs, pol_first);
+        }
+        const int ka = kb + SA;    // the activation stage of slab kb is free once its MMAs have run
+        if (ka < nkb) {
+          const int as = ka % SA;
+          if (!mbar_wait(bar_a_empty + 8 * as, ((ka / SA) & 1) ^ 1, error, 6, abort_slot)) { ok = false; break; }
+          mbar_expect_tx(bar_a_full + 8 * as, L::kAStageBytes);
+          tma_load_2d(base + L::kAOff + as * L::kAStageBytes, &map_a, (kb0 + ka) * kBlockK, t0, bar_a_full + 8 * as, pol_last);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(tn >> 3) << 17) |
+                             (static_cast<uint32_t>(kBlockM >> 4) << 24);
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int ws = kb % SW, as = kb % SA;
+        if (!mbar_wait(bar_w_full + 8 * ws, (kb / SW) & 1, error, 2, abort_slot)) { ok = false; break; }
+        if (!mbar_wait(bar_a_full + 8 * as, (kb / SA) & 1, error, 7, abort_slot)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint64_t adesc = umma_desc(base + L::kWOff + ws * kWStageBytes);
+        const uint64_t bdesc = umma_desc(base + L::kAOff + as * L::kAStageBytes);
+#pragma unroll
+        for (int kk = 0; kk < kBlockK / 16; ++kk)
+          umma_bf16(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+        umma_commit(bar_w_empty + 8 * ws);
+        umma_commit(bar_a_empty + 8 * as);
+      }
+      if (ok) umma_commit(bar_acc);
+    }
+  } else {
+    // Conversion: the four warps of group g take slabs g, g + 4, ... into bf16 stage g, 32 of the 128 rows each -
+    // four slabs are in work at once and every SM part has four warps to switch between.
+    const int cw = warp - 2, pair = cw >> 2, row_base = (cw & 3) * 32;
+    const int quad = warp & 3;                      // tensor-memory lanes 32 * (warp % 4) .. + 31
+    for (int kb = pair; ok && kb < nkb; kb += SW) {
+      const int rs = kb % R, ws = pair;
+      if (!mbar_wait(bar_raw_full + 8 * rs, (kb / R) & 1, error, 8, abort_slot)) ok = false;
+      if (ok && !mbar_wait(bar_w_empty + 8 * ws, ((kb / SW) & 1) ^ 1, error, 10, abort_slot)) ok = false;
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const uint8_t* raw = base_ptr + L::kRawOff + rs * kW8StageBytes;
+      uint8_t* wst = base_ptr + L::kWOff + ws * kWStageBytes;
+#pragma unroll
+      {
+        const int row = row_base + lane;            // consecutive lanes, consecutive 16-byte pieces: no bank conflicts
+        uint8_t* dst = wst + row * 128;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const uint4 v = *reinterpret_cast<const uint4*>(raw + c * (kBlockM * 16) + row * 16);
+          uint4 o0, o1;
+          e4m3x4_to_bf16(v.x, o0.x, o0.y);
+          e4m3x4_to_bf16(v.y, o0.z, o0.w);
+          e4m3x4_to_bf16(v.z, o1.x, o1.y);
+          e4m3x4_to_bf16(v.w, o1.z, o1.w);
+          *reinterpret_cast<uint4*>(dst + (((2 * c) ^ (row & 7)) << 4)) = o0;       // 16-byte chunks of the 128-byte row,
+          *reinterpret_cast<uint4*>(dst + (((2 * c + 1) ^ (row & 7)) << 4)) = o1;   // swizzled as TMA would have
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read through the async proxy
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar_w_full + 8 * ws);
+        mbar_arrive(bar_raw_empty + 8 * rs);
+      }
+    }
+    // epilogue
+    if (ok && warp < 6 && nkb > 0) ok = mbar_wait(bar_acc, 0, error, 3, abort_slot);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok && warp < 6) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int n = m_tile * kBlockM + quad * 32 + lane;
+      const float sc = n < N ? __ldg(scale + n) : 0.f;
+      float* dstp = out + static_cast<long long>(split) * split_stride;
+      for (int c0 = 0; c0 < tn; c0 += 16) {
+        uint32_t v[16];
+        if (nkb > 0) {
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+              : "r"(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(c0)));
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = 0u;
+        }
+        float val[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) val[i] = __uint_as_float(v[i]) * sc;
+        emit16(epi, dstp, N, T, n, t0 + c0, val);
+      }
+    }
+  }
+
+  // teardown
+  if (!ok) *abort_slot = 1;
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    if (*abort_slot != 0) {
+      const long long t1 = clock64();
+      while (clock64() - t1 < 2000000LL) __nanosleep(1000);
+    }
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(static_cast<uint32_t>(kTmemCols)) : "memory");
+  }
+  stamp_time(epi.stamp_end, true);
+}
+
+// row-major e4m3 bytes [N][K] -> tiles: block (m, kb) = four groups [128 rows][16 bytes], zero where the matrix ends
+__global__ void __launch_bounds__(256) retile_w8_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int N, int K,
+                                                        int n_kslabs) {
+  const int kb = blockIdx.x, mt = blockIdx.y;
+  uint8_t* out = dst + (static_cast<long long>(mt) * n_kslabs + kb) * kW8StageBytes;
+  for (int i = threadIdx.x; i < kW8StageBytes; i += blockDim.x) {
+    const int c = i / (kBlockM * 16), r = (i / 16) % kBlockM, b = i % 16;
+    const int n = mt * kBlockM + r, k = kb * kBlockK + c * 16 + b;
+    out[i] = (n < N && k < K) ? src[static_cast<long long>(n) * K + k] : static_cast<uint8_t>(0);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // CTA-pair kernel for steps of more than 128 tokens (the tensor-bound regime).
 //
 // Two CTAs of a cluster own two neighbouring 128-row weight tiles and the same token tile; one
@@ -638,6 +892,23 @@ int tc_weight_init(TcWeight* w, const void* rowmajor, void* tiled, int N, int K)
   return 0;
 }
 
+size_t tc_weight_w8_tiled_bytes(int N, int K) {
+  return static_cast<size_t>((N + kBlockM - 1) / kBlockM) * ((K + kBlockK - 1) / kBlockK) * kW8StageBytes;
+}
+
+int tc_weight_init_w8(TcWeight* w, const void* rowmajor_bytes, void* tiled, const float* scale, int N, int K) {
+  if (K % 8 || !scale || (reinterpret_cast<uintptr_t>(tiled) & 15)) return -1;
+  const int n_mtiles = (N + kBlockM - 1) / kBlockM, n_kslabs = (K + kBlockK - 1) / kBlockK;
+  retile_w8_kernel<<<dim3(n_kslabs, n_mtiles), 256>>>(static_cast<const uint8_t*>(rowmajor_bytes), static_cast<uint8_t*>(tiled), N, K, n_kslabs);
+  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+  w->w8 = static_cast<const uint8_t*>(tiled);
+  w->scale = scale;
+  w->N = N;
+  w->K = K;
+  w->ready = true;
+  return 0;
+}
+
 void tc_weight_free(TcWeight* w) { w->ready = false; }
 
 int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K) {
@@ -680,6 +951,44 @@ int tc_gemm_split(int T, int N, int K, int n_sm) {
   s = std::min(s, 16);
   const int kb_per = (kb_total + s - 1) / s;
   return (kb_total + kb_per - 1) / kb_per;
+}
+
+// 8-bit weights: one CTA per SM, so K slices fill n_sm slots; at least 4 slabs each
+int tc_gemm_split_w8(int T, int N, int K, int n_sm) {
+  const int tn = T <= kSingleTileMax ? T : 128;
+  const int tiles = ((N + kBlockM - 1) / kBlockM) * ((T + tn - 1) / tn);
+  const int kb_total = (K + kBlockK - 1) / kBlockK;
+  int s = std::max(1, n_sm / tiles);
+  s = std::min(s, std::max(1, kb_total / 4));
+  s = std::min(s, 16);
+  const int kb_per = (kb_total + s - 1) / s;
+  return (kb_total + kb_per - 1) / kb_per;
+}
+
+template <int TN_MAX>
+static int launch_w8(const TcWeight& w, const CUtensorMap& ma, int T, int n_split, float* out, int64_t split_stride,
+                     int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
+  using L = W8SmemLayout<TN_MAX>;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(tc_gemm_w8_kernel<TN_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess) return -1;
+    configured = true;
+  }
+  const int kb_total = (w.K + kBlockK - 1) / kBlockK;
+  const int kb_per = (kb_total + n_split - 1) / n_split;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((T + TN_MAX - 1) / TN_MAX, (w.N + kBlockM - 1) / kBlockM, n_split);
+  cfg.blockDim = dim3(kW8Threads, 1, 1);
+  cfg.dynamicSmemBytes = L::kTotal;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const long long stride = split_stride;
+  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_w8_kernel<TN_MAX>, w.w8, w.scale, ma, T, w.N, kb_total, kb_per, out, stride, error, epi);
+  return err == cudaSuccess ? 1 : -1;
 }
 
 template <int TN_MAX, int STAGES>
@@ -750,6 +1059,14 @@ int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split,
                    int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
   if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
   if (epi.mode != kEpiStore && n_split != 1) return -1;   // a fused epilogue needs the complete sum
+  if (w.w8) {   // 8-bit weights: every step size on the converting kernel (wide steps as 128-token tiles)
+    if (T <= 32) return launch_w8<32>(w, a.map[0], T, n_split, out, split_stride, error, epi, s);
+    if (T <= 64) return launch_w8<64>(w, a.map[1], T, n_split, out, split_stride, error, epi, s);
+    if (T <= 96) return launch_w8<96>(w, a.map[2], T, n_split, out, split_stride, error, epi, s);
+    if (T <= 128) return launch_w8<128>(w, a.map[3], T, n_split, out, split_stride, error, epi, s);
+    if (T <= kSingleTileMax) return launch_w8<160>(w, a.map[4], T, n_split, out, split_stride, error, epi, s);
+    return launch_w8<128>(w, a.map[3], T, n_split, out, split_stride, error, epi, s);
+  }
   // token tile = the smallest box that holds the step; what the narrower activation stage saves goes into ring depth
   if (T <= 32) return launch_split<32, 5>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (T <= 64) return launch_split<64, 4>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);

@@ -14,6 +14,9 @@ struct TcWeight {       // [N][K] bf16 weights, stored as 128 x 64 tiles of 16 K
   CUtensorMap map;      // over the tiled array seen as rows of 128 bytes; box = one tile, 128-byte swizzle
   int N = 0, K = 0;
   bool ready = false;
+  // 8-bit weights instead (tc_weight_init_w8): e4m3 bytes in 8 KB tiles and one fp32 scale per output row
+  const uint8_t* w8 = nullptr;
+  const float* scale = nullptr;
 };
 
 constexpr int kTokenTiles = 6;
@@ -39,10 +42,16 @@ int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int
 // needed afterwards.  Synchronises the device.
 size_t tc_weight_tiled_bytes(int N, int K);
 int tc_weight_init(TcWeight* w, const void* rowmajor, void* tiled, int N, int K);
+// The same for e4m3 bytes [N][K] (row-major, device) with `scale` [N] fp32 (device; must stay valid): W[n][k] =
+// scale[n] * e4m3(byte).  `tiled` holds tc_weight_w8_tiled_bytes(N, K) bytes.  The byte patterns 0x7f / 0xff (NaN in
+// e4m3) must not occur.
+size_t tc_weight_w8_tiled_bytes(int N, int K);
+int tc_weight_init_w8(TcWeight* w, const void* rowmajor_bytes, void* tiled, const float* scale, int N, int K);
 void tc_weight_free(TcWeight* w);
 int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K);
-// number of partial-sum slices [slice][T][N] a launch leaves behind for this shape
+// number of partial-sum slices [slice][T][N] a launch leaves behind for this shape (bf16 weights / 8-bit weights)
 int tc_gemm_split(int T, int N, int K, int n_sm);
+int tc_gemm_split_w8(int T, int N, int K, int n_sm);
 // out[slice][T][N] = A[T][K slice] . W[N][K slice]^T; returns kernels launched (1) or a negative value;
 // `error` is a device word set if a bounded wait ran out
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,

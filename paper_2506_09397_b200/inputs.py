@@ -107,6 +107,43 @@ def make_weights(shape: ModelShape, seed: int = 0, device: str = "cpu") -> dict:
     return w
 
 
+LINEAR_NAMES = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down")
+
+
+def to_e4m3_rows(w: torch.Tensor):
+    """Storage format of the 8-bit weight path: every row of a matrix divided by its scale = max|row| / 448 and
+    rounded to the nearest e4m3 value.  Returns (bytes uint8 [N, K], scale fp32 [N])."""
+    w32 = w.to(torch.float32)
+    scale = w32.abs().amax(dim=1) / 448.0
+    scale = torch.where(scale > 0, scale, torch.ones_like(scale))
+    q = (w32 / scale[:, None]).to(torch.float8_e4m3fn)
+    return q.view(torch.uint8).contiguous(), scale.contiguous()
+
+
+def from_e4m3_rows(q: torch.Tensor, scale: torch.Tensor) -> torch.Tensor:
+    """The matrix those bytes and scales stand for, in fp32 (scale * e4m3 value, one rounding)."""
+    return q.view(torch.float8_e4m3fn).to(torch.float32) * scale[:, None]
+
+
+def quantize_linear_weights(w: dict, dequantised: bool = True):
+    """(weights for the 8-bit path, the same model with its linear layers as fp32 matrices - or None when
+    `dequantised` is off).  The first holds e4m3 bytes and `<name>_scale` for the linear layers and the LM head,
+    everything else as in `w`; the second is what those bytes mean, for whoever wants to compute with them in
+    another way."""
+    q, deq = dict(w), (dict(w) if dequantised else None)
+    b, sc = to_e4m3_rows(w["lm_head"])
+    q["lm_head"], q["lm_head_scale"] = b, sc
+    if dequantised:
+        deq["lm_head"] = from_e4m3_rows(b, sc)
+    for name in LINEAR_NAMES:
+        pairs = [to_e4m3_rows(t) for t in w[name]]
+        q[name] = [p[0] for p in pairs]
+        q[name + "_scale"] = [p[1] for p in pairs]
+        if dequantised:
+            deq[name] = [from_e4m3_rows(*p) for p in pairs]
+    return q, deq
+
+
 def weights_to(w: dict, device: str) -> dict:
     return {k: ([t.to(device) for t in v] if isinstance(v, list) else v.to(device)) for k, v in w.items()}
 

@@ -1,0 +1,98 @@
+"""The 8-bit weight path (linear_weight_bits = 8: e4m3 bytes with one fp32 scale per output row, bf16 activations)
+against the oracle run on the matrices those bytes stand for.  Nothing is quantised on the device: both sides are
+given the same bytes and scales, so the comparison is the bf16 path's (inputs of every product rounded to bf16, fp32
+sums), with the same tolerance."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2506_09397_b200 import binding as B
+from paper_2506_09397_b200 import inputs as I
+from test_gpu_forward import TOL, _verify_both
+
+pytestmark = pytest.mark.gpu
+
+
+def _both_sides(shape, w_bf16, **eng_args):
+    """Engine on the bytes, oracle on the fp32 matrices they mean (embedding and gains widened exactly)."""
+    q, deq = I.quantize_linear_weights(w_bf16)
+    eng = B.Engine(shape, q, linear_weight_bits=8, **eng_args)
+    f32 = {k: ([t.float().numpy() for t in v] if isinstance(v, list) else v.float().numpy())
+           for k, v in deq.items() if not k.endswith("_scale")}
+    orc = O.OracleModel(dataclasses.replace(shape, weight_dtype="fp32"), f32)
+    return eng, orc
+
+
+def test_every_byte_pattern_is_decoded():
+    # LM-head row n holds byte n in every column (scale 1): its logit is e4m3(n) x (sum of the normalised hidden
+    # state).  All 254 patterns - subnormals and both zeros among them - against the oracle's fp32 matrix.
+    shape = I.ModelShape("w8_bytes", 1, 256, 4, 2, 64, 512, 256, 5e5, "bf16", "bf16")
+    w = I.make_weights(shape, seed=3)
+    q, deq = I.quantize_linear_weights(w)
+    pattern = torch.arange(256, dtype=torch.uint8)
+    pattern[0x7f] = 0
+    pattern[0xff] = 0
+    q["lm_head"] = pattern[:, None].repeat(1, shape.d_model).contiguous()
+    q["lm_head_scale"] = torch.ones(256)
+    deq["lm_head"] = I.from_e4m3_rows(q["lm_head"], q["lm_head_scale"])
+    values = deq["lm_head"][:, 0]
+    assert float(values[0x01]) == 2.0 ** -9 and float(values[0x7e]) == 448.0 and float(values[0x88]) == -(2.0 ** -6)
+    eng = B.Engine(shape, q, linear_weight_bits=8, n_pages=8, max_batch=2, max_k=2, max_step_tokens=8)
+    f32 = {k: ([t.float().numpy() for t in v] if isinstance(v, list) else v.float().numpy())
+           for k, v in deq.items() if not k.endswith("_scale")}
+    orc = O.OracleModel(dataclasses.replace(shape, weight_dtype="fp32"), f32)
+    p = I.make_prompt(shape.vocab, 5, 3, 1)
+    eng.prefill(1, p)
+    orc.prefill(1, p)
+    d, qq = I.make_drafts(shape.vocab, 2, 3, 1)
+    eng.set_commit(False)
+    eng.verify_batch([(1, d.numpy(), qq.numpy())], 0)
+    glog = eng.logits(3)
+    st, n_acc, nxt, ol, mg = orc.verify(1, d.numpy(), qq.numpy(), 0, commit=False)
+    hidden_sum = ol[:, 0x38] / float(values[0x38])                     # byte 0x38 is 1.0
+    assert np.all(np.abs(hidden_sum) > 1.0), hidden_sum
+    mag = np.maximum(np.abs(values.numpy()), 2.0 ** -9)
+    for row in range(3):
+        want = values.numpy() * hidden_sum[row]
+        assert np.max(np.abs(ol[row] - want)) <= 1e-3 * np.max(np.abs(want))          # the oracle itself
+        # a wrongly decoded byte is off by an eighth of its value at least; bf16 inputs cost far less
+        assert np.all(np.abs(glog[row] - want) <= mag * (2e-2 * np.abs(hidden_sum[row]) + 0.05)), row
+    eng.shutdown()
+
+
+@pytest.mark.parametrize("n_req,k", [(4, 4), (16, 8), (40, 8)])
+def test_steps_with_8bit_weights_match_the_oracle(n_req, k):
+    # narrow and wide steps (20, 144 and 360 tokens: token tiles of 32, 160 and 3 x 128), prefill in chunks, commit
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=5)
+    eng, orc = _both_sides(shape, w, n_pages=4 * n_req + 32, max_batch=n_req, max_k=8, max_step_tokens=max(n_req * (k + 1), 64))
+    checked = sorted({0, n_req // 2, n_req - 1})
+    for c in range(n_req):
+        p = I.make_prompt(shape.vocab, 3 + (5 * c) % 31, 5, c)
+        eng.prefill(c, p)
+        if c in checked:
+            orc.prefill(c, p)
+    explain = []
+    for step in range(2):
+        reqs = [(c,) + tuple(I.make_drafts(shape.vocab, k, 5, c, step)) for c in range(n_req)]
+        if step == 0:
+            # every request on the device, the checked ones on both sides
+            eng.set_commit(False)
+            eng.verify_batch([(c, d.numpy(), q.numpy()) for c, d, q in reqs], step)
+            eng.set_commit(True)
+        _verify_both(eng, orc, [r for r in reqs if r[0] in checked], seed=step, tau=1.0, greedy=False, tol=TOL["bf16"],
+                     explain=explain)
+    eng.shutdown()
+
+
+def test_8bit_weights_need_scales_and_bf16():
+    shape = I.SMALL_GQA
+    w = I.make_weights(shape, seed=5)
+    with pytest.raises(B.SledError):
+        B.Engine(I.TINY, I.quantize_linear_weights(I.make_weights(I.TINY, 0))[0], linear_weight_bits=8, n_pages=8,
+                 max_batch=1, max_k=1, max_step_tokens=8)      # fp32 model
+    with pytest.raises(B.SledError):
+        B.Engine(shape, w, linear_weight_bits=4, n_pages=8, max_batch=1, max_k=1, max_step_tokens=8)

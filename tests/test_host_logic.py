@@ -196,3 +196,19 @@ def test_page_manager_goes_back_to_a_base_length():
     assert m2.commit(1, 3, 5) == 0
     assert m2.history(1)[1] == (6, [5])
     assert m2.reserve_batch([1], [1], [6]) == B.SLED_ERR_BASE_LEN and m2.reserve_batch([1], [1], [7]) == 0
+
+
+def test_e4m3_storage_format_round_trip():
+    # what inputs.to_e4m3_rows stores is within half a step of the row-scaled value, the largest entry of a row lands
+    # on the largest e4m3 number, and the NaN patterns never occur
+    import torch
+    from paper_2506_09397_b200 import inputs as I
+    w = torch.randn(64, 256, generator=torch.Generator().manual_seed(1)) * 0.02
+    b, sc = I.to_e4m3_rows(w)
+    back = I.from_e4m3_rows(b, sc)
+    assert b.dtype == torch.uint8 and not bool(((b & 0x7f) == 0x7f).any())
+    assert torch.all((back - w).abs() <= w.abs() * 2.0 ** -4 + sc[:, None] * 2.0 ** -10)
+    assert torch.allclose(back.abs().amax(dim=1), w.abs().amax(dim=1))
+    table = I.from_e4m3_rows(torch.arange(256, dtype=torch.uint8)[:, None], torch.ones(256))[:, 0]
+    assert float(table[0x01]) == 2.0 ** -9 and float(table[0x08]) == 2.0 ** -6 and float(table[0x38]) == 1.0
+    assert float(table[0x7e]) == 448.0 and float(table[0xb8]) == -1.0
