@@ -89,7 +89,11 @@ typedef struct sled_config {
                              exponent bits with bias 7, 3 mantissa bits, subnormals, no infinities; the patterns 0x7f and
                              0xff must not occur) and every output row has an fp32 scale: W[n][k] = scale[n] *
                              e4m3(byte[n][k]).  Half the weight bytes per step (the paper sweeps 16-, 8- and 4-bit
-                             precision, Section 4); activations, embedding and norms stay bf16, sums fp32. */
+                             precision, Section 4).  The linear layers then run on fp8 tensor-core instructions, which
+                             take both operands in 8 bits: every bf16 activation goes in as the sum of two e4m3 numbers
+                             times a per-token scale - eight significant bits, as in bf16 - and the products are summed
+                             in fp32; embedding, norms, attention and cache are as with 16-bit weights.  d_model, ffn_dim
+                             and n_q_heads * head_dim must be multiples of 16. */
 } sled_config;
 
 /* Target weights, row-major [out][in], all of type weight_dtype.  HOST or DEVICE

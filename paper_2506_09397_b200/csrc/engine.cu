@@ -93,6 +93,8 @@ struct sled_engine {
   float* q_stage = nullptr;
   bool attn_tc = false;          // head_dim 128, bf16 cache, 16-token pages: attention may run on tcgen05
   TcActivation tc_norm, tc_attn, tc_ffn;
+  TcActivation8 a8_norm, a8_attn, a8_ffn;   // 8-bit weights: the same activations as two e4m3 parts + token scales
+  bool norm_split = false;                  // the normalisation kernel has filled a8_norm for the act_norm now in place
   int32_t* tc_error = nullptr;  // device word set by a kernel whose bounded wait ran out: the first word of the
                                 // results block (d_results), so the step's one result copy brings it along
 
@@ -186,7 +188,7 @@ int simt_split(int T, int N, int K, int n_sm) {
 }
 
 int linear_split(const sled_engine* e, int T, const Linear& L) {
-  if (L.tc.w8) return tc_gemm_split_w8(T, L.N, L.K, e->n_sm);
+  if (L.tc.f8) return tc_gemm_split_f8(T, L.N, L.K, e->n_sm);
   if (e->cfg.weight_dtype == SLED_BF16) return tc_gemm_split(T, L.N, L.K, e->n_sm);
   return simt_split(T, L.N, L.K, e->n_sm);
 }
@@ -198,6 +200,17 @@ int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Lin
   float* out = dst ? dst : e->partial;
   const int64_t stride = static_cast<int64_t>(T) * L.N;
   if (!dst && static_cast<size_t>(split) * stride > e->partial_elems) return SLED_ERR_DEVICE;
+  const TcActivation8* a8 = nullptr;
+  if (L.tc.f8) {   // fp8 MMAs: the input goes in as two e4m3 parts per element and a scale per token
+    a8 = tcA == &e->tc_norm ? &e->a8_norm : tcA == &e->tc_attn ? &e->a8_attn : &e->a8_ffn;
+    if (!(a8 == &e->a8_norm && e->norm_split)) {
+      e->mark(K_OTHER);
+      const Stamp ss = e->stamp(K_OTHER);
+      const int ns = tc_split_rows_launch(A, T, *a8, e->stream, ss.begin, ss.end);
+      if (ns < 0) return SLED_ERR_DEVICE;
+      e->count(ns, K_OTHER);
+    }
+  }
   e->mark(K_LINEAR);
   const Stamp st = e->stamp(K_LINEAR);
   int n;
@@ -205,7 +218,8 @@ int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Lin
     TcEpilogue ep = epi;
     ep.stamp_begin = st.begin;
     ep.stamp_end = st.end;
-    n = tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_error, ep, e->stream);
+    n = a8 ? tc_gemm_f8_launch(*a8, L.tc, T, split, out, stride, e->tc_error, ep, e->stream)
+           : tc_gemm_launch(*tcA, L.tc, T, split, out, stride, e->tc_error, ep, e->stream);
   } else {
     n = launch_gemm_simt(A, e->adtype(), L.w, e->cfg.weight_dtype, T, L.N, L.K, split, out, stride, e->stream, st);
   }
@@ -428,6 +442,7 @@ AttnArgs attn_args(sled_engine* e, const Packed& pk, int layer, const void* q, v
 int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
   const sled_config& c = e->cfg;
   const int T = pk.T, d = c.d_model, ad = e->adtype();
+  const bool f8 = !e->layers.empty() && e->layers[0].qkv.tc.f8;   // fp8 linear layers: the normalisation also splits its output
   int n;
   e->mark(K_OTHER);
   n = launch_embed(e->tok_emb, c.weight_dtype, pk.ids, T, d, e->x, e->stream, e->stamp(K_OTHER));
@@ -440,7 +455,8 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
     Layer& L = e->layers[l];
     e->mark(K_OTHER);
     n = launch_add_rmsnorm(e->x, e->partial, split, stride, L.attn_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm,
-                           ad, e->stream, e->stamp(K_OTHER));
+                           ad, e->stream, e->stamp(K_OTHER), f8 ? e->a8_norm.data : nullptr, e->a8_norm.rows,
+                           f8 ? e->a8_norm.scale : nullptr, &e->norm_split);
     if (n < 0) return SLED_ERR_DEVICE;
     e->count(n, K_OTHER);
     int s_qkv;
@@ -461,7 +477,8 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
     stride = static_cast<int64_t>(T) * L.o.N;
     e->mark(K_OTHER);
     n = launch_add_rmsnorm(e->x, e->partial, split, stride, L.ffn_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm, ad,
-                           e->stream, e->stamp(K_OTHER));
+                           e->stream, e->stamp(K_OTHER), f8 ? e->a8_norm.data : nullptr, e->a8_norm.rows,
+                           f8 ? e->a8_norm.scale : nullptr, &e->norm_split);
     e->count(n, K_OTHER);
     int s_gu;
     if (c.weight_dtype == SLED_BF16 && linear_split(e, T, L.gate_up) == 1) {
@@ -487,7 +504,8 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
   if (need_logits) {
     e->mark(K_OTHER);
     n = launch_add_rmsnorm(e->x, e->partial, split, stride, e->final_norm, c.weight_dtype, c.rms_eps, T, d, e->act_norm,
-                           ad, e->stream, e->stamp(K_OTHER));
+                           ad, e->stream, e->stamp(K_OTHER), f8 ? e->a8_norm.data : nullptr, e->a8_norm.rows,
+                           f8 ? e->a8_norm.scale : nullptr, &e->norm_split);
     e->count(n, K_OTHER);
     int s1;
     int rc = run_linear(e, e->act_norm, &e->tc_norm, e->lm_head, T, e->logits, &s1);
@@ -617,8 +635,8 @@ int finish_linear(sled_engine* e, Linear* L, void* rowmajor, float* scale, int N
   if (w8(e)) {
     L->scale = scale;
     e->allocs.push_back(scale);
-    int rc = dmalloc(e, &L->w, tc_weight_w8_tiled_bytes(N, K));
-    if (!rc && tc_weight_init_w8(&L->tc, rowmajor, L->w, scale, N, K) != 0) rc = SLED_ERR_ARG;
+    int rc = dmalloc(e, &L->w, tc_weight_f8_tiled_bytes(N, K));
+    if (!rc && tc_weight_init_f8(&L->tc, rowmajor, L->w, scale, N, K) != 0) rc = SLED_ERR_ARG;
     cudaFree(rowmajor);
     return rc;
   }
@@ -702,6 +720,7 @@ int check_cfg(const sled_config& c) {
   if (c.attention_impl != 0 && c.attention_impl != 1) return SLED_ERR_ARG;
   if (c.linear_weight_bits != 0 && c.linear_weight_bits != 16 && c.linear_weight_bits != 8) return SLED_ERR_ARG;
   if (c.linear_weight_bits == 8 && c.weight_dtype != SLED_BF16) return SLED_ERR_ARG;
+  if (c.linear_weight_bits == 8 && (c.d_model % 16 || c.ffn_dim % 16 || (c.n_q_heads * c.head_dim) % 16)) return SLED_ERR_ARG;
   if (c.page_size <= 0 || c.n_pages <= 0 || c.max_batch <= 0 || c.max_k < 0 || c.max_step_tokens <= 0)
     return SLED_ERR_ARG;
   if (c.max_step_tokens < c.max_k + 1) return SLED_ERR_ARG;
@@ -848,6 +867,18 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
         tc_activation_init(&e->tc_attn, e->attn_out, static_cast<int>(padT), qd) ||
         tc_activation_init(&e->tc_ffn, e->act_ffn, static_cast<int>(padT), F))
       return fail(SLED_ERR_DEVICE);
+    if (c.linear_weight_bits == 8) {
+      struct { TcActivation8* a; int K; } parts[3] = {{&e->a8_norm, d}, {&e->a8_attn, qd}, {&e->a8_ffn, F}};
+      for (auto& p : parts) {
+        void* data = nullptr;
+        float* sc = nullptr;
+        if ((rc = dmalloc(e, &data, 2 * padT * p.K)) || (rc = dmalloc(e, reinterpret_cast<void**>(&sc), padT * sizeof(float))))
+          return fail(rc);
+        if (cudaMemset(data, 0, 2 * padT * p.K) != cudaSuccess || cudaMemset(sc, 0, padT * sizeof(float)) != cudaSuccess ||
+            tc_activation8_init(p.a, data, sc, static_cast<int>(padT), p.K))
+          return fail(SLED_ERR_DEVICE);
+      }
+    }
   }
 
   // metadata staging: tokens, requests, page table (every page at most once, plus one partial page per request), items
@@ -1402,7 +1433,7 @@ int sled_debug_set_commit(sled_engine* e, int32_t commit) {
 int sled_debug_set_timing(sled_engine* e, int32_t mode) {
   if (!e || mode < 0 || mode > 2) return SLED_ERR_ARG;
   cudaSetDevice(e->cfg.device_index);
-  const size_t n = 16 + 12 * static_cast<size_t>(e->cfg.n_layers);
+  const size_t n = 16 + 20 * static_cast<size_t>(e->cfg.n_layers);   // launches (or kernel groups) of a step, with room to spare
   if (mode == 2 && e->ev_pool.empty()) {
     e->ev_pool.resize(n);
     e->ev_kind.assign(n, K_OTHER);

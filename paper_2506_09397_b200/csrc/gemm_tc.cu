@@ -23,6 +23,7 @@
 #include <algorithm>
 #include <cstdio>
 
+#include "fp8_split.cuh"
 #include "gemm_tc.h"
 
 namespace sled {
@@ -288,78 +289,58 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
 }
 
 // ------------------------------------------------------------------------------------------------
-// Linear layer with 8-bit weights (e4m3 bytes, one fp32 scale per output row; activations stay bf16).
-//
-// The weight bytes are what a narrow step streams, so they cross DRAM and L2 as bytes: a tile (128 rows x 64 k) is
-// 8 KB, stored as four groups [128 rows][16 bytes] (group c = bytes 16c .. 16c+15 of every row) and fetched with one
-// bulk copy into a deep ring (10-14 stages, 80-112 KB in flight per SM).  Warps 2-5 - idle until the epilogue in the
-// bf16 kernel - turn raw stages into the 128-byte-swizzled bf16 tiles the MMA reads: a lane takes the 16 bytes of a
-// row's group (consecutive lanes read consecutive 16-byte pieces: no bank conflicts), widens every byte
-// s.eeee.mmm to the bf16 pattern s.0000eeee.mmm0000 - the same number times 2^-120, subnormals included - and
-// multiplies by 2^120 (an exact bf16 x bf16 product), then stores two 16-byte chunks at their swizzled places.
-// The MMAs run exactly as in the bf16 kernel; the row's scale multiplies the fp32 sums in the epilogue.
-// One CTA per SM (224 KB of shared memory): rings of 10-14 raw stages, 4 bf16 weight stages, 4 activation stages.
-//   warp 0    : bulk copies of raw weight tiles (before the wait on the previous kernel) and TMA loads of activations
-//   warp 1    : tensor memory, MMAs; commits a slab to the "bf16 stage free" and "activation stage free" barriers
-//   warps 2-17: conversion; warps 2-5 then run the epilogue
-// All waits are bounded as above.
-constexpr int kW8StageBytes = kBlockM * kBlockK;   // 8 KB
-constexpr int kW8MmaStages = 4;
-constexpr int kW8ConvWarps = 16;                   // warps 2..17 convert: four per bf16 stage, 32 rows each
-constexpr int kW8Threads = 64 + 32 * kW8ConvWarps;
-static_assert(kW8ConvWarps == 4 * kW8MmaStages, "four conversion warps per bf16 weight stage");
-template <int TN_MAX>
-struct W8SmemLayout {
-  // every ring has to cover its own latency at the pace DRAM delivers a slab (about 350 cycles): raw tiles come
-  // from DRAM, activation tiles from L2, and a bf16 stage is busy from the start of its conversion to the end of its MMAs
-  static constexpr int kActStages = TN_MAX <= 96 ? 8 : TN_MAX <= 128 ? 6 : 4;
-  static constexpr int kRawStages = TN_MAX <= 32 ? 16 : TN_MAX <= 64 ? 12 : TN_MAX <= 128 ? 8 : 10;
-  static constexpr int kAStageBytes = TN_MAX * kBlockK * 2;
-  static constexpr int kWOff = 0;                                          // bf16 weight stages (1024-byte aligned)
-  static constexpr int kAOff = kW8MmaStages * kWStageBytes;                // activation stages (multiples of 1 KB)
-  static constexpr int kRawOff = kAOff + kActStages * kAStageBytes;         // raw weight stages
-  static constexpr int kTiles = kRawOff + kRawStages * kW8StageBytes;
-  static constexpr int kBars = 2 * kRawStages + 2 * kW8MmaStages + 2 * kActStages + 1;
-  static constexpr int kTotal = kTiles + 8 * kBars + 16;
-};
+// Linear layer with 8-bit weights, fp8 MMAs (tcgen05 kind::f8f6f4): nothing is converted on the way to the tensor
+// cores.  The instruction wants both operands in 8 (or fewer) bits, so the bf16 activations are handed over as TWO
+// e4m3 numbers each, a = s_t * (hi + lo) with hi = e4m3(a / s_t), lo = e4m3(a / s_t - hi) and one scale s_t per
+// token (split_rows_f8_kernel, run once per activation tensor): the products W * hi and W * lo are exact in the
+// fp32 accumulators, so the sum carries eight significant bits of every activation, as bf16 does.  Per k-slab
+// (128 k = one 128-byte swizzle row) a CTA streams a 16 KB weight tile - the same bytes per slab as the bf16 kernel,
+// twice the reduction length - and fetches the token tile's hi rows and lo rows into one stage; one MMA per 32-k
+// step takes the whole stage as its N side (N = 2 x token tile), so W * hi and W * lo land side by side in tensor
+// memory, and the epilogue adds them and applies both scales.  (Two MMAs per step into separate or into the same
+// columns measured slower: at these widths an instruction costs about the same whether N is 96 or 192.)
+// Structure, roles and waits as in tc_gemm_split_kernel; the weight ring and the activation ring are separate
+// (4 + 2 stages at 96 tokens) so that two CTAs still fit an SM.  Wider steps run as 128-token tiles.
+constexpr int kBlockK8 = 128;
 
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+__device__ __forceinline__ void umma_f8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar), "l"(policy)
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
       : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// four e4m3 bytes -> four bf16 (two packed pairs), exact
-__device__ __forceinline__ void e4m3x4_to_bf16(uint32_t w, uint32_t& lo, uint32_t& hi) {
-  const uint32_t y0 = __byte_perm(w, 0u, 0x1404);   // bytes 0 and 1 into the high byte of each 16-bit half
-  const uint32_t y1 = __byte_perm(w, 0u, 0x3424);   // bytes 2 and 3
-  const uint32_t v0 = (y0 & 0x80008000u) | ((y0 >> 4) & 0x07f007f0u);
-  const uint32_t v1 = (y1 & 0x80008000u) | ((y1 >> 4) & 0x07f007f0u);
-  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(lo) : "r"(v0), "r"(0x7B807B80u));   // x 2^120
-  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(hi) : "r"(v1), "r"(0x7B807B80u));
-}
 
 template <int TN_MAX>
-__global__ void __launch_bounds__(kW8Threads) tc_gemm_w8_kernel(const uint8_t* __restrict__ w8, const float* __restrict__ scale,
+struct F8SmemLayout {
+  static constexpr int kWStages = TN_MAX <= 64 ? 5 : TN_MAX <= 96 ? 4 : 3;
+  static constexpr int kAStages = TN_MAX <= 32 ? 3 : 2;
+  static constexpr int kAStageBytes = 2 * TN_MAX * kBlockK8;               // hi rows, then lo rows
+  static constexpr int kAOff = kWStages * kWStageBytes;
+  static constexpr int kTiles = kAOff + kAStages * kAStageBytes;
+  static constexpr int kTotal = kTiles + 256;
+  static_assert(2 * (kTotal + 1024) <= 228 * 1024, "two CTAs per SM");
+};
+
+template <int TN_MAX>
+__global__ void __launch_bounds__(192) tc_gemm_f8_kernel(const __grid_constant__ CUtensorMap map_w,
                                                          const __grid_constant__ CUtensorMap map_a, int T, int N,
-                                                         int kb_total, int kb_per_split, float* __restrict__ out,
-                                                         long long split_stride, int32_t* error, TcEpilogue epi) {
-  using L = W8SmemLayout<TN_MAX>;
-  constexpr int R = L::kRawStages, SW = kW8MmaStages, SA = L::kActStages;
-  static_assert(L::kTotal <= 227 * 1024, "one CTA's shared memory");
-  constexpr int kTmemCols = TN_MAX <= 32 ? 32 : TN_MAX <= 64 ? 64 : TN_MAX <= 128 ? 128 : 256;
+                                                         int kb_total, int kb_per_split, int lo_row0,
+                                                         const float* __restrict__ wscale, const float* __restrict__ ascale,
+                                                         float* __restrict__ out, long long split_stride, int32_t* error,
+                                                         TcEpilogue epi) {
+  using L = F8SmemLayout<TN_MAX>;
+  constexpr int SW = L::kWStages, SA = L::kAStages;
+  constexpr int kTmemCols = TN_MAX <= 32 ? 64 : TN_MAX <= 64 ? 128 : 256;   // W * hi | W * lo, TN_MAX columns each
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   uint8_t* base_ptr = smem_raw;
   const uint32_t bars = base + L::kTiles;
-  const uint32_t bar_raw_full = bars, bar_raw_empty = bars + 8 * R, bar_w_full = bars + 16 * R,
-                 bar_w_empty = bar_w_full + 8 * SW, bar_a_full = bar_w_empty + 8 * SW, bar_a_empty = bar_a_full + 8 * SA,
+  const uint32_t bar_w_full = bars, bar_w_empty = bars + 8 * SW, bar_a_full = bars + 16 * SW, bar_a_empty = bar_a_full + 8 * SA,
                  bar_acc = bar_a_empty + 8 * SA;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kTiles + 8 * L::kBars);
-  volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * L::kBars + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kTiles + 8 * (2 * SW + 2 * SA + 1));
+  volatile int* abort_slot = reinterpret_cast<volatile int*>(base_ptr + L::kTiles + 8 * (2 * SW + 2 * SA + 1) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   stamp_time(epi.stamp_begin, false);
@@ -375,11 +356,9 @@ __global__ void __launch_bounds__(kW8Threads) tc_gemm_w8_kernel(const uint8_t* _
     *abort_slot = (base & 1023u) ? 1 : 0;
   }
   if (warp == 0 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
-    for (int i = 0; i < R; ++i) { mbar_init(bar_raw_full + 8 * i, 1); mbar_init(bar_raw_empty + 8 * i, 4); }
-    for (int i = 0; i < SW; ++i) { mbar_init(bar_w_full + 8 * i, 4); mbar_init(bar_w_empty + 8 * i, 1); }
-    for (int i = 0; i < SA; ++i) { mbar_init(bar_a_full + 8 * i, 1); mbar_init(bar_a_empty + 8 * i, 1); }
-    mbar_init(bar_acc, 1);
+    for (int i = 0; i < 2 * SW + 2 * SA + 1; ++i) mbar_init(bars + 8 * i, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -392,129 +371,98 @@ __global__ void __launch_bounds__(kW8Threads) tc_gemm_w8_kernel(const uint8_t* _
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
   bool ok = true;
-  if (threadIdx.x == 32 && *reinterpret_cast<volatile int32_t*>(error) != 0) *abort_slot = 1;
+  if (threadIdx.x == 64 && *reinterpret_cast<volatile int32_t*>(error) != 0) *abort_slot = 1;
 
   if (warp == 0) {
     if (lane == 0 && *abort_slot == 0) {
       uint64_t pol_first, pol_last;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_last));
-      const uint8_t* w_mine = w8 + (static_cast<long long>(m_tile) * kb_total + kb0) * kW8StageBytes;
-      const int pre_raw = min(R, nkb);
-      for (int kb = 0; kb < pre_raw; ++kb) {   // weights do not depend on the previous kernel
-        mbar_expect_tx(bar_raw_full + 8 * kb, kW8StageBytes);
-        bulk_load(base + L::kRawOff + kb * kW8StageBytes, w_mine + static_cast<long long>(kb) * kW8StageBytes, kW8StageBytes,
-                  bar_raw_full + 8 * kb, pol_first);
-      }
+      auto load_w = [&](int kb, int st) {
+        mbar_expect_tx(bar_w_full + 8 * st, kWStageBytes);
+        tma_load_2d(base + st * kWStageBytes, &map_w, 0, (m_tile * kb_total + kb0 + kb) * kBlockM, bar_w_full + 8 * st, pol_first);
+      };
+      auto load_a = [&](int kb, int st) {
+        mbar_expect_tx(bar_a_full + 8 * st, L::kAStageBytes);
+        const uint32_t dst = base + L::kAOff + st * L::kAStageBytes;
+        tma_load_2d(dst, &map_a, (kb0 + kb) * kBlockK8, t0, bar_a_full + 8 * st, pol_last);
+        tma_load_2d(dst + TN_MAX * kBlockK8, &map_a, (kb0 + kb) * kBlockK8, lo_row0 + t0, bar_a_full + 8 * st, pol_last);
+      };
+      for (int kb = 0; kb < min(SW, nkb); ++kb) load_w(kb, kb);   // weights do not depend on the previous kernel
       pdl_wait_here();
-      const int pre_a = min(SA, nkb);
-      for (int kb = 0; kb < pre_a; ++kb) {
-        mbar_expect_tx(bar_a_full + 8 * kb, L::kAStageBytes);
-        tma_load_2d(base + L::kAOff + kb * L::kAStageBytes, &map_a, (kb0 + kb) * kBlockK, t0, bar_a_full + 8 * kb, pol_last);
-      }
+      for (int kb = 0; kb < min(SA, nkb); ++kb) load_a(kb, kb);
       for (int kb = 0; ok && kb < nkb; ++kb) {
-        const int kr = kb + R;     // the raw stage of slab kb is free once it has been converted
-        if (kr < nkb) {
-          const int rs = kr % R;
-          if (!mbar_wait(bar_raw_empty + 8 * rs, ((kr / R) & 1) ^ 1, error, 1, abort_slot)) { ok = false; break; }
-          mbar_expect_tx(bar_raw_full + 8 * rs, kW8StageBytes);
-          bulk_load(base + L::kRawOff + rs * kW8StageBytes, w_mine + static_cast<long long>(kr) * kW8StageBytes, kW8StageBytes,
-                    bar_raw_full + 8 * rs, pol_first);
-        }
-        const int ka = kb + SA;    // the activation stage of slab kb is free once its MMAs have run
+        const int kw = kb + SW, ka = kb + SA;
         if (ka < nkb) {
-          const int as = ka % SA;
-          if (!mbar_wait(bar_a_empty + 8 * as, ((ka / SA) & 1) ^ 1, error, 6, abort_slot)) { ok = false; break; }
-          mbar_expect_tx(bar_a_full + 8 * as, L::kAStageBytes);
-          tma_load_2d(base + L::kAOff + as * L::kAStageBytes, &map_a, (kb0 + ka) * kBlockK, t0, bar_a_full + 8 * as, pol_last);
+          if (!mbar_wait(bar_a_empty + 8 * (ka % SA), ((ka / SA) & 1) ^ 1, error, 6, abort_slot)) { ok = false; break; }
+          load_a(ka, ka % SA);
+        }
+        if (kw < nkb) {
+          if (!mbar_wait(bar_w_empty + 8 * (kw % SW), ((kw / SW) & 1) ^ 1, error, 1, abort_slot)) { ok = false; break; }
+          load_w(kw, kw % SW);
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(tn >> 3) << 17) |
-                             (static_cast<uint32_t>(kBlockM >> 4) << 24);
+      // instruction descriptor: fp32 accumulate, e4m3 x e4m3 (format code 0 for both), K-major, M = 128, and
+      // N = the whole activation stage - hi rows and lo rows in one instruction, their sums side by side
+      const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>((2 * TN_MAX) >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
       for (int kb = 0; kb < nkb; ++kb) {
         const int ws = kb % SW, as = kb % SA;
         if (!mbar_wait(bar_w_full + 8 * ws, (kb / SW) & 1, error, 2, abort_slot)) { ok = false; break; }
         if (!mbar_wait(bar_a_full + 8 * as, (kb / SA) & 1, error, 7, abort_slot)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t adesc = umma_desc(base + L::kWOff + ws * kWStageBytes);
+        const uint64_t adesc = umma_desc(base + ws * kWStageBytes);
         const uint64_t bdesc = umma_desc(base + L::kAOff + as * L::kAStageBytes);
 #pragma unroll
-        for (int kk = 0; kk < kBlockK / 16; ++kk)
-          umma_bf16(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+        for (int kk = 0; kk < kBlockK8 / 32; ++kk)   // 32 fp8 = 32 bytes further along K inside the swizzled row
+          umma_f8(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
         umma_commit(bar_w_empty + 8 * ws);
         umma_commit(bar_a_empty + 8 * as);
       }
       if (ok) umma_commit(bar_acc);
     }
   } else {
-    // Conversion: the four warps of group g take slabs g, g + 4, ... into bf16 stage g, 32 of the 128 rows each -
-    // four slabs are in work at once and every SM part has four warps to switch between.
-    const int cw = warp - 2, pair = cw >> 2, row_base = (cw & 3) * 32;
     const int quad = warp & 3;                      // tensor-memory lanes 32 * (warp % 4) .. + 31
-    for (int kb = pair; ok && kb < nkb; kb += SW) {
-      const int rs = kb % R, ws = pair;
-      if (!mbar_wait(bar_raw_full + 8 * rs, (kb / R) & 1, error, 8, abort_slot)) ok = false;
-      if (ok && !mbar_wait(bar_w_empty + 8 * ws, ((kb / SW) & 1) ^ 1, error, 10, abort_slot)) ok = false;
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      const uint8_t* raw = base_ptr + L::kRawOff + rs * kW8StageBytes;
-      uint8_t* wst = base_ptr + L::kWOff + ws * kWStageBytes;
-#pragma unroll
-      {
-        const int row = row_base + lane;            // consecutive lanes, consecutive 16-byte pieces: no bank conflicts
-        uint8_t* dst = wst + row * 128;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint4 v = *reinterpret_cast<const uint4*>(raw + c * (kBlockM * 16) + row * 16);
-          uint4 o0, o1;
-          e4m3x4_to_bf16(v.x, o0.x, o0.y);
-          e4m3x4_to_bf16(v.y, o0.z, o0.w);
-          e4m3x4_to_bf16(v.z, o1.x, o1.y);
-          e4m3x4_to_bf16(v.w, o1.z, o1.w);
-          *reinterpret_cast<uint4*>(dst + (((2 * c) ^ (row & 7)) << 4)) = o0;       // 16-byte chunks of the 128-byte row,
-          *reinterpret_cast<uint4*>(dst + (((2 * c + 1) ^ (row & 7)) << 4)) = o1;   // swizzled as TMA would have
-        }
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read through the async proxy
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(bar_w_full + 8 * ws);
-        mbar_arrive(bar_raw_empty + 8 * rs);
-      }
-    }
-    // epilogue
-    if (ok && warp < 6 && nkb > 0) ok = mbar_wait(bar_acc, 0, error, 3, abort_slot);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok && warp < 6) {
+    if (nkb > 0) ok = mbar_wait(bar_acc, 0, error, 3, abort_slot);
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int n = m_tile * kBlockM + quad * 32 + lane;
-      const float sc = n < N ? __ldg(scale + n) : 0.f;
-      float* dstp = out + static_cast<long long>(split) * split_stride;
+      const float ws = n < N ? __ldg(wscale + n) : 0.f;
+      float* dst = out + static_cast<long long>(split) * split_stride;
       for (int c0 = 0; c0 < tn; c0 += 16) {
-        uint32_t v[16];
+        uint32_t vh[16], vl[16];
         if (nkb > 0) {
+          const uint32_t addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(c0);
           asm volatile(
               "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-              : "r"(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(c0)));
+              : "=r"(vh[0]), "=r"(vh[1]), "=r"(vh[2]), "=r"(vh[3]), "=r"(vh[4]), "=r"(vh[5]), "=r"(vh[6]), "=r"(vh[7]),
+                "=r"(vh[8]), "=r"(vh[9]), "=r"(vh[10]), "=r"(vh[11]), "=r"(vh[12]), "=r"(vh[13]), "=r"(vh[14]), "=r"(vh[15])
+              : "r"(addr));
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+              : "=r"(vl[0]), "=r"(vl[1]), "=r"(vl[2]), "=r"(vl[3]), "=r"(vl[4]), "=r"(vl[5]), "=r"(vl[6]), "=r"(vl[7]),
+                "=r"(vl[8]), "=r"(vl[9]), "=r"(vl[10]), "=r"(vl[11]), "=r"(vl[12]), "=r"(vl[13]), "=r"(vl[14]), "=r"(vl[15])
+              : "r"(addr + static_cast<uint32_t>(TN_MAX)));
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         } else {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) v[i] = 0u;
+          for (int i = 0; i < 16; ++i) vh[i] = vl[i] = 0u;
         }
         float val[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) val[i] = __uint_as_float(v[i]) * sc;
-        emit16(epi, dstp, N, T, n, t0 + c0, val);
+        for (int i = 0; i < 16; ++i) {
+          const int t = t0 + c0 + i;
+          const float as = t < T ? __ldg(ascale + t) : 0.f;
+          val[i] = (__uint_as_float(vh[i]) + __uint_as_float(vl[i])) * (ws * as);
+        }
+        emit16(epi, dst, N, T, n, t0 + c0, val);
       }
     }
   }
 
-  // teardown
   if (!ok) *abort_slot = 1;
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -529,14 +477,65 @@ __global__ void __launch_bounds__(kW8Threads) tc_gemm_w8_kernel(const uint8_t* _
   stamp_time(epi.stamp_end, true);
 }
 
-// row-major e4m3 bytes [N][K] -> tiles: block (m, kb) = four groups [128 rows][16 bytes], zero where the matrix ends
-__global__ void __launch_bounds__(256) retile_w8_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int N, int K,
+// One block per token: a[t][k] (bf16) -> s_t = max|a[t]| / 448, hi = e4m3(a / s_t), lo = e4m3(a / s_t - hi);
+// hi rows at out[t], lo rows at out[lo_row0 + t], s_t at scale[t].
+__global__ void __launch_bounds__(256) split_rows_f8_kernel(const __nv_bfloat16* __restrict__ a, int K, uint8_t* __restrict__ out,
+                                                            int lo_row0, float* __restrict__ scale,
+                                                            unsigned long long* stamp_begin, unsigned long long* stamp_end) {
+  __shared__ float red[8];
+  stamp_time(stamp_begin, false);
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  pdl_wait_here();
+  const int t = blockIdx.x;
+  const uint4* row = reinterpret_cast<const uint4*>(a + static_cast<long long>(t) * K);
+  float amax = 0.f;
+  for (int i = threadIdx.x; i < K / 8; i += blockDim.x) {
+    const uint4 v = row[i];
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      amax = fmaxf(amax, fabsf(__uint_as_float(w[j] << 16)));
+      amax = fmaxf(amax, fabsf(__uint_as_float(w[j] & 0xffff0000u)));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  amax = red[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) amax = fmaxf(amax, red[i]);
+  const float s = token_scale_e4m3(amax);
+  const float inv = 1.f / s;
+  if (threadIdx.x == 0) scale[t] = s;
+  uint2* hi = reinterpret_cast<uint2*>(out + static_cast<long long>(t) * K);
+  uint2* lo = reinterpret_cast<uint2*>(out + static_cast<long long>(lo_row0 + t) * K);
+  for (int i = threadIdx.x; i < K / 8; i += blockDim.x) {
+    const uint4 v = row[i];
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t h[2] = {0, 0}, l[2] = {0, 0};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t hq, lq;
+      split_pair_e4m3(__uint_as_float(w[j] << 16) * inv, __uint_as_float(w[j] & 0xffff0000u) * inv, hq, lq);
+      h[j >> 1] |= hq << (16 * (j & 1));
+      l[j >> 1] |= lq << (16 * (j & 1));
+    }
+    hi[i] = make_uint2(h[0], h[1]);
+    lo[i] = make_uint2(l[0], l[1]);
+  }
+  __syncthreads();
+  stamp_time(stamp_end, true);
+}
+
+// row-major e4m3 bytes [N][K] -> tiles of 128 rows x 128 bytes (k), zero where the matrix ends
+__global__ void __launch_bounds__(256) retile_f8_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int N, int K,
                                                         int n_kslabs) {
   const int kb = blockIdx.x, mt = blockIdx.y;
-  uint8_t* out = dst + (static_cast<long long>(mt) * n_kslabs + kb) * kW8StageBytes;
-  for (int i = threadIdx.x; i < kW8StageBytes; i += blockDim.x) {
-    const int c = i / (kBlockM * 16), r = (i / 16) % kBlockM, b = i % 16;
-    const int n = mt * kBlockM + r, k = kb * kBlockK + c * 16 + b;
+  uint8_t* out = dst + (static_cast<long long>(mt) * n_kslabs + kb) * (kBlockM * kBlockK8);
+  for (int i = threadIdx.x; i < kBlockM * kBlockK8; i += blockDim.x) {
+    const int r = i / kBlockK8, b = i % kBlockK8;
+    const int n = mt * kBlockM + r, k = kb * kBlockK8 + b;
     out[i] = (n < N && k < K) ? src[static_cast<long long>(n) * K + k] : static_cast<uint8_t>(0);
   }
 }
@@ -863,6 +862,24 @@ int make_map(CUtensorMap* map, const void* ptr, long long rows, int K, int box_r
   return 0;
 }
 
+// the same for an array of bytes: boxes of 128 bytes x box_rows rows
+int make_map_u8(CUtensorMap* map, const void* ptr, long long rows, int K, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return -1;
+  if (K % 16 || (reinterpret_cast<uintptr_t>(ptr) & 15)) return -1;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(K)};
+  cuuint32_t box[2] = {kBlockK8, static_cast<cuuint32_t>(box_rows)};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    std::fprintf(stderr, "sled: cuTensorMapEncodeTiled (bytes) failed (%d) rows=%lld K=%d box=%d\n", static_cast<int>(r), rows, K, box_rows);
+    return -1;
+  }
+  return 0;
+}
 
 }  // namespace
 
@@ -892,21 +909,52 @@ int tc_weight_init(TcWeight* w, const void* rowmajor, void* tiled, int N, int K)
   return 0;
 }
 
-size_t tc_weight_w8_tiled_bytes(int N, int K) {
-  return static_cast<size_t>((N + kBlockM - 1) / kBlockM) * ((K + kBlockK - 1) / kBlockK) * kW8StageBytes;
+size_t tc_weight_f8_tiled_bytes(int N, int K) {
+  return static_cast<size_t>((N + kBlockM - 1) / kBlockM) * ((K + kBlockK8 - 1) / kBlockK8) * kWStageBytes;
 }
 
-int tc_weight_init_w8(TcWeight* w, const void* rowmajor_bytes, void* tiled, const float* scale, int N, int K) {
-  if (K % 8 || !scale || (reinterpret_cast<uintptr_t>(tiled) & 15)) return -1;
-  const int n_mtiles = (N + kBlockM - 1) / kBlockM, n_kslabs = (K + kBlockK - 1) / kBlockK;
-  retile_w8_kernel<<<dim3(n_kslabs, n_mtiles), 256>>>(static_cast<const uint8_t*>(rowmajor_bytes), static_cast<uint8_t*>(tiled), N, K, n_kslabs);
+int tc_weight_init_f8(TcWeight* w, const void* rowmajor_bytes, void* tiled, const float* scale, int N, int K) {
+  if (K % 16 || !scale || (reinterpret_cast<uintptr_t>(tiled) & 15)) return -1;
+  const int n_mtiles = (N + kBlockM - 1) / kBlockM, n_kslabs = (K + kBlockK8 - 1) / kBlockK8;
+  retile_f8_kernel<<<dim3(n_kslabs, n_mtiles), 256>>>(static_cast<const uint8_t*>(rowmajor_bytes), static_cast<uint8_t*>(tiled), N, K, n_kslabs);
   if (cudaDeviceSynchronize() != cudaSuccess) return -1;
-  w->w8 = static_cast<const uint8_t*>(tiled);
+  if (make_map_u8(&w->map8, tiled, static_cast<long long>(n_mtiles) * n_kslabs * kBlockM, kBlockK8, kBlockM)) return -1;
   w->scale = scale;
   w->N = N;
   w->K = K;
+  w->f8 = true;
   w->ready = true;
   return 0;
+}
+
+int tc_activation8_init(TcActivation8* a, void* data, float* scale, int rows, int K) {
+  if (rows % 128 || K % 16 || !data || !scale) return -1;
+  const int boxes[4] = {32, 64, 96, 128};
+  for (int i = 0; i < 4; ++i)
+    if (make_map_u8(&a->map[i], data, 2LL * rows, K, boxes[i])) return -1;
+  a->data = static_cast<uint8_t*>(data);
+  a->scale = scale;
+  a->rows = rows;
+  a->K = K;
+  return 0;
+}
+
+int tc_split_rows_launch(const void* a_bf16, int T, const TcActivation8& dst, cudaStream_t s,
+                         unsigned long long* stamp_begin, unsigned long long* stamp_end) {
+  if (T <= 0) return 0;
+  if (T > dst.rows || (reinterpret_cast<uintptr_t>(a_bf16) & 15)) return -1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(T, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t err = cudaLaunchKernelEx(&cfg, split_rows_f8_kernel, static_cast<const __nv_bfloat16*>(a_bf16), dst.K, dst.data, dst.rows,
+                                       dst.scale, stamp_begin, stamp_end);
+  return err == cudaSuccess ? 1 : -1;
 }
 
 void tc_weight_free(TcWeight* w) { w->ready = false; }
@@ -953,32 +1001,33 @@ int tc_gemm_split(int T, int N, int K, int n_sm) {
   return (kb_total + kb_per - 1) / kb_per;
 }
 
-// 8-bit weights: one CTA per SM, so K slices fill n_sm slots; at least 4 slabs each
-int tc_gemm_split_w8(int T, int N, int K, int n_sm) {
-  const int tn = T <= kSingleTileMax ? T : 128;
-  const int tiles = ((N + kBlockM - 1) / kBlockM) * ((T + tn - 1) / tn);
-  const int kb_total = (K + kBlockK - 1) / kBlockK;
-  int s = std::max(1, n_sm / tiles);
-  s = std::min(s, std::max(1, kb_total / 4));
+// fp8 MMAs, 128-wide k-slabs: one weight tile per CTA and two CTAs per SM, as in the bf16 kernel
+int tc_gemm_split_f8(int T, int N, int K, int n_sm) {
+  const int tn = T <= 128 ? T : 128;
+  const int m_tiles = (N + kBlockM - 1) / kBlockM;
+  const int tiles = m_tiles * ((T + tn - 1) / tn);
+  const int kb_total = (K + kBlockK8 - 1) / kBlockK8;
+  int s = std::max(1, (2 * n_sm) / tiles);
+  s = std::min(s, std::max(1, kb_total / 2));
   s = std::min(s, 16);
   const int kb_per = (kb_total + s - 1) / s;
   return (kb_total + kb_per - 1) / kb_per;
 }
 
 template <int TN_MAX>
-static int launch_w8(const TcWeight& w, const CUtensorMap& ma, int T, int n_split, float* out, int64_t split_stride,
+static int launch_f8(const TcWeight& w, const TcActivation8& a, int box, int T, int n_split, float* out, int64_t split_stride,
                      int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
-  using L = W8SmemLayout<TN_MAX>;
+  using L = F8SmemLayout<TN_MAX>;
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(tc_gemm_w8_kernel<TN_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess) return -1;
+    if (cudaFuncSetAttribute(tc_gemm_f8_kernel<TN_MAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess) return -1;
     configured = true;
   }
-  const int kb_total = (w.K + kBlockK - 1) / kBlockK;
+  const int kb_total = (w.K + kBlockK8 - 1) / kBlockK8;
   const int kb_per = (kb_total + n_split - 1) / n_split;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((T + TN_MAX - 1) / TN_MAX, (w.N + kBlockM - 1) / kBlockM, n_split);
-  cfg.blockDim = dim3(kW8Threads, 1, 1);
+  cfg.blockDim = dim3(192, 1, 1);
   cfg.dynamicSmemBytes = L::kTotal;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
@@ -987,8 +1036,19 @@ static int launch_w8(const TcWeight& w, const CUtensorMap& ma, int T, int n_spli
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   const long long stride = split_stride;
-  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_w8_kernel<TN_MAX>, w.w8, w.scale, ma, T, w.N, kb_total, kb_per, out, stride, error, epi);
+  cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_f8_kernel<TN_MAX>, w.map8, a.map[box], T, w.N, kb_total, kb_per, a.rows, w.scale,
+                                       static_cast<const float*>(a.scale), out, stride, error, epi);
   return err == cudaSuccess ? 1 : -1;
+}
+
+int tc_gemm_f8_launch(const TcActivation8& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
+                      int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
+  if (!w.ready || !w.f8 || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
+  if (epi.mode != kEpiStore && n_split != 1) return -1;
+  if (T <= 32) return launch_f8<32>(w, a, 0, T, n_split, out, split_stride, error, epi, s);
+  if (T <= 64) return launch_f8<64>(w, a, 1, T, n_split, out, split_stride, error, epi, s);
+  if (T <= 96) return launch_f8<96>(w, a, 2, T, n_split, out, split_stride, error, epi, s);
+  return launch_f8<128>(w, a, 3, T, n_split, out, split_stride, error, epi, s);   // wider steps: 128-token tiles
 }
 
 template <int TN_MAX, int STAGES>
@@ -1059,14 +1119,7 @@ int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split,
                    int32_t* error, const TcEpilogue& epi, cudaStream_t s) {
   if (!w.ready || a.K != w.K || T <= 0 || T > a.rows || n_split < 1) return -1;
   if (epi.mode != kEpiStore && n_split != 1) return -1;   // a fused epilogue needs the complete sum
-  if (w.w8) {   // 8-bit weights: every step size on the converting kernel (wide steps as 128-token tiles)
-    if (T <= 32) return launch_w8<32>(w, a.map[0], T, n_split, out, split_stride, error, epi, s);
-    if (T <= 64) return launch_w8<64>(w, a.map[1], T, n_split, out, split_stride, error, epi, s);
-    if (T <= 96) return launch_w8<96>(w, a.map[2], T, n_split, out, split_stride, error, epi, s);
-    if (T <= 128) return launch_w8<128>(w, a.map[3], T, n_split, out, split_stride, error, epi, s);
-    if (T <= kSingleTileMax) return launch_w8<160>(w, a.map[4], T, n_split, out, split_stride, error, epi, s);
-    return launch_w8<128>(w, a.map[3], T, n_split, out, split_stride, error, epi, s);
-  }
+  if (w.f8) return -1;   // 8-bit weights go through tc_gemm_f8_launch
   // token tile = the smallest box that holds the step; what the narrower activation stage saves goes into ring depth
   if (T <= 32) return launch_split<32, 5>(w.map, a.map[0], T, w.N, w.K, n_split, out, split_stride, error, epi, s);
   if (T <= 64) return launch_split<64, 4>(w.map, a.map[1], T, w.N, w.K, n_split, out, split_stride, error, epi, s);

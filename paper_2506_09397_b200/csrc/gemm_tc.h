@@ -14,9 +14,19 @@ struct TcWeight {       // [N][K] bf16 weights, stored as 128 x 64 tiles of 16 K
   CUtensorMap map;      // over the tiled array seen as rows of 128 bytes; box = one tile, 128-byte swizzle
   int N = 0, K = 0;
   bool ready = false;
-  // 8-bit weights instead (tc_weight_init_w8): e4m3 bytes in 8 KB tiles and one fp32 scale per output row
-  const uint8_t* w8 = nullptr;
+  // 8-bit weights instead (tc_weight_init_f8): e4m3 bytes as 128 x 128 tiles of 16 KB behind map8 and one fp32 scale
+  // per output row
+  CUtensorMap map8;
   const float* scale = nullptr;
+  bool f8 = false;
+};
+
+struct TcActivation8 {  // an activation tensor as two e4m3 parts per element and one fp32 scale per token (see
+                        // tc_split_rows_launch): [2 * rows][K] bytes - hi rows first, lo rows from row `rows` on
+  CUtensorMap map[4];   // boxes of 128 (k) x {32, 64, 96, 128} rows
+  uint8_t* data = nullptr;
+  float* scale = nullptr;   // [rows]
+  int rows = 0, K = 0;
 };
 
 constexpr int kTokenTiles = 6;
@@ -42,16 +52,25 @@ int tma_map_bf16_rows(CUtensorMap* map, const void* dev_ptr, long long rows, int
 // needed afterwards.  Synchronises the device.
 size_t tc_weight_tiled_bytes(int N, int K);
 int tc_weight_init(TcWeight* w, const void* rowmajor, void* tiled, int N, int K);
-// The same for e4m3 bytes [N][K] (row-major, device) with `scale` [N] fp32 (device; must stay valid): W[n][k] =
-// scale[n] * e4m3(byte).  `tiled` holds tc_weight_w8_tiled_bytes(N, K) bytes.  The byte patterns 0x7f / 0xff (NaN in
-// e4m3) must not occur.
-size_t tc_weight_w8_tiled_bytes(int N, int K);
-int tc_weight_init_w8(TcWeight* w, const void* rowmajor_bytes, void* tiled, const float* scale, int N, int K);
+// The same for e4m3 bytes [N][K] (row-major, device; K a multiple of 16) with `scale` [N] fp32 (device; must stay
+// valid): W[n][k] = scale[n] * e4m3(byte).  `tiled` holds tc_weight_f8_tiled_bytes(N, K) bytes.  The byte patterns
+// 0x7f / 0xff (NaN in e4m3) must not occur.
+size_t tc_weight_f8_tiled_bytes(int N, int K);
+int tc_weight_init_f8(TcWeight* w, const void* rowmajor_bytes, void* tiled, const float* scale, int N, int K);
+// `data`: 2 * rows * K bytes, `scale`: rows floats (device, zero-initialised by the caller); rows a multiple of 128
+int tc_activation8_init(TcActivation8* a, void* data, float* scale, int rows, int K);
+// a[T][K] bf16 (device) -> the two e4m3 parts and the token scales of `dst`; returns kernels launched or < 0
+int tc_split_rows_launch(const void* a_bf16, int T, const TcActivation8& dst, cudaStream_t s,
+                         unsigned long long* stamp_begin, unsigned long long* stamp_end);
+int tc_gemm_split_f8(int T, int N, int K, int n_sm);
+// out[slice][T][N] = scale_t * scale_n * (hi + lo)[T][K slice] . W8[N][K slice]^T
+int tc_gemm_f8_launch(const TcActivation8& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,
+                      int32_t* error, const TcEpilogue& epi, cudaStream_t s);
 void tc_weight_free(TcWeight* w);
 int tc_activation_init(TcActivation* a, const void* dev_ptr, int rows, int K);
-// number of partial-sum slices [slice][T][N] a launch leaves behind for this shape (bf16 weights / 8-bit weights)
+// number of partial-sum slices [slice][T][N] a launch leaves behind for this shape (bf16 weights; tc_gemm_split_f8:
+// 8-bit weights)
 int tc_gemm_split(int T, int N, int K, int n_sm);
-int tc_gemm_split_w8(int T, int N, int K, int n_sm);
 // out[slice][T][N] = A[T][K slice] . W[N][K slice]^T; returns kernels launched (1) or a negative value;
 // `error` is a device word set if a bounded wait ran out
 int tc_gemm_launch(const TcActivation& a, const TcWeight& w, int T, int n_split, float* out, int64_t split_stride,

@@ -20,8 +20,11 @@ struct Stamp {
 int launch_embed(const void* table, int wdtype, const int32_t* ids, int T, int d, float* x, cudaStream_t s,
                  Stamp st = Stamp());
 // x += sum_s partial[s] (if partial), then out = RMSNorm(x) * gain in the activation type
+// out8 / lo_row0 / scale8 (optional, bf16 only): the outputs once more as two e4m3 parts per element and a scale per
+// token, where the kernel can do it (*split_done tells)
 int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t split_stride, const void* gain, int wdtype,
-                       float eps, int T, int d, void* out, int adtype, cudaStream_t s, Stamp st = Stamp());
+                       float eps, int T, int d, void* out, int adtype, cudaStream_t s, Stamp st = Stamp(),
+                       uint8_t* out8 = nullptr, int lo_row0 = 0, float* scale8 = nullptr, bool* split_done = nullptr);
 int launch_rope_table(const int32_t* tok_pos, int T, int h, float theta, float2* cs, cudaStream_t s, Stamp st = Stamp());
 // sums the QKV partials, rotates Q and K, writes Q to q_out and K, V into their cache slots
 int launch_rope_kv(const float* partial, int n_split, int64_t split_stride, const float2* cs, const int32_t* tok_slot,

@@ -4,6 +4,7 @@
 // The linear layers leave split-K partial sums behind; the kernel that consumes a
 // linear layer's output adds them up, in a fixed order, while it does its own work.
 #include "common.cuh"
+#include "fp8_split.cuh"
 #include "kernels.h"
 
 namespace sled {
@@ -65,8 +66,66 @@ __global__ void add_rmsnorm_kernel(float* __restrict__ x, const float* __restric
   }
 }
 
+// The same with bf16 gains and outputs for rows of at most four features per thread, which stay in registers, and
+// the outputs written a second time as two e4m3 parts per element plus the token's scale (the operand format of the
+// fp8 linear layers): hi rows at out8[t], lo rows at out8[lo_row0 + t].
+__global__ void add_rmsnorm_split_kernel(float* __restrict__ x, const float* __restrict__ partial, int n_split,
+                                         int64_t split_stride, const __nv_bfloat16* __restrict__ gain, float eps, int d,
+                                         __nv_bfloat16* __restrict__ out, uint8_t* __restrict__ out8, int lo_row0,
+                                         float* __restrict__ scale8, LaunchStamp stamp) {
+  __shared__ float scratch[32];
+  StampScope scope(stamp);
+  pdl_enter();
+  const int64_t base = static_cast<int64_t>(blockIdx.x) * d;
+  const int i = threadIdx.x * 4;
+  const bool mine = i < d;
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (mine) {
+    v = *reinterpret_cast<const float4*>(x + base + i);
+#pragma unroll 8
+    for (int sp = 0; sp < n_split; ++sp) {
+      const float4 p = __ldcg(reinterpret_cast<const float4*>(partial + sp * split_stride + base + i));
+      v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+    }
+    if (n_split > 0) *reinterpret_cast<float4*>(x + base + i) = v;
+  }
+  const float ss = block_sum(v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w, scratch);
+  const float scale = rsqrtf(ss / static_cast<float>(d) + eps);
+  float y[4] = {0.f, 0.f, 0.f, 0.f};
+  if (mine) {
+    const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const __nv_bfloat16 r = __float2bfloat16_rn(vv[j] * scale * __bfloat162float(gain[i + j]));
+      out[base + i + j] = r;
+      y[j] = __bfloat162float(r);
+    }
+  }
+  // the row's largest output: a maximum is a sum in the (max, +) sense, and exact in any order
+  float amax = fmaxf(fmaxf(fabsf(y[0]), fabsf(y[1])), fmaxf(fabsf(y[2]), fabsf(y[3])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  amax = 0.f;
+  for (int w = 0; w < (blockDim.x + 31) / 32; ++w) amax = fmaxf(amax, scratch[w]);
+  const float s8 = token_scale_e4m3(amax);
+  const float inv = 1.f / s8;
+  if (threadIdx.x == 0) scale8[blockIdx.x] = s8;
+  if (mine) {
+    uint32_t h0, l0, h1, l1;
+    split_pair_e4m3(y[0] * inv, y[1] * inv, h0, l0);
+    split_pair_e4m3(y[2] * inv, y[3] * inv, h1, l1);
+    *reinterpret_cast<uint32_t*>(out8 + static_cast<int64_t>(blockIdx.x) * d + i) = h0 | (h1 << 16);
+    *reinterpret_cast<uint32_t*>(out8 + static_cast<int64_t>(lo_row0 + blockIdx.x) * d + i) = l0 | (l1 << 16);
+  }
+}
+
 int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t split_stride, const void* gain, int wdtype,
-                       float eps, int T, int d, void* out, int adtype, cudaStream_t s, Stamp st) {
+                       float eps, int T, int d, void* out, int adtype, cudaStream_t s, Stamp st, uint8_t* out8, int lo_row0,
+                       float* scale8, bool* split_done) {
+  if (split_done) *split_done = false;
   if (T <= 0) return 0;
   if (!partial) n_split = 0;
   int nt = d >= 4096 ? 1024 : (d >= 2048 ? 512 : 256);   // d is a multiple of 8 (checked at init)
@@ -79,6 +138,12 @@ int launch_add_rmsnorm(float* x, const float* partial, int n_split, int64_t spli
     n_sm = (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess) ? prop.multiProcessorCount : 1;
   }
   while (nt > 128 && static_cast<long long>(T) * nt > 2048LL * n_sm) nt /= 2;
+  if (out8 && scale8 && wdtype == BF16 && adtype == BF16 && d <= 4 * nt && d % 4 == 0) {
+    SLED_LAUNCH_PDL(add_rmsnorm_split_kernel, dim3(T), dim3(nt), 0, s, x, partial, n_split, split_stride,
+                    static_cast<const __nv_bfloat16*>(gain), eps, d, static_cast<__nv_bfloat16*>(out), out8, lo_row0, scale8, dev_stamp(st));
+    if (split_done) *split_done = true;
+    return 1;
+  }
   if (wdtype == BF16 && adtype == BF16)
     SLED_LAUNCH_PDL((add_rmsnorm_kernel<__nv_bfloat16, __nv_bfloat16>), dim3(T), dim3(nt), 0, s, x, partial, n_split,
                     split_stride, static_cast<const __nv_bfloat16*>(gain), eps, d, static_cast<__nv_bfloat16*>(out), dev_stamp(st));

@@ -1,7 +1,7 @@
-"""The 8-bit weight path (linear_weight_bits = 8: e4m3 bytes with one fp32 scale per output row, bf16 activations)
-against the oracle run on the matrices those bytes stand for.  Nothing is quantised on the device: both sides are
-given the same bytes and scales, so the comparison is the bf16 path's (inputs of every product rounded to bf16, fp32
-sums), with the same tolerance."""
+"""The 8-bit weight path (linear_weight_bits = 8: e4m3 bytes with one fp32 scale per output row) against the oracle
+run on the matrices those bytes stand for.  No weight is quantised on the device: both sides are given the same bytes
+and scales.  The device feeds its bf16 activations to fp8 MMAs as two e4m3 parts per element (eight significant
+bits, like bf16) and sums in fp32, so the comparison is the bf16 path's, with the same tolerance."""
 import dataclasses
 
 import numpy as np
