@@ -507,8 +507,8 @@ def run_sled(args):
     dev = f"cuda:{local_rank}"
     peaks, peak_src = load_peaks()
     w = I.make_weights(shape, seed, device=dev)
+    global WEIGHT_BITS
     if args.weight_bits == 8:
-        global WEIGHT_BITS
         WEIGHT_BITS = 8
         args.no_cpu_baseline = True          # the oracle arm is timed on the 16-bit workload
         w, _ = I.quantize_linear_weights(w, dequantised=False)
@@ -623,6 +623,33 @@ def run_sled(args):
             del dh, qd, rq
             sp.close()
         line["sweep"] = sweep
+
+    # ---- the same step with 8-bit weights in the linear layers (the paper sweeps 16-, 8- and 4-bit precision)
+    if not args.no_sweep and world == 1 and args.weight_bits == 16 and shape.weight_dtype == "bf16":
+        w8, _ = I.quantize_linear_weights(w, dequantised=False)
+        args8 = argparse.Namespace(**{**vars(args), "weight_bits": 8})
+        WEIGHT_BITS = 8
+        rows = []
+        for b in sorted({args.batch, 1}, reverse=True):
+            sp = Point(B, args8, shape, w8, b, rank, local_rank, world, stream)
+            dh, qd = sp.correlated_drafts() if correlated else sp.independent_drafts()
+            torch.cuda.synchronize()
+            rq = sp.marshal(dh, qd)
+            n_steps = max(5, args.steps // 2)
+            c_s, ms_s, _ = sp.timed(rq, n_steps, 3)
+            km_s, n_lin_s, n_rej_s = sp.kernel_times(rq, 1, steps=3)
+            entry = {"batch": b, "tokens_scored_per_step": sp.T, "steps": n_steps, "workload": sp.name}
+            entry.update(sp.summary(c_s, ms_s, n_steps, n_rej_s, peaks))
+            entry["kernel_ms"] = km_s
+            r = sp.linear_roofline(km_s, n_lin_s, peaks, peak_src)
+            entry["linear_layers"] = {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac") if k in r}
+            rows.append(entry)
+            del dh, qd, rq
+            sp.close()
+        WEIGHT_BITS = 16
+        line["weights_8bit"] = {"format": "e4m3 bytes + one fp32 scale per output row; fp8 MMAs on activations split into "
+                                          "two e4m3 parts; bytes counted with one byte per weight", "points": rows}
+        del w8
     del w
     torch.cuda.empty_cache()
 
