@@ -768,6 +768,8 @@ def run_serve(args):
     counts = [int(x) for x in args.devices.split(",") if x]
     max_k, V = 8, shape.vocab
     w = I.make_weights(shape, args.seed, device=dev)
+    if args.weight_bits == 8:
+        w, _ = I.quantize_linear_weights(w, dequantised=False)
     stream = torch.cuda.Stream(device=dev)
     n_max = max(counts)
     ctx_len = I.draw_context_lengths(n_max, 128, 512, args.seed)
@@ -776,7 +778,8 @@ def run_serve(args):
     n_pages = max(sum((c + 4 * rounds_for(n) * (max_k + 1) + 16 + 15) // 16 for c in ctx_len[:n]) for n in counts) + 64
     max_batch = min(args.max_batch, n_max)
     eng = B.Engine(shape, w, n_pages=n_pages, max_batch=max_batch, max_k=max_k, max_step_tokens=max_batch * (max_k + 1),
-                   temperature=1.0, greedy=False, device_index=0, stream=stream.cuda_stream, probs_on_device=True)
+                   temperature=1.0, greedy=False, device_index=0, stream=stream.cuda_stream, probs_on_device=True,
+                   linear_weight_bits=args.weight_bits)
     del w
     eng.server_config(B.SLED_BATCH_STATIC if args.policy == "static" else B.SLED_BATCH_CONTINUOUS,
                       min(args.static_batch, max_batch))
@@ -881,7 +884,8 @@ def run_serve(args):
                                              f"devices drafting {args.draft_rate} tokens/s, c_th={args.c_th}, max_k={max_k}, "
                                              f"contexts 128..512, about {args.rounds} verification rounds per device simulated "
                                              "(more for small populations; the first quarter of the time is not counted)",
-                                 "draft_distributions": "independent of the target (softmax of N(0,1) logits)"},
+                                 "draft_distributions": "independent of the target (softmax of N(0,1) logits)",
+                                 "linear_weight_bits": args.weight_bits},
                       "capacity_devices": {"value": max(ok) if ok else 0, "rule": "largest simulated count whose devices still get >= 90 % of "
                                            "the token rate of the smallest population's", "reached_largest_simulated": bool(ok) and max(ok) == max(counts)},
                       "by_devices": out}))
