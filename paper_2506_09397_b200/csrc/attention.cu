@@ -10,6 +10,7 @@
 // This file holds the CUDA-core kernel (any storage type, used by the fp32
 // configuration) and the merge kernel.
 #include "common.cuh"
+#include "fp8_split.cuh"
 #include "kernels.h"
 
 namespace sled {
@@ -188,6 +189,61 @@ __global__ void attn_merge_kernel(AttnArgs a) {
   static_cast<AT*>(a.out)[(static_cast<int64_t>(t) * a.Hq + head) * a.h + i] = from_f32<AT>(num / den);
 }
 
+// The merge and the split in one launch (bf16 outputs; one block per token, four consecutive elements of the token's
+// [Hq][h] row per thread): a token of a split request has its chunks merged exactly as attn_merge_kernel does, any
+// other token's output is read back; then the row maximum, the token's scale, and the two e4m3 parts.
+__global__ void attn_merge_split_kernel(AttnArgs a) {
+  __shared__ float red[32];
+  StampScope scope(LaunchStamp{a.stamp_merge.begin, a.stamp_merge.end});
+  pdl_enter();
+  const int t = blockIdx.x, e0 = threadIdx.x * 4, head = e0 / a.h, i = e0 % a.h;
+  const int row_len = a.Hq * a.h;
+  __nv_bfloat16* orow = static_cast<__nv_bfloat16*>(a.out) + static_cast<int64_t>(t) * row_len;
+  const int n = a.part_acc ? a.req_chunks[a.tok_req[t]] : 1;
+  float y[4];
+  if (n <= 1) {
+    const uint2 v = *reinterpret_cast<const uint2*>(orow + e0);
+    y[0] = __uint_as_float(v.x << 16); y[1] = __uint_as_float(v.x & 0xffff0000u);
+    y[2] = __uint_as_float(v.y << 16); y[3] = __uint_as_float(v.y & 0xffff0000u);
+  } else {
+    const int64_t first = static_cast<int64_t>(a.tok_part[t]);
+    float M = -INFINITY;
+    for (int c = 0; c < n; ++c) M = fmaxf(M, a.part_ml[((first + c) * a.Hq + head) * 2]);
+    float num[4] = {0.f, 0.f, 0.f, 0.f}, den = 0.f;
+    for (int c = 0; c < n; ++c) {
+      const int64_t prow = (first + c) * a.Hq + head;
+      const float mc = a.part_ml[prow * 2];
+      if (mc == -INFINITY) continue;  // this chunk held no visible key
+      const float w = exp2f(mc - M);
+      den = fmaf(w, a.part_ml[prow * 2 + 1], den);
+      const float4 acc = *reinterpret_cast<const float4*>(a.part_acc + prow * a.h + i);
+      num[0] = fmaf(w, acc.x, num[0]); num[1] = fmaf(w, acc.y, num[1]);
+      num[2] = fmaf(w, acc.z, num[2]); num[3] = fmaf(w, acc.w, num[3]);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const __nv_bfloat16 r = __float2bfloat16_rn(num[j] / den);
+      orow[e0 + j] = r;
+      y[j] = __bfloat162float(r);
+    }
+  }
+  float amax = fmaxf(fmaxf(fabsf(y[0]), fabsf(y[1])), fmaxf(fabsf(y[2]), fabsf(y[3])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  amax = 0.f;
+  for (int w = 0; w < (blockDim.x + 31) / 32; ++w) amax = fmaxf(amax, red[w]);
+  const float s8 = token_scale_e4m3(amax);
+  const float inv = 1.f / s8;
+  if (threadIdx.x == 0) a.out8_scale[t] = s8;
+  uint32_t h0, l0, h1, l1;
+  split_pair_e4m3(y[0] * inv, y[1] * inv, h0, l0);
+  split_pair_e4m3(y[2] * inv, y[3] * inv, h1, l1);
+  *reinterpret_cast<uint32_t*>(a.out8 + static_cast<int64_t>(t) * row_len + e0) = h0 | (h1 << 16);
+  *reinterpret_cast<uint32_t*>(a.out8 + static_cast<int64_t>(a.out8_lo_row0 + t) * row_len + e0) = l0 | (l1 << 16);
+}
+
 template <typename KT, typename AT>
 int launch_typed(const AttnArgs& a, cudaStream_t s) {
   if (a.h == 64)
@@ -203,7 +259,8 @@ int launch_typed(const AttnArgs& a, cudaStream_t s) {
 
 }  // namespace
 
-int launch_attention(const AttnArgs& a, cudaStream_t s) {
+int launch_attention(const AttnArgs& a, cudaStream_t s, bool* split_done) {
+  if (split_done) *split_done = false;
   if (a.n_items <= 0 || a.T <= 0) return 0;
   int n = -1;
   if (a.use_tc && a.kvdtype == BF16 && a.adtype == BF16 && a.map_k && a.page_size == 16 && a.h == 128)
@@ -214,6 +271,12 @@ int launch_attention(const AttnArgs& a, cudaStream_t s) {
   else if (a.kvdtype == F32 && a.adtype == F32) n = launch_typed<float, float>(a, s);
   else if (a.kvdtype == BF16 && a.adtype == F32) n = launch_typed<__nv_bfloat16, float>(a, s);
   if (n < 0) return n;
+  const int row_len = a.Hq * a.h;
+  if (a.out8 && a.out8_scale && a.adtype == BF16 && a.h % 4 == 0 && row_len / 4 <= 1024 && (row_len / 4) % 32 == 0) {
+    SLED_LAUNCH_PDL(attn_merge_split_kernel, dim3(a.T), dim3(row_len / 4), 0, s, a);
+    if (split_done) *split_done = true;
+    return n + 1;
+  }
   if (a.part_acc) {  // some request was split
     dim3 grid(a.T, a.Hq);
     if (a.adtype == BF16) SLED_LAUNCH_PDL(attn_merge_kernel<__nv_bfloat16>, grid, dim3(a.h), 0, s, a);

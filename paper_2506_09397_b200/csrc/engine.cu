@@ -95,6 +95,7 @@ struct sled_engine {
   TcActivation tc_norm, tc_attn, tc_ffn;
   TcActivation8 a8_norm, a8_attn, a8_ffn;   // 8-bit weights: the same activations as two e4m3 parts + token scales
   bool norm_split = false;                  // the normalisation kernel has filled a8_norm for the act_norm now in place
+  bool attn_split = false;                  // the same for a8_attn and the attention output
   int32_t* tc_error = nullptr;  // device word set by a kernel whose bounded wait ran out: the first word of the
                                 // results block (d_results), so the step's one result copy brings it along
 
@@ -203,7 +204,7 @@ int run_linear(sled_engine* e, const void* A, const TcActivation* tcA, const Lin
   const TcActivation8* a8 = nullptr;
   if (L.tc.f8) {   // fp8 MMAs: the input goes in as two e4m3 parts per element and a scale per token
     a8 = tcA == &e->tc_norm ? &e->a8_norm : tcA == &e->tc_attn ? &e->a8_attn : &e->a8_ffn;
-    if (!(a8 == &e->a8_norm && e->norm_split)) {
+    if (!(a8 == &e->a8_norm && e->norm_split) && !(a8 == &e->a8_attn && e->attn_split)) {
       e->mark(K_OTHER);
       const Stamp ss = e->stamp(K_OTHER);
       const int ns = tc_split_rows_launch(A, T, *a8, e->stream, ss.begin, ss.end);
@@ -469,7 +470,13 @@ int run_forward(sled_engine* e, const Packed& pk, bool need_logits) {
     if (n < 0) return SLED_ERR_DEVICE;
     e->count(n, K_OTHER);
     e->mark(K_ATTN);
-    n = launch_attention(attn_args(e, pk, l, e->q_buf, e->attn_out), e->stream);
+    AttnArgs aa = attn_args(e, pk, l, e->q_buf, e->attn_out);
+    if (f8) {   // fp8 linear layers: the merge kernel also writes the attention output as two e4m3 parts per element
+      aa.out8 = e->a8_attn.data;
+      aa.out8_lo_row0 = e->a8_attn.rows;
+      aa.out8_scale = e->a8_attn.scale;
+    }
+    n = launch_attention(aa, e->stream, &e->attn_split);
     if (n < 0) return SLED_ERR_DEVICE;
     e->count(n, K_ATTN);
     rc = run_linear(e, e->attn_out, &e->tc_attn, L.o, T, nullptr, &split);

@@ -69,8 +69,14 @@ struct AttnArgs {
   int32_t* error = nullptr;
   Stamp stamp, stamp_merge;   // of the attention kernel and of the merge kernel that may follow it
   int use_tc = 0;             // 1: every item has at most 48 query rows and head_dim is 128: the tcgen05 kernel runs
+  // optional (bf16 activations): the output once more as two e4m3 parts per element and a scale per token, the
+  // operand format of the fp8 linear layers - hi rows at out8[t], lo rows at out8[out8_lo_row0 + t]
+  uint8_t* out8 = nullptr;
+  int out8_lo_row0 = 0;
+  float* out8_scale = nullptr;
 };
-int launch_attention(const AttnArgs& a, cudaStream_t s);
+// *split_done (optional) tells whether out8 / out8_scale were written
+int launch_attention(const AttnArgs& a, cudaStream_t s, bool* split_done = nullptr);
 // warp-level tensor-core kernel alone (attention_mma.cu); returns 1 or a negative value
 int launch_attention_mma(const AttnArgs& a, cudaStream_t s);
 // tcgen05 kernel alone (attention_tc.cu): head_dim 128, at most 48 query rows per item; returns 1 or a negative value
