@@ -292,8 +292,9 @@ __global__ void __launch_bounds__(192) tc_gemm_split_kernel(const __grid_constan
 // Linear layer with 8-bit weights, fp8 MMAs (tcgen05 kind::f8f6f4): nothing is converted on the way to the tensor
 // cores.  The instruction wants both operands in 8 (or fewer) bits, so the bf16 activations are handed over as TWO
 // e4m3 numbers each, a = s_t * (hi + lo) with hi = e4m3(a / s_t), lo = e4m3(a / s_t - hi) and one scale s_t per
-// token (split_rows_f8_kernel, run once per activation tensor): the products W * hi and W * lo are exact in the
-// fp32 accumulators, so the sum carries eight significant bits of every activation, as bf16 does.  Per k-slab
+// token (written by the kernel that produces the activation, or by split_rows_f8_kernel): every product of two
+// e4m3 numbers is exact and is added in fp32, so the sum carries eight significant bits of every activation, as
+// with a bf16 operand.  Per k-slab
 // (128 k = one 128-byte swizzle row) a CTA streams a 16 KB weight tile - the same bytes per slab as the bf16 kernel,
 // twice the reduction length - and fetches the token tile's hi rows and lo rows into one stage; one MMA per 32-k
 // step takes the whole stage as its N side (N = 2 x token tile), so W * hi and W * lo land side by side in tensor
