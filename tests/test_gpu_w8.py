@@ -63,12 +63,13 @@ def test_every_byte_pattern_is_decoded():
     eng.shutdown()
 
 
-@pytest.mark.parametrize("n_req,k", [(4, 4), (16, 8), (40, 8)])
-def test_steps_with_8bit_weights_match_the_oracle(n_req, k):
+@pytest.mark.parametrize("n_req,k,attention_impl", [(4, 4, 0), (16, 8, 0), (40, 8, 0), (5, 8, 1)])
+def test_steps_with_8bit_weights_match_the_oracle(n_req, k, attention_impl):
     # narrow and wide steps (20, 144 and 360 tokens: token tiles of 32, 160 and 3 x 128), prefill in chunks, commit
     shape = I.SMALL_GQA
     w = I.make_weights(shape, seed=5)
-    eng, orc = _both_sides(shape, w, n_pages=4 * n_req + 32, max_batch=n_req, max_k=8, max_step_tokens=max(n_req * (k + 1), 64))
+    eng, orc = _both_sides(shape, w, n_pages=4 * n_req + 32, max_batch=n_req, max_k=8, max_step_tokens=max(n_req * (k + 1), 64),
+                           attention_impl=attention_impl)   # 1: the tcgen05 attention kernel in front of the merge + split
     checked = sorted({0, n_req // 2, n_req - 1})
     for c in range(n_req):
         p = I.make_prompt(shape.vocab, 3 + (5 * c) % 31, 5, c)
