@@ -79,7 +79,7 @@ def parse_args(argv=None):
                     help="8: the linear layers' weights as e4m3 bytes with one scale per output row (step workload)")
     ap.add_argument("--attention-impl", type=int, default=0, choices=[0, 1],
                     help="0: warp-level tensor-core attention kernel (default), 1: the tcgen05 kernel (head_dim 128)")
-    ap.add_argument("--sweep", default="1,64,128", help="other batch sizes measured after the headline one")
+    ap.add_argument("--sweep", default="1,8,32,64,128", help="other batch sizes measured after the headline one")
     ap.add_argument("--no-sweep", action="store_true")
     return ap.parse_args(argv)
 
