@@ -3,7 +3,8 @@
 synthetic device requests, commit / rollback included).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-                    [--shape llama8b] [--batch 16] [--layers L] [--greedy]
+                    [--shape llama8b] [--batch 16] [--layers L] [--greedy] [--weight-bits 8]
+                    [--workload step|accept|attention|serve]
 
 Prints ONE JSON line.  Metric: verified (committed) tokens per second at the Llama-3-8B shape.
 `value` is measured with the draft distributions already in device memory, `e2e` with them in
@@ -12,7 +13,8 @@ distributions correlated with the target's own logits (`--drafts independent`: f
 that ignore the target).  `roofline` is for the tensor-core linear-layer kernel, the dominant one;
 `kernel_ms` splits an untouched step by kind of kernel from per-launch device timestamps,
 `kernel_ms_serialised` is the same with events between the kernels.  `sweep` repeats the step at
-other batch sizes (fewer steps, no end-to-end leg).  `--impl reference` times the CPU oracle.
+other batch sizes (fewer steps, no end-to-end leg), `weights_8bit` with the linear layers' weights as e4m3
+bytes (`--weight-bits 8` runs everything that way).  `--impl reference` times the CPU oracle.
 Under torchrun every rank runs its own replica on its own requests (no data-path collective).
 """
 from __future__ import annotations
