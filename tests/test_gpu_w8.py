@@ -89,6 +89,26 @@ def test_steps_with_8bit_weights_match_the_oracle(n_req, k, attention_impl):
     eng.shutdown()
 
 
+def test_8bit_weights_with_ragged_matrix_shapes():
+    # inner sizes that are not multiples of the 128-wide k-slab (320 = 2.5 slabs, 784 = 6.125) and row counts that are
+    # not multiples of the 128-row weight tile (960, 320, 1568, 4200): the last slab and the last tile are partly empty
+    shape = I.ModelShape("odd_w8", 2, 320, 5, 5, 64, 784, 4200, 5e5, "bf16", "bf16")
+    w = I.make_weights(shape, seed=7)
+    eng, orc = _both_sides(shape, w, n_pages=200, max_batch=12, max_k=8, max_step_tokens=108)
+    for c in range(12):
+        p = I.make_prompt(shape.vocab, 2 + (5 * c) % 23, 7, c)
+        eng.prefill(c, p)
+        if c % 4 == 0:
+            orc.prefill(c, p)
+    explain = []
+    reqs = [(c,) + tuple(I.make_drafts(shape.vocab, 5 + c % 4, 7, c)) for c in range(12)]
+    eng.set_commit(False)
+    eng.verify_batch([(c, d.numpy(), q.numpy()) for c, d, q in reqs], 1)
+    eng.set_commit(True)
+    _verify_both(eng, orc, [r for r in reqs if r[0] % 4 == 0], seed=1, tau=1.0, greedy=False, tol=TOL["bf16"], explain=explain)
+    eng.shutdown()
+
+
 def test_8bit_weights_need_scales_and_bf16():
     shape = I.SMALL_GQA
     w = I.make_weights(shape, seed=5)
