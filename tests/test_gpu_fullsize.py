@@ -132,6 +132,11 @@ def test_llama8b_shapes_two_layers_8bit_weights():
     ks = I.draw_k(64, [3, 5, 8], 1)
     ctx = I.draw_context_lengths(64, 512, 4096, 1)
     _full_step(shape, 64, ks, ctx, 1, check=_pick(ks, ctx, 2), weight_bits=8, gpu_vs_exact=W8_VS_EXACT, gpu_vs_rounded=W8_VS_ROUNDED)
+    # the 1B layer shapes (head_dim 64, 2048-wide rows: the normalisation writes the e4m3 parts with 512 threads)
+    shape = replace(I.LLAMA_1B, n_layers=2)
+    ks = I.draw_k(16, list(range(2, 9)), 2)
+    ctx = I.draw_context_lengths(16, 256, 2048, 2)
+    _full_step(shape, 16, ks, ctx, 2, check=_pick(ks, ctx, 2), weight_bits=8, gpu_vs_exact=W8_VS_EXACT, gpu_vs_rounded=W8_VS_ROUNDED)
 
 
 def test_llama8b_step_batch16():
