@@ -1,6 +1,6 @@
 // Fused vocabulary softmax + speculative acceptance + corrective / bonus draw.
 //
-// One block (or, for small batches, one thread-block cluster) per request walks its rows in
+// One thread-block cluster per request walks its rows in
 // order and stops at the deciding row: rows behind the first rejection are never read.  All quantities that decide anything are
 // order-independent: the row maximum, integer softmax numerators E_v (a fixed sequence
 // of correctly rounded fp32 operations followed by an exact scaling to 2^40), their
@@ -13,8 +13,7 @@ namespace sled {
 
 namespace {
 
-constexpr int kVec = 4;                       // consecutive vocabulary entries per thread per tile
-constexpr int kMaxTiles = 1024;               // vocabularies up to 4M entries
+constexpr int kVec = 4;                       // consecutive vocabulary entries per lane and step
 
 enum { ST_OK = 0, ST_NONFINITE = -8 };
 
@@ -105,8 +104,8 @@ __device__ __forceinline__ Exp2Consts exp2_consts(float inv_tau, float m) {
   c.one = pack2(1.0f, 1.0f);
   return c;
 }
-__device__ __forceinline__ void fixed_exp_pair(float z0, float z1, const Exp2Consts& c, unsigned long long& e0,
-                                               unsigned long long& e1) {
+// the two scaled numerators as floats (zero below the cut-off); their truncation is the integer numerator
+__device__ __forceinline__ void fixed_exp_pair_f(float z0, float z1, const Exp2Consts& c, float& s0, float& s1) {
   const unsigned long long x = add2(mul2(pack2(z0, z1), c.inv_tau), c.neg_m);   // a - m == a + (-m), rounded once
   const unsigned long long t = fma2(x, c.log2e, c.shift);
   const unsigned long long nf = add2(t, c.neg_shift);
@@ -124,10 +123,17 @@ __device__ __forceinline__ void fixed_exp_pair(float z0, float z1, const Exp2Con
   unpack2(p, p0, p1);
   // bits(t) - bits(1.5 * 2^23) = n; scaled = p * 2^(n + 40) by adding (n + 40) to p's exponent field
   const uint32_t base = 0x4B400000u - 40u;
-  const float s0 = __uint_as_float(__float_as_uint(p0) + ((__float_as_uint(t0) - base) << 23));
-  const float s1 = __uint_as_float(__float_as_uint(p1) + ((__float_as_uint(t1) - base) << 23));
-  e0 = __float2ull_rz(x0 >= -30.0f ? s0 : 0.0f);
-  e1 = __float2ull_rz(x1 >= -30.0f ? s1 : 0.0f);
+  const float f0 = __uint_as_float(__float_as_uint(p0) + ((__float_as_uint(t0) - base) << 23));
+  const float f1 = __uint_as_float(__float_as_uint(p1) + ((__float_as_uint(t1) - base) << 23));
+  s0 = x0 >= -30.0f ? f0 : 0.0f;
+  s1 = x1 >= -30.0f ? f1 : 0.0f;
+}
+__device__ __forceinline__ void fixed_exp_pair(float z0, float z1, const Exp2Consts& c, unsigned long long& e0,
+                                               unsigned long long& e1) {
+  float s0, s1;
+  fixed_exp_pair_f(z0, z1, c, s0, s1);
+  e0 = __float2ull_rz(s0);
+  e1 = __float2ull_rz(s1);
 }
 
 __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
@@ -149,11 +155,12 @@ __device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v
 }
 
 constexpr int kMaxCluster = 8;
+constexpr int kCacheBytes = 64 * 1024;        // a block's share of a row kept in shared memory (cached form)
+constexpr int kStep = 32 * kVec;              // entries a warp covers per step (512 contiguous bytes of fp32)
 
 struct Shared {
   unsigned long long sum_scratch[32];
-  unsigned long long tile_sum[kMaxTiles];
-  unsigned long long warp_pref[32];
+  unsigned long long warp_tot[32];            // deciding row: sum of the weights in each warp's range
   // exchange slots, one per CTA of the cluster (written by every CTA into every CTA's copy)
   unsigned long long x_sum[2][kMaxCluster];   // Z, then W of the deciding row (double-buffered)
   float x_max[2][kMaxCluster];                // row maximum (double-buffered over rows)
@@ -163,7 +170,9 @@ struct Shared {
   int idx_scratch[32];
   int flag;
   int decision;      // 1 accepted, 0 decide here
-  int pick;
+  // what the accept test of the row in work needs besides Z, fetched while the row is being read
+  float dec_z, dec_q;
+  uint32_t dec_u[2];
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -176,13 +185,28 @@ __device__ __forceinline__ void cluster_barrier() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-// One cluster of C blocks per request; block `rank` owns a contiguous run of 4096-entry vocabulary tiles.
-// Per examined row the blocks exchange (maximum, argmax, finiteness), then the integer sums, through
-// each other's shared memory; every block then takes the same decision from the same numbers.
-template <int kThreads>
+// Entries of the vocabulary that one warp owns: the row is cut into C * kWarps contiguous ranges of `per_warp`
+// entries (a multiple of kStep), block after block and warp after warp in vocabulary order.
+__host__ __device__ inline int entries_per_warp(int V, int C, int warps) {
+  const int64_t cut = static_cast<int64_t>(C) * warps * kStep;
+  return static_cast<int>((V + cut - 1) / cut) * kStep;
+}
+
+// One cluster of C blocks per request.  Every warp owns one contiguous range of the vocabulary, so that the sum a
+// warp forms over its range is one entry of a prefix structure in vocabulary order: block totals (exchanged through
+// each other's shared memory), warp totals, and - for the one warp in whose range the draw falls - a scan over its
+// steps.  Per examined row the blocks exchange (maximum, argmax, finiteness), then the integer sums; every block
+// then takes the same decision from the same numbers.
+//
+// kCache (sampling, 16-byte aligned rows whose share per block fits kCacheBytes): a row is read from global memory
+// once.  The first pass leaves the block's share of the logits in shared memory, the second replaces each by its
+// scaled numerator (the float whose truncation is E_v), the third - on the deciding row - converts those instead of
+// evaluating the exponential again.  A lane meets the same entries in every pass.
+template <int kThreads, bool kCache>
 __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kernel(AcceptArgs a, int C) {
-  constexpr int kTile = kThreads * kVec;        // entries per tile: 4096 with 1024 threads, 2048 with 512
+  constexpr int kWarps = kThreads / 32;
   __shared__ Shared sh;
+  extern __shared__ __align__(16) float zc[];   // kCache: entries b_lo.. of the row in work
   StampScope scope(LaunchStamp{a.stamp.begin, a.stamp.end});
   pdl_enter();
   const int req = blockIdx.x / C, rank = blockIdx.x % C;
@@ -196,10 +220,14 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     return q16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(qbase)[idx]) : static_cast<const float*>(qbase)[idx];
   };
   int32_t* res = a.results + 3 * req;
-  const int n_tiles = (V + kTile - 1) / kTile;
-  const int tiles_per_rank = (n_tiles + C - 1) / C;
-  const int tl_lo = min(n_tiles, rank * tiles_per_rank), tl_hi = min(n_tiles, tl_lo + tiles_per_rank);
-  const int v_lo = tl_lo * kTile, v_hi = min(V, tl_hi * kTile);   // this block's vocabulary range
+  const int per_warp = entries_per_warp(V, C, kWarps);
+  const int64_t b_first = static_cast<int64_t>(rank) * kWarps * per_warp;
+  const int b_lo = static_cast<int>(b_first < V ? b_first : V);                       // this block's range
+  const int b_hi = static_cast<int>(b_first + kWarps * per_warp < V ? b_first + kWarps * per_warp : V);
+  const int w_lo = min(b_hi, b_lo + warp * per_warp), w_hi = min(b_hi, w_lo + per_warp);   // this warp's range
+  const bool vec = ((V & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
+  // the draft rows are the caller's memory: any 4-byte aligned address is legal, 16-byte loads need more
+  const bool q_vec = vec && ((reinterpret_cast<uintptr_t>(qbase) & (q16 ? 7 : 15)) == 0);   // four entries per load
   int xphase = 0;   // parity of the sum exchange slots
 
   for (int j = 0; j <= k; ++j) {
@@ -208,9 +236,18 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     float best = -INFINITY;
     int best_i = 0x7fffffff;
     int bad = 0;
-    const bool vec = ((V & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.logits) & 15) == 0);
-    // the draft rows are the caller's memory: any 4-byte aligned address is legal, 16-byte loads need more
-    const bool q_vec = vec && ((reinterpret_cast<uintptr_t>(qbase) & (q16 ? 7 : 15)) == 0);   // four entries per load
+    if (!a.greedy && threadIdx.x == 32) {          // the two uniforms of this position
+      uint32_t w[4];
+      philox4x32_10(static_cast<uint32_t>(a.seed), static_cast<uint32_t>(a.seed >> 32), a.ctx_lo[req], a.ctx_hi[req],
+                    static_cast<uint32_t>(a.pos0[req] + j + 1), 0u, w);
+      sh.dec_u[0] = w[0];
+      sh.dec_u[1] = w[1];
+    }
+    if (!a.greedy && threadIdx.x == 64 && j < k) {   // the draft's logit and its draft probability
+      const int d = a.ids[row0 + 1 + j];
+      sh.dec_z = z[d];
+      sh.dec_q = q_at(static_cast<int64_t>(j) * V + d);
+    }
     if (vec && !a.greedy) {
       // sampling needs the maximum only, and rounding is monotone: max(z * inv_tau) = max(z) * inv_tau.  A NaN or an
       // infinity anywhere turns the running sum of z * 0 into a NaN.
@@ -222,47 +259,55 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
         nan2 = fma2(pack2(x4.x, x4.y), zero2, nan2);
         nan2 = fma2(pack2(x4.z, x4.w), zero2, nan2);
       };
-      constexpr int kStep = kThreads * 4;
-      int v = v_lo + threadIdx.x * 4;
-      for (; v + 3 * kStep < v_hi; v += 4 * kStep) {
+      int v = w_lo + lane * kVec;
+      for (; v + 3 * kStep < w_hi; v += 4 * kStep) {
         const float4 x0 = *reinterpret_cast<const float4*>(z + v);
         const float4 x1 = *reinterpret_cast<const float4*>(z + v + kStep);
         const float4 x2 = *reinterpret_cast<const float4*>(z + v + 2 * kStep);
         const float4 x3 = *reinterpret_cast<const float4*>(z + v + 3 * kStep);
         look(x0); look(x1); look(x2); look(x3);
+        if constexpr (kCache) {
+          *reinterpret_cast<float4*>(zc + (v - b_lo)) = x0;
+          *reinterpret_cast<float4*>(zc + (v - b_lo) + kStep) = x1;
+          *reinterpret_cast<float4*>(zc + (v - b_lo) + 2 * kStep) = x2;
+          *reinterpret_cast<float4*>(zc + (v - b_lo) + 3 * kStep) = x3;
+        }
       }
-      for (; v < v_hi; v += kStep) look(*reinterpret_cast<const float4*>(z + v));
+      for (; v < w_hi; v += kStep) {
+        const float4 x0 = *reinterpret_cast<const float4*>(z + v);
+        look(x0);
+        if constexpr (kCache) *reinterpret_cast<float4*>(zc + (v - b_lo)) = x0;
+      }
       float n0, n1;
       unpack2(nan2, n0, n1);
       bad = !(n0 == 0.f) || !(n1 == 0.f);
-      best = __fmul_rn(mx, a.inv_tau);   // -inf when this thread saw no entry
+      best = __fmul_rn(mx, a.inv_tau);   // -inf when this lane saw no entry
       best_i = 0;                        // not used when sampling
-    } else if (vec) {   // four consecutive entries per thread and step (16-byte loads), four steps in flight
+    } else if (vec) {   // four consecutive entries per lane and step (16-byte loads), four steps in flight
       auto look = [&](int v, const float4& x4) {
         const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           bad |= !(fabsf(xs[e]) < INFINITY);
           const float sv = a.greedy ? xs[e] : __fmul_rn(xs[e], a.inv_tau);
-          if (sv > best) { best = sv; best_i = v + e; }   // ascending v per thread: first maximum kept
+          if (sv > best) { best = sv; best_i = v + e; }   // ascending v per lane: first maximum kept
         }
       };
-      constexpr int kStep = kThreads * 4;
-      int v = v_lo + threadIdx.x * 4;
-      for (; v + 3 * kStep < v_hi; v += 4 * kStep) {
+      int v = w_lo + lane * kVec;
+      for (; v + 3 * kStep < w_hi; v += 4 * kStep) {
         const float4 x0 = *reinterpret_cast<const float4*>(z + v);
         const float4 x1 = *reinterpret_cast<const float4*>(z + v + kStep);
         const float4 x2 = *reinterpret_cast<const float4*>(z + v + 2 * kStep);
         const float4 x3 = *reinterpret_cast<const float4*>(z + v + 3 * kStep);
         look(v, x0); look(v + kStep, x1); look(v + 2 * kStep, x2); look(v + 3 * kStep, x3);
       }
-      for (; v < v_hi; v += kStep) look(v, *reinterpret_cast<const float4*>(z + v));
+      for (; v < w_hi; v += kStep) look(v, *reinterpret_cast<const float4*>(z + v));
     } else {
-      for (int v = v_lo + threadIdx.x; v < v_hi; v += kThreads) {
+      for (int v = w_lo + lane; v < w_hi; v += 32) {
         const float x = z[v];
         bad |= !(fabsf(x) < INFINITY);
         const float sv = a.greedy ? x : __fmul_rn(x, a.inv_tau);
-        if (sv > best) { best = sv; best_i = v; }   // ascending v per thread: first maximum kept
+        if (sv > best) { best = sv; best_i = v; }   // ascending v per lane: first maximum kept
       }
     }
 #pragma unroll
@@ -274,11 +319,12 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     bad = __syncthreads_or(bad);
     if (lane == 0) { sh.max_scratch[warp] = best; sh.idx_scratch[warp] = best_i; }
     __syncthreads();
-    best = sh.max_scratch[0];
-    best_i = sh.idx_scratch[0];
-    for (int w = 1; w < kThreads / 32; ++w) {
-      const float ob = sh.max_scratch[w];
-      const int oi = sh.idx_scratch[w];
+    best = lane < kWarps ? sh.max_scratch[lane] : -INFINITY;
+    best_i = lane < kWarps ? sh.idx_scratch[lane] : 0x7fffffff;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
       if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
     }
     if (C > 1) {
@@ -313,25 +359,34 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     // ---- pass 2: Z = sum of the integer numerators
     unsigned long long zsum = 0;
     const Exp2Consts ec = exp2_consts(a.inv_tau, m);
-    if (vec) {
+    if constexpr (kCache) {
+      // numerators from the share in shared memory; each entry is replaced by its scaled numerator
+      for (int o = w_lo - b_lo + lane * kVec; o < w_hi - b_lo; o += kStep) {
+        const float4 x4 = *reinterpret_cast<const float4*>(zc + o);
+        float4 s4;
+        fixed_exp_pair_f(x4.x, x4.y, ec, s4.x, s4.y);
+        fixed_exp_pair_f(x4.z, x4.w, ec, s4.z, s4.w);
+        zsum += (__float2ull_rz(s4.x) + __float2ull_rz(s4.y)) + (__float2ull_rz(s4.z) + __float2ull_rz(s4.w));
+        *reinterpret_cast<float4*>(zc + o) = s4;
+      }
+    } else if (vec) {
       auto add4 = [&](const float4& x4) {
         unsigned long long e0, e1, e2, e3;
         fixed_exp_pair(x4.x, x4.y, ec, e0, e1);
         fixed_exp_pair(x4.z, x4.w, ec, e2, e3);
         zsum += (e0 + e1) + (e2 + e3);
       };
-      constexpr int kStep = kThreads * 4;
-      int v = v_lo + threadIdx.x * 4;
-      for (; v + 3 * kStep < v_hi; v += 4 * kStep) {
+      int v = w_lo + lane * kVec;
+      for (; v + 3 * kStep < w_hi; v += 4 * kStep) {
         const float4 x0 = *reinterpret_cast<const float4*>(z + v);
         const float4 x1 = *reinterpret_cast<const float4*>(z + v + kStep);
         const float4 x2 = *reinterpret_cast<const float4*>(z + v + 2 * kStep);
         const float4 x3 = *reinterpret_cast<const float4*>(z + v + 3 * kStep);
         add4(x0); add4(x1); add4(x2); add4(x3);
       }
-      for (; v < v_hi; v += kStep) add4(*reinterpret_cast<const float4*>(z + v));
+      for (; v < w_hi; v += kStep) add4(*reinterpret_cast<const float4*>(z + v));
     } else {
-      for (int v = v_lo + threadIdx.x; v < v_hi; v += kThreads) zsum += fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
+      for (int v = w_lo + lane; v < w_hi; v += 32) zsum += fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
     }
     unsigned long long Z = block_sum_u64<kThreads>(zsum, sh.sum_scratch);
     if (C > 1) {
@@ -346,79 +401,98 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     int64_t q_off = -1;     // first entry of the deciding row's draft distribution, -1: none (bonus row)
     uint32_t u_smp = 0;
     if (threadIdx.x == 0) {
-      uint32_t w[4];
-      philox4x32_10(static_cast<uint32_t>(a.seed), static_cast<uint32_t>(a.seed >> 32), a.ctx_lo[req], a.ctx_hi[req],
-                    static_cast<uint32_t>(a.pos0[req] + j + 1), 0u, w);
       int accepted = 0;
       if (j < k) {
-        const int d = a.ids[row0 + 1 + j];
-        const unsigned long long Ed = fixed_exp(__fsub_rn(__fmul_rn(z[d], a.inv_tau), m));
-        const float qd = q_at(static_cast<int64_t>(j) * V + d);
-        const double lhs = __dmul_rn(__dmul_rn(static_cast<double>(w[0] >> 8), static_cast<double>(qd)),
+        const unsigned long long Ed = fixed_exp(__fsub_rn(__fmul_rn(sh.dec_z, a.inv_tau), m));
+        const double lhs = __dmul_rn(__dmul_rn(static_cast<double>(sh.dec_u[0] >> 8), static_cast<double>(sh.dec_q)),
                                      __ull2double_rn(Z));
         const double rhs = __dmul_rn(__ull2double_rn(Ed), 16777216.0);
         accepted = lhs < rhs;
       }
       sh.decision = accepted;
-      sh.flag = static_cast<int>(w[1]);
+      sh.flag = static_cast<int>(sh.dec_u[1]);
     }
     __syncthreads();
     if (sh.decision) continue;
     u_smp = static_cast<uint32_t>(sh.flag);
     if (j < k) q_off = static_cast<int64_t>(j) * V;
 
-    // ---- deciding row: weights R_v = max(E_v - trunc(q_v * Z), 0) (or E_v), tile sums in vocabulary order
+    // ---- deciding row: weights R_v = max(E_v - trunc(q_v * Z), 0) (or E_v), summed per warp range
     const double Zd = __ull2double_rn(Z);
     bool use_q = q_off >= 0;
-    unsigned long long W = 0, before_me = 0;
-    for (int attempt = 0; attempt < 2; ++attempt) {
-      for (int tl = threadIdx.x; tl < n_tiles; tl += kThreads) sh.tile_sum[tl] = 0ull;
-      __syncthreads();
-      for (int tl = tl_lo; tl < tl_hi; ++tl) {
-        unsigned long long mine = 0;
-        const int v0 = tl * kTile + threadIdx.x * kVec;
-        float zs[kVec], qs[kVec];
-        if (vec && v0 + kVec <= V) {
+    if (use_q && b_lo < b_hi) {
+      // this block's share of the draft row is wanted step by step: ask for all of its lines now
+      const int es = q16 ? 2 : 4;
+      const char* qb = static_cast<const char*>(qbase) + (q_off + b_lo) * es;
+      const int bytes = (b_hi - b_lo) * es;
+      for (int b = threadIdx.x * 128; b < bytes; b += kThreads * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(qb + b));
+    }
+    // the four weights of a lane at entries v0..v0+3 (entries from w_hi on count zero)
+    auto fetch = [&](int v0, float (&zs)[kVec], float (&qs)[kVec]) {
+      if (vec) {   // V % 4 == 0: a lane's four entries are inside the row together
+        if constexpr (!kCache) {
           const float4 z4 = *reinterpret_cast<const float4*>(z + v0);
           zs[0] = z4.x; zs[1] = z4.y; zs[2] = z4.z; zs[3] = z4.w;
-          if (use_q && q_vec && !q16) {
-            const float4 q4 = *reinterpret_cast<const float4*>(static_cast<const float*>(qbase) + q_off + v0);
-            qs[0] = q4.x; qs[1] = q4.y; qs[2] = q4.z; qs[3] = q4.w;
-          } else if (use_q && q_vec) {
-            const uint2 q4 = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(qbase) + q_off + v0);
-            qs[0] = __uint_as_float(q4.x << 16); qs[1] = __uint_as_float(q4.x & 0xffff0000u);
-            qs[2] = __uint_as_float(q4.y << 16); qs[3] = __uint_as_float(q4.y & 0xffff0000u);
-          } else if (use_q) {
-#pragma unroll
-            for (int e = 0; e < kVec; ++e) qs[e] = q_at(q_off + v0 + e);
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < kVec; ++e) {
-            zs[e] = v0 + e < V ? z[v0 + e] : 0.f;
-            qs[e] = (use_q && v0 + e < V) ? q_at(q_off + v0 + e) : 0.f;
-          }
         }
-        unsigned long long Es[kVec];
+        if (use_q && q_vec && !q16) {
+          const float4 q4 = *reinterpret_cast<const float4*>(static_cast<const float*>(qbase) + q_off + v0);
+          qs[0] = q4.x; qs[1] = q4.y; qs[2] = q4.z; qs[3] = q4.w;
+        } else if (use_q && q_vec) {
+          const uint2 q4 = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(qbase) + q_off + v0);
+          qs[0] = __uint_as_float(q4.x << 16); qs[1] = __uint_as_float(q4.x & 0xffff0000u);
+          qs[2] = __uint_as_float(q4.y << 16); qs[3] = __uint_as_float(q4.y & 0xffff0000u);
+        } else if (use_q) {
 #pragma unroll
-        for (int e = 0; e < kVec; e += 2) fixed_exp_pair(zs[e], zs[e + 1], ec, Es[e], Es[e + 1]);
+          for (int e = 0; e < kVec; ++e) qs[e] = q_at(q_off + v0 + e);
+        }
+      } else {
 #pragma unroll
         for (int e = 0; e < kVec; ++e) {
-          if (v0 + e < V) {
-            unsigned long long E = Es[e];
-            if (use_q) {
-              const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(qs[e]), Zd));
-              E = E > Q ? E - Q : 0ull;
-            }
-            mine += E;
-          }
+          zs[e] = v0 + e < w_hi ? z[v0 + e] : 0.f;
+          qs[e] = (use_q && v0 + e < w_hi) ? q_at(q_off + v0 + e) : 0.f;
         }
-        mine = warp_sum_u64(mine);
-        if (lane == 0 && mine) atomicAdd(&sh.tile_sum[tl], mine);  // integer adds: any order, same sum
       }
+    };
+    auto weights = [&](int v0, const float (&zs)[kVec], const float (&qs)[kVec], unsigned long long (&r)[kVec]) {
+      if constexpr (kCache) {   // the scaled numerators the second pass left behind
+        const float4 s4 = *reinterpret_cast<const float4*>(zc + (v0 - b_lo));
+        r[0] = __float2ull_rz(s4.x); r[1] = __float2ull_rz(s4.y);
+        r[2] = __float2ull_rz(s4.z); r[3] = __float2ull_rz(s4.w);
+      } else {
+#pragma unroll
+        for (int e = 0; e < kVec; e += 2) fixed_exp_pair(zs[e], zs[e + 1], ec, r[e], r[e + 1]);
+      }
+#pragma unroll
+      for (int e = 0; e < kVec; ++e) {
+        if (use_q) {
+          const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(qs[e]), Zd));
+          r[e] = r[e] > Q ? r[e] - Q : 0ull;
+        }
+        if (v0 + e >= w_hi) r[e] = 0ull;
+      }
+    };
+    unsigned long long W = 0, before_me = 0, mine_w = 0;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+      unsigned long long mine = 0;
+      // the loads of the next step are in flight while this one is worked on
+      float zn[kVec] = {0.f, 0.f, 0.f, 0.f}, qn[kVec] = {0.f, 0.f, 0.f, 0.f};
+      int v0 = w_lo + lane * kVec;
+      if (v0 < w_hi) fetch(v0, zn, qn);
+      for (; v0 < w_hi; v0 += kStep) {
+        float zs[kVec], qs[kVec];
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) { zs[e] = zn[e]; qs[e] = qn[e]; }
+        if (v0 + kStep < w_hi) fetch(v0 + kStep, zn, qn);
+        unsigned long long r[kVec];
+        weights(v0, zs, qs, r);
+        mine += (r[0] + r[1]) + (r[2] + r[3]);
+      }
+      mine = warp_sum_u64(mine);   // integer adds: any order, same sum
       __syncthreads();
-      unsigned long long mine_w = 0;
-      for (int tl = tl_lo; tl < tl_hi; ++tl) mine_w += sh.tile_sum[tl];
+      if (lane == 0) sh.warp_tot[warp] = mine;
+      __syncthreads();
+      mine_w = warp_sum_u64(lane < kWarps ? sh.warp_tot[lane] : 0ull);
       W = mine_w;
       before_me = 0;
       if (C > 1) {
@@ -434,77 +508,63 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
       }
       if (W != 0 || !use_q) break;
       use_q = false;   // residual mass zero (p <= q everywhere after rounding): draw from p itself
-      __syncthreads();
     }
     // ---- inverse CDF: tgt = (U' * W) >> 32, first v whose running sum exceeds tgt
     const unsigned long long tgt = __umul64hi(W, static_cast<unsigned long long>(u_smp) << 32);
-    unsigned long long my_w = 0;
-    for (int tl = tl_lo; tl < tl_hi; ++tl) my_w += sh.tile_sum[tl];
-    if (!(before_me <= tgt && tgt < before_me + my_w)) return;   // the crossing lies in another block's range
-    int tl_hit = tl_lo;
-    unsigned long long before = before_me;
-    for (int tl = tl_lo; tl < tl_hi; ++tl) {
-      const unsigned long long nx = before + sh.tile_sum[tl];
-      if (nx > tgt) { tl_hit = tl; break; }
-      before = nx;
-      tl_hit = tl;
-    }
-    unsigned long long r[kVec];
-    unsigned long long mine = 0;
-    {
-      const int v0 = tl_hit * kTile + threadIdx.x * kVec;
+    if (!(before_me <= tgt && tgt < before_me + mine_w)) return;   // the crossing lies in another block's range
+    unsigned long long run = before_me;
+    for (int w = 0; w < warp; ++w) run += sh.warp_tot[w];
+    if (!(run <= tgt && tgt < run + sh.warp_tot[warp])) return;    // ... or in another warp's
+    // this warp scans its range step by step (all lanes take the same path)
+    for (int base = w_lo; base < w_hi; base += kStep) {
+      const int v0 = base + lane * kVec;
+      unsigned long long r[kVec] = {0ull, 0ull, 0ull, 0ull};
+      if (v0 < w_hi) {
+        float zs[kVec] = {0.f, 0.f, 0.f, 0.f}, qs[kVec] = {0.f, 0.f, 0.f, 0.f};
+        fetch(v0, zs, qs);
+        weights(v0, zs, qs, r);
+      }
+      const unsigned long long lane_sum = (r[0] + r[1]) + (r[2] + r[3]);
+      unsigned long long incl = lane_sum;
 #pragma unroll
-      for (int e = 0; e < kVec; ++e) {
-        const int v = v0 + e;
-        unsigned long long E = 0;
-        if (v < V) {
-          E = fixed_exp(__fsub_rn(__fmul_rn(z[v], a.inv_tau), m));
-          if (use_q) {
-            const unsigned long long Q = __double2ull_rz(__dmul_rn(static_cast<double>(q_at(q_off + v)), Zd));
-            E = E > Q ? E - Q : 0ull;
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      const unsigned long long step_sum = __shfl_sync(0xffffffffu, incl, 31);
+      if (run + step_sum > tgt) {
+        unsigned long long at = run + incl - lane_sum;   // weight in front of this lane's entries
+        if (at <= tgt && tgt < at + lane_sum) {          // exactly one lane sees the crossing
+          int pick = v0;
+#pragma unroll
+          for (int e = 0; e < kVec; ++e) {
+            at += r[e];
+            if (at > tgt) { pick = v0 + e; break; }
           }
+          res[0] = j; res[1] = pick; res[2] = ST_OK;
         }
-        r[e] = E;
-        mine += E;
+        return;
       }
+      run += step_sum;
     }
-    // exclusive prefix of `mine` over the block in thread order
-    unsigned long long incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += up;
-    }
-    __syncthreads();
-    if (lane == 31) sh.warp_pref[warp] = incl;
-    if (threadIdx.x == 0) sh.pick = V - 1;
-    __syncthreads();
-    unsigned long long run = before + incl - mine;
-    for (int w = 0; w < warp; ++w) run += sh.warp_pref[w];
-    // exactly one thread sees the crossing
-    if (run <= tgt && run + mine > tgt) {
-      int pick = tl_hit * kTile + threadIdx.x * kVec;
-#pragma unroll
-      for (int e = 0; e < kVec; ++e) {
-        run += r[e];
-        if (run > tgt) { pick += e; break; }
-      }
-      sh.pick = pick;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) { res[0] = j; res[1] = sh.pick; res[2] = ST_OK; }
     return;
   }
 }
 
 }  // namespace
 
-template <int kThreads>
+template <int kThreads, bool kCache>
 static int launch_accept_t(const AcceptArgs& a, int C, cudaStream_t s) {
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(a.B * C, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = 0;
+  if (kCache) {
+    // the cached form's dynamic shared memory is above the default limit (set per device; cheap enough per launch)
+    if (cudaFuncSetAttribute(accept_kernel<kThreads, kCache>, cudaFuncAttributeMaxDynamicSharedMemorySize, kCacheBytes) != cudaSuccess)
+      return -1;
+    cfg.dynamicSmemBytes = static_cast<size_t>(kThreads / 32) * entries_per_warp(a.V, C, kThreads / 32) * sizeof(float);
+  }
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -515,7 +575,16 @@ static int launch_accept_t(const AcceptArgs& a, int C, cudaStream_t s) {
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, accept_kernel<kThreads>, a, C) == cudaSuccess ? 1 : -1;
+  return cudaLaunchKernelEx(&cfg, accept_kernel<kThreads, kCache>, a, C) == cudaSuccess ? 1 : -1;
+}
+
+// Whether the cached form applies with C blocks per request: sampling, 16-byte aligned rows, and a block's share of
+// a row within kCacheBytes.  (More blocks per request than occupancy asks for, only to make a row fit, measured slower
+// on 512 requests: a row then costs six exchanges between eight blocks, and those, not the arithmetic, set the pace.)
+template <int kThreads>
+static bool cached_form_fits(const AcceptArgs& a, int C) {
+  if (a.greedy || (a.V & 3) || (reinterpret_cast<uintptr_t>(a.logits) & 15)) return false;
+  return static_cast<size_t>(kThreads / 32) * entries_per_warp(a.V, C, kThreads / 32) * sizeof(float) <= kCacheBytes;
 }
 
 int launch_accept(const AcceptArgs& a, cudaStream_t s) {
@@ -528,18 +597,19 @@ int launch_accept(const AcceptArgs& a, cudaStream_t s) {
   }
   // Small batches: blocks of 1024 threads, as many blocks per request (a cluster) as it takes to occupy the machine.
   // Large batches: blocks of 512 threads, compiled for three per SM (one 1024-thread block fits otherwise), so that
-  // several requests hide each other's latencies - and two blocks per request (measured best among 1 / 2 / 4).
-  if (a.B * kMaxCluster >= 2 * n_sm && a.V <= 512 * kVec * kMaxTiles) {
+  // several requests hide each other's latencies - and two blocks per request (measured best among 1 / 2 / 4).  Either
+  // way a row stays in shared memory between the passes (the cached form) where a block's share of it fits.
+  if (a.V > (1 << 30)) return -1;
+  if (a.B * kMaxCluster >= 2 * n_sm) {
     constexpr int kTile = 512 * kVec;
     int C = 1;
     while (C < kMaxCluster && a.B * C < 6 * n_sm && (a.V + kTile - 1) / kTile >= 2 * C) C *= 2;
-    return launch_accept_t<512>(a, C, s);
+    return cached_form_fits<512>(a, C) ? launch_accept_t<512, true>(a, C, s) : launch_accept_t<512, false>(a, C, s);
   }
   constexpr int kTile = 1024 * kVec;
-  if (a.V > kTile * kMaxTiles) return -1;
   int C = 1;
   while (C < kMaxCluster && a.B * C < 128 && (a.V + kTile - 1) / kTile >= 2 * C) C *= 2;
-  return launch_accept_t<1024>(a, C, s);
+  return cached_form_fits<1024>(a, C) ? launch_accept_t<1024, true>(a, C, s) : launch_accept_t<1024, false>(a, C, s);
 }
 
 }  // namespace sled
