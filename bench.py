@@ -3,7 +3,7 @@
 synthetic device requests, commit / rollback included).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-                    [--shape llama8b] [--batch 16] [--layers L] [--greedy] [--weight-bits 8]
+                    [--shape llama8b] [--batch 16] [--layers L] [--greedy] [--weight-bits 8|4]
                     [--workload step|accept|attention|serve]
 
 Prints ONE JSON line.  Metric: verified (committed) tokens per second at the Llama-3-8B shape.
@@ -13,8 +13,8 @@ distributions correlated with the target's own logits (`--drafts independent`: f
 that ignore the target).  `roofline` is for the tensor-core linear-layer kernel, the dominant one;
 `kernel_ms` splits an untouched step by kind of kernel from per-launch device timestamps,
 `kernel_ms_serialised` is the same with events between the kernels.  `sweep` repeats the step at
-other batch sizes (fewer steps, no end-to-end leg), `weights_8bit` with the linear layers' weights as e4m3
-bytes (`--weight-bits 8` runs everything that way).  `--impl reference` times the CPU oracle.
+other batch sizes (fewer steps, no end-to-end leg), `weights_8bit` / `weights_4bit` with the linear layers'
+weights as e4m3 bytes / e2m1 nibbles (`--weight-bits 8` / `4` runs everything that way).  `--impl reference` times the CPU oracle.
 Under torchrun every rank runs its own replica on its own requests (no data-path collective).
 """
 from __future__ import annotations
@@ -77,7 +77,7 @@ def parse_args(argv=None):
     ap.add_argument("--drafts", default="correlated", choices=["correlated", "independent"],
                     help="correlated: draft distributions built from the target's own logits (rho = 0.8), "
                          "independent: softmax of N(0,1) logits")
-    ap.add_argument("--weight-bits", type=int, default=16, choices=[16, 8],
+    ap.add_argument("--weight-bits", type=int, default=16, choices=[16, 8, 4],
                     help="8: the linear layers' weights as e4m3 bytes with one scale per output row (step workload)")
     ap.add_argument("--attention-impl", type=int, default=0, choices=[0, 1],
                     help="0: warp-level tensor-core attention kernel (default), 1: the tcgen05 kernel (head_dim 128)")
@@ -200,15 +200,15 @@ def linear_shapes(shape):
     return per_layer * s.n_layers + [(s.vocab, s.d_model)]
 
 
-WEIGHT_BITS = 16   # --weight-bits 8: e4m3 bytes + one fp32 scale per output row
+WEIGHT_BITS = 16   # --weight-bits 8 / 4: e4m3 bytes / e2m1 nibbles + one fp32 scale per output row
 
 
 def linear_bytes(shape, T: int) -> float:
     """Bytes the linear layers must move in one step: every weight once (bf16, or a byte and the rows' scales),
     their bf16 inputs, their fp32 outputs."""
     es = 2 if shape.weight_dtype == "bf16" else 4
-    if WEIGHT_BITS == 8:
-        return float(sum(n * k + n * 4 + T * k * es + T * n * 4 for n, k in linear_shapes(shape)))
+    if WEIGHT_BITS in (8, 4):
+        return float(sum(n * k * WEIGHT_BITS // 8 + n * 4 + T * k * es + T * n * 4 for n, k in linear_shapes(shape)))
     return float(sum(n * k * es + T * k * es + T * n * 4 for n, k in linear_shapes(shape)))
 
 
@@ -510,10 +510,10 @@ def run_sled(args):
     peaks, peak_src = load_peaks()
     w = I.make_weights(shape, seed, device=dev)
     global WEIGHT_BITS
-    if args.weight_bits == 8:
-        WEIGHT_BITS = 8
+    if args.weight_bits in (8, 4):
+        WEIGHT_BITS = args.weight_bits
         args.no_cpu_baseline = True          # the oracle arm is timed on the 16-bit workload
-        w, _ = I.quantize_linear_weights(w, dequantised=False)
+        w, _ = I.quantize_linear_weights(w, dequantised=False, bits=args.weight_bits)
         torch.cuda.empty_cache()
     need_host_w = (rank == 0 and world == 1 and not args.no_cpu_baseline)
     w_host = I.weights_to(w, "cpu") if need_host_w else None
@@ -561,12 +561,12 @@ def run_sled(args):
     step_s = ms_all / args.steps / 1e3
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_all / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": ("bf16 (e4m3 weights)" if args.weight_bits == 8 else "bf16") if shape.weight_dtype == "bf16" else "f32",
+            "dtype": ({8: "bf16 (e4m3 weights)", 4: "bf16 (e2m1 weights)"}.get(args.weight_bits, "bf16")) if shape.weight_dtype == "bf16" else "f32",
             "data": "synthetic",
             "config": {"workload": pt.name, "tokens_scored_per_step": T,
                        "attention_kernel": "tcgen05" if args.attention_impl == 1 else "warp-level mma",
                        "linear_weight_bits": args.weight_bits,
-                       "l2": "inputs larger than L2 (a step streams %.2f GB of weights)" % ((1e-9 if args.weight_bits == 8 else 2e-9) * shape.streamed_params()),
+                       "l2": "inputs larger than L2 (a step streams %.2f GB of weights)" % (args.weight_bits / 8 * 1e-9 * shape.streamed_params()),
                        "draft_distributions": ("target-correlated: draft logits = 0.8 z + 0.6 std(z) noise, z the target's "
                                                "own logits at that position (untimed passes), q = softmax, d ~ q"
                                                if correlated else "independent of the target (softmax of N(0,1) logits)"),
@@ -626,32 +626,34 @@ def run_sled(args):
             sp.close()
         line["sweep"] = sweep
 
-    # ---- the same step with 8-bit weights in the linear layers (the paper sweeps 16-, 8- and 4-bit precision)
+    # ---- the same step with 8-bit and 4-bit weights in the linear layers (the paper sweeps 16-, 8- and 4-bit precision)
     if not args.no_sweep and world == 1 and args.weight_bits == 16 and shape.weight_dtype == "bf16":
-        w8, _ = I.quantize_linear_weights(w, dequantised=False)
-        args8 = argparse.Namespace(**{**vars(args), "weight_bits": 8})
-        WEIGHT_BITS = 8
-        rows = []
-        for b in sorted({args.batch, 1}, reverse=True):
-            sp = Point(B, args8, shape, w8, b, rank, local_rank, world, stream)
-            dh, qd = sp.correlated_drafts() if correlated else sp.independent_drafts()
-            torch.cuda.synchronize()
-            rq = sp.marshal(dh, qd)
-            n_steps = max(5, args.steps // 2)
-            c_s, ms_s, _ = sp.timed(rq, n_steps, 3)
-            km_s, n_lin_s, n_rej_s = sp.kernel_times(rq, 1, steps=3)
-            entry = {"batch": b, "tokens_scored_per_step": sp.T, "steps": n_steps, "workload": sp.name}
-            entry.update(sp.summary(c_s, ms_s, n_steps, n_rej_s, peaks))
-            entry["kernel_ms"] = km_s
-            r = sp.linear_roofline(km_s, n_lin_s, peaks, peak_src)
-            entry["linear_layers"] = {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac") if k in r}
-            rows.append(entry)
-            del dh, qd, rq
-            sp.close()
-        WEIGHT_BITS = 16
-        line["weights_8bit"] = {"format": "e4m3 bytes + one fp32 scale per output row; fp8 MMAs on activations split into "
-                                          "two e4m3 parts; bytes counted with one byte per weight", "points": rows}
-        del w8
+        for bits, key, fmt in ((8, "weights_8bit", "e4m3 bytes"), (4, "weights_4bit", "e2m1 nibbles, two to a byte,")):
+            wn, _ = I.quantize_linear_weights(w, dequantised=False, bits=bits)
+            argsn = argparse.Namespace(**{**vars(args), "weight_bits": bits})
+            WEIGHT_BITS = bits
+            rows = []
+            for b in sorted({args.batch, 1}, reverse=True):
+                sp = Point(B, argsn, shape, wn, b, rank, local_rank, world, stream)
+                dh, qd = sp.correlated_drafts() if correlated else sp.independent_drafts()
+                torch.cuda.synchronize()
+                rq = sp.marshal(dh, qd)
+                n_steps = max(5, args.steps // 2)
+                c_s, ms_s, _ = sp.timed(rq, n_steps, 3)
+                km_s, n_lin_s, n_rej_s = sp.kernel_times(rq, 1, steps=3)
+                entry = {"batch": b, "tokens_scored_per_step": sp.T, "steps": n_steps, "workload": sp.name}
+                entry.update(sp.summary(c_s, ms_s, n_steps, n_rej_s, peaks))
+                entry["kernel_ms"] = km_s
+                r = sp.linear_roofline(km_s, n_lin_s, peaks, peak_src)
+                entry["linear_layers"] = {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac") if k in r}
+                rows.append(entry)
+                del dh, qd, rq
+                sp.close()
+            WEIGHT_BITS = 16
+            line[key] = {"format": fmt + " + one fp32 scale per output row; fp8 MMAs on activations split into two e4m3 "
+                                         "parts; bytes counted with %d bits per weight" % bits, "points": rows}
+            del wn
+            torch.cuda.empty_cache()
     del w
     torch.cuda.empty_cache()
 
@@ -770,8 +772,8 @@ def run_serve(args):
     counts = [int(x) for x in args.devices.split(",") if x]
     max_k, V = 8, shape.vocab
     w = I.make_weights(shape, args.seed, device=dev)
-    if args.weight_bits == 8:
-        w, _ = I.quantize_linear_weights(w, dequantised=False)
+    if args.weight_bits in (8, 4):
+        w, _ = I.quantize_linear_weights(w, dequantised=False, bits=args.weight_bits)
     stream = torch.cuda.Stream(device=dev)
     n_max = max(counts)
     ctx_len = I.draw_context_lengths(n_max, 128, 512, args.seed)

@@ -93,7 +93,11 @@ typedef struct sled_config {
                              take both operands in 8 bits: every bf16 activation goes in as the sum of two e4m3 numbers
                              times a per-token scale - eight significant bits, as in bf16 - and the products are summed
                              in fp32; embedding, norms, attention and cache are as with 16-bit weights.  d_model, ffn_dim
-                             and n_q_heads * head_dim must be multiples of 16. */
+                             and n_q_heads * head_dim must be multiples of 16.
+                             4: the same with 4-bit weights - e2m1 codes (1 sign, 2 exponent bits with bias 1, 1 mantissa
+                             bit: 0, 0.5, 1, 1.5, 2, 3, 4, 6 and their negatives), two to a byte, the even column in the
+                             low half, rows of in/2 bytes: W[n][k] = scale[n] * e2m1(code[n][k]).  A quarter of the
+                             weight bytes per step; only the weight operand of the fp8 instructions changes. */
 } sled_config;
 
 /* Target weights, row-major [out][in], all of type weight_dtype.  HOST or DEVICE
@@ -112,7 +116,7 @@ typedef struct sled_weights {
   const void* const* w_gate;      /* [ffn_dim][d_model] */
   const void* const* w_up;        /* [ffn_dim][d_model] */
   const void* const* w_down;      /* [d_model][ffn_dim] */
-  /* linear_weight_bits = 8 only (ignored otherwise): fp32 scales, one per output row of the matrix of the same name */
+  /* linear_weight_bits = 8 or 4 only (ignored otherwise): fp32 scales, one per output row of the matrix of the same name */
   const float* lm_head_scale;         /* [vocab] */
   const float* const* wq_scale;       /* [n_q_heads*head_dim] */
   const float* const* wk_scale;       /* [n_kv_heads*head_dim] */

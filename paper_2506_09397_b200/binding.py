@@ -181,7 +181,8 @@ class Engine:
                  page_size: int = 16, stream: int | None = None, draft_probs_dtype: str = "fp32",
                  attention_impl: int = 0, linear_weight_bits: int = 16):
         """linear_weight_bits = 8: weights["wq"] .. ["w_down"] and ["lm_head"] are uint8 tensors of e4m3 bytes and
-        weights["wq_scale"] .. / ["lm_head_scale"] fp32 tensors with one scale per output row."""
+        weights["wq_scale"] .. / ["lm_head_scale"] fp32 tensors with one scale per output row; 4: the same with two
+        e2m1 codes per byte (uint8 tensors [N, K / 2])."""
         self.shape = shape
         cfg = SledConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                          shape.ffn_dim, shape.vocab, shape.rms_eps, shape.rope_theta, _DT[shape.weight_dtype],
@@ -195,7 +196,7 @@ class Engine:
             arr = (C.c_void_p * shape.n_layers)(*[_addr(t) for t in weights[name]])
             keep.append(arr)
             setattr(w, name, C.cast(arr, C.POINTER(C.c_void_p)))
-        if linear_weight_bits == 8:
+        if linear_weight_bits in (8, 4):
             w.lm_head_scale = _addr(weights["lm_head_scale"])
             for name in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down"):
                 arr = (C.c_void_p * shape.n_layers)(*[_addr(t) for t in weights[name + "_scale"]])

@@ -632,8 +632,13 @@ int upload(sled_engine* e, const void* src, size_t bytes, void** dst) {
 }
 
 // bf16 weights: replaces the row-major matrix `rowmajor` (a plain cudaMalloc that this call frees) by its tiled copy
-bool w8(const sled_engine* e) { return e->cfg.linear_weight_bits == 8; }
-size_t weight_elem_size(const sled_engine* e) { return w8(e) ? 1 : dtype_size(e->cfg.weight_dtype); }
+// 8- and 4-bit weights share everything but the weight operand's storage (w8: either of them)
+bool w8(const sled_engine* e) { return e->cfg.linear_weight_bits == 8 || e->cfg.linear_weight_bits == 4; }
+bool w4(const sled_engine* e) { return e->cfg.linear_weight_bits == 4; }
+// bytes of one row of K weights as the caller stores them
+size_t weight_row_bytes(const sled_engine* e, int K) {
+  return w4(e) ? static_cast<size_t>(K) / 2 : w8(e) ? static_cast<size_t>(K) : static_cast<size_t>(K) * dtype_size(e->cfg.weight_dtype);
+}
 
 // takes over `rowmajor` (device, cudaMalloc'ed) and, for 8-bit weights, `scale` (device, [N], kept)
 int finish_linear(sled_engine* e, Linear* L, void* rowmajor, float* scale, int N, int K) {
@@ -642,8 +647,10 @@ int finish_linear(sled_engine* e, Linear* L, void* rowmajor, float* scale, int N
   if (w8(e)) {
     L->scale = scale;
     e->allocs.push_back(scale);
-    int rc = dmalloc(e, &L->w, tc_weight_f8_tiled_bytes(N, K));
-    if (!rc && tc_weight_init_f8(&L->tc, rowmajor, L->w, scale, N, K) != 0) rc = SLED_ERR_ARG;
+    int rc = dmalloc(e, &L->w, w4(e) ? tc_weight_f4_tiled_bytes(N, K) : tc_weight_f8_tiled_bytes(N, K));
+    if (!rc && (w4(e) ? tc_weight_init_f4(&L->tc, rowmajor, L->w, scale, N, K)
+                      : tc_weight_init_f8(&L->tc, rowmajor, L->w, scale, N, K)) != 0)
+      rc = SLED_ERR_ARG;
     cudaFree(rowmajor);
     return rc;
   }
@@ -662,7 +669,7 @@ struct Part { const void* w; const float* scale; int rows; };
 
 int make_linear(sled_engine* e, Linear* L, std::initializer_list<Part> parts, int K) {
   // concatenates the row blocks of `parts` (and, for 8-bit weights, their scales) into one [N][K] matrix
-  const size_t es = weight_elem_size(e);
+  const size_t row_bytes = weight_row_bytes(e, K);
   int N = 0;
   for (auto& p : parts) {
     if (!p.w || (w8(e) && !p.scale)) return SLED_ERR_ARG;
@@ -670,14 +677,14 @@ int make_linear(sled_engine* e, Linear* L, std::initializer_list<Part> parts, in
   }
   void* tmp = nullptr;
   float* scale = nullptr;
-  CU_TRY(cudaMalloc(&tmp, static_cast<size_t>(N) * K * es));
+  CU_TRY(cudaMalloc(&tmp, static_cast<size_t>(N) * row_bytes));
   if (w8(e) && cudaMalloc(reinterpret_cast<void**>(&scale), sizeof(float) * N) != cudaSuccess) {
     cudaFree(tmp);
     return SLED_ERR_DEVICE;
   }
   size_t off = 0, row = 0;
   for (auto& p : parts) {
-    const size_t bytes = static_cast<size_t>(p.rows) * K * es;
+    const size_t bytes = static_cast<size_t>(p.rows) * row_bytes;
     if (cudaMemcpy(static_cast<char*>(tmp) + off, p.w, bytes, cudaMemcpyDefault) != cudaSuccess ||
         (scale && cudaMemcpy(scale + row, p.scale, sizeof(float) * p.rows, cudaMemcpyDefault) != cudaSuccess)) {
       cudaFree(tmp);
@@ -694,7 +701,7 @@ int make_linear(sled_engine* e, Linear* L, std::initializer_list<Part> parts, in
 // so that a pair sits in neighbouring rows of an output tile and SwiGLU can be applied where the sums end up
 int make_gate_up(sled_engine* e, Linear* L, const Part& gate, const Part& up, int F, int K) {
   if (!gate.w || !up.w || (w8(e) && (!gate.scale || !up.scale))) return SLED_ERR_ARG;
-  const size_t row = static_cast<size_t>(K) * weight_elem_size(e);
+  const size_t row = weight_row_bytes(e, K);
   void* tmp = nullptr;
   float* scale = nullptr;
   CU_TRY(cudaMalloc(&tmp, 2 * static_cast<size_t>(F) * row));
@@ -725,9 +732,10 @@ int check_cfg(const sled_config& c) {
   if (c.weight_dtype == SLED_BF16 && c.kv_dtype != SLED_BF16) return SLED_ERR_ARG;
   if (c.draft_probs_dtype != SLED_F32 && c.draft_probs_dtype != SLED_BF16) return SLED_ERR_ARG;
   if (c.attention_impl != 0 && c.attention_impl != 1) return SLED_ERR_ARG;
-  if (c.linear_weight_bits != 0 && c.linear_weight_bits != 16 && c.linear_weight_bits != 8) return SLED_ERR_ARG;
-  if (c.linear_weight_bits == 8 && c.weight_dtype != SLED_BF16) return SLED_ERR_ARG;
-  if (c.linear_weight_bits == 8 && (c.d_model % 16 || c.ffn_dim % 16 || (c.n_q_heads * c.head_dim) % 16)) return SLED_ERR_ARG;
+  const bool narrow = c.linear_weight_bits == 8 || c.linear_weight_bits == 4;
+  if (c.linear_weight_bits != 0 && c.linear_weight_bits != 16 && !narrow) return SLED_ERR_ARG;
+  if (narrow && c.weight_dtype != SLED_BF16) return SLED_ERR_ARG;
+  if (narrow && (c.d_model % 16 || c.ffn_dim % 16 || (c.n_q_heads * c.head_dim) % 16)) return SLED_ERR_ARG;
   if (c.page_size <= 0 || c.n_pages <= 0 || c.max_batch <= 0 || c.max_k < 0 || c.max_step_tokens <= 0)
     return SLED_ERR_ARG;
   if (c.max_step_tokens < c.max_k + 1) return SLED_ERR_ARG;
@@ -797,7 +805,7 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
   const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kd = c.n_kv_heads * c.head_dim, F = c.ffn_dim;
   if ((rc = upload(e, w->tok_emb, static_cast<size_t>(c.vocab) * d * es, &e->tok_emb))) return fail(rc);
   if ((rc = upload(e, w->final_norm, d * es, &e->final_norm))) return fail(rc);
-  const bool q8 = c.linear_weight_bits == 8;
+  const bool q8 = c.linear_weight_bits == 8 || c.linear_weight_bits == 4;
   if (q8 && (!w->wq_scale || !w->wk_scale || !w->wv_scale || !w->wo_scale || !w->w_gate_scale || !w->w_up_scale ||
              !w->w_down_scale))
     return fail(SLED_ERR_ARG);
@@ -874,7 +882,7 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out) 
         tc_activation_init(&e->tc_attn, e->attn_out, static_cast<int>(padT), qd) ||
         tc_activation_init(&e->tc_ffn, e->act_ffn, static_cast<int>(padT), F))
       return fail(SLED_ERR_DEVICE);
-    if (c.linear_weight_bits == 8) {
+    if (q8) {
       struct { TcActivation8* a; int K; } parts[3] = {{&e->a8_norm, d}, {&e->a8_attn, qd}, {&e->a8_ffn, F}};
       for (auto& p : parts) {
         void* data = nullptr;

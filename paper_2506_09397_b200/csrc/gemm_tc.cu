@@ -330,7 +330,7 @@ __global__ void __launch_bounds__(192) tc_gemm_f8_kernel(const __grid_constant__
                                                          int kb_total, int kb_per_split, int lo_row0,
                                                          const float* __restrict__ wscale, const float* __restrict__ ascale,
                                                          float* __restrict__ out, long long split_stride, int32_t* error,
-                                                         TcEpilogue epi) {
+                                                         TcEpilogue epi, int w4) {
   using L = F8SmemLayout<TN_MAX>;
   constexpr int SW = L::kWStages, SA = L::kAStages;
   constexpr int kTmemCols = TN_MAX <= 32 ? 64 : TN_MAX <= 64 ? 128 : 256;   // W * hi | W * lo, TN_MAX columns each
@@ -380,7 +380,9 @@ __global__ void __launch_bounds__(192) tc_gemm_f8_kernel(const __grid_constant__
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_last));
       auto load_w = [&](int kb, int st) {
-        mbar_expect_tx(bar_w_full + 8 * st, kWStageBytes);
+        // 4-bit weights: the copy reads 8 KB of nibbles and spreads them over the 16 KB stage (every 16 bytes of
+        // shared memory hold 16 nibbles and 8 unused bytes); the bytes counted are the ones read
+        mbar_expect_tx(bar_w_full + 8 * st, w4 ? kWStageBytes / 2 : kWStageBytes);
         tma_load_2d(base + st * kWStageBytes, &map_w, 0, (m_tile * kb_total + kb0 + kb) * kBlockM, bar_w_full + 8 * st, pol_first);
       };
       auto load_a = [&](int kb, int st) {
@@ -408,7 +410,9 @@ __global__ void __launch_bounds__(192) tc_gemm_f8_kernel(const __grid_constant__
     if (lane == 0) {
       // instruction descriptor: fp32 accumulate, e4m3 x e4m3 (format code 0 for both), K-major, M = 128, and
       // N = the whole activation stage - hi rows and lo rows in one instruction, their sums side by side
-      const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>((2 * TN_MAX) >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+      // (4-bit weights: format code 5, e2m1, for the weight operand; a k-step is still 32 bytes of the swizzled row)
+      const uint32_t idesc = (1u << 4) | (w4 ? (5u << 7) : 0u) | (static_cast<uint32_t>((2 * TN_MAX) >> 3) << 17) |
+                             (static_cast<uint32_t>(kBlockM >> 4) << 24);
       for (int kb = 0; kb < nkb; ++kb) {
         const int ws = kb % SW, as = kb % SA;
         if (!mbar_wait(bar_w_full + 8 * ws, (kb / SW) & 1, error, 2, abort_slot)) { ok = false; break; }
@@ -538,6 +542,19 @@ __global__ void __launch_bounds__(256) retile_f8_kernel(const uint8_t* __restric
     const int r = i / kBlockK8, b = i % kBlockK8;
     const int n = mt * kBlockM + r, k = kb * kBlockK8 + b;
     out[i] = (n < N && k < K) ? src[static_cast<long long>(n) * K + k] : static_cast<uint8_t>(0);
+  }
+}
+
+// row-major e2m1 nibbles [N][K / 2] bytes -> tiles of 128 rows x 64 bytes (128 k), zero where the matrix ends
+__global__ void __launch_bounds__(256) retile_f4_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int N, int K,
+                                                        int n_kslabs) {
+  constexpr int kRowBytes = kBlockK8 / 2;
+  const int kb = blockIdx.x, mt = blockIdx.y;
+  uint8_t* out = dst + (static_cast<long long>(mt) * n_kslabs + kb) * (kBlockM * kRowBytes);
+  for (int i = threadIdx.x; i < kBlockM * kRowBytes; i += blockDim.x) {
+    const int r = i / kRowBytes, b = i % kRowBytes;
+    const int n = mt * kBlockM + r, k = kb * kBlockK8 + 2 * b;   // K is even: a byte's two entries end together
+    out[i] = (n < N && k < K) ? src[static_cast<long long>(n) * (K / 2) + k / 2] : static_cast<uint8_t>(0);
   }
 }
 
@@ -882,6 +899,26 @@ int make_map_u8(CUtensorMap* map, const void* ptr, long long rows, int K, int bo
   return 0;
 }
 
+// tiles of 128 rows x 128 nibbles (64 bytes a row in global memory): the element type "16 x 4 bits, 16-byte aligned"
+// lets the copy write each 8 bytes of nibbles into the first half of a 16-byte piece of shared memory
+int make_map_u4(CUtensorMap* map, const void* ptr, long long rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return -1;
+  if (reinterpret_cast<uintptr_t>(ptr) & 31) return -1;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(kBlockK8), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(kBlockK8 / 2)};
+  cuuint32_t box[2] = {kBlockK8, kBlockM};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    std::fprintf(stderr, "sled: cuTensorMapEncodeTiled (nibbles) failed (%d) rows=%lld\n", static_cast<int>(r), rows);
+    return -1;
+  }
+  return 0;
+}
+
 }  // namespace
 
 int tc_wait_probe_launch(int32_t* error, long long limit_cycles, cudaStream_t s) {
@@ -924,6 +961,25 @@ int tc_weight_init_f8(TcWeight* w, const void* rowmajor_bytes, void* tiled, cons
   w->N = N;
   w->K = K;
   w->f8 = true;
+  w->ready = true;
+  return 0;
+}
+
+size_t tc_weight_f4_tiled_bytes(int N, int K) {
+  return static_cast<size_t>((N + kBlockM - 1) / kBlockM) * ((K + kBlockK8 - 1) / kBlockK8) * (kWStageBytes / 2);
+}
+
+int tc_weight_init_f4(TcWeight* w, const void* rowmajor_nibbles, void* tiled, const float* scale, int N, int K) {
+  if (K % 16 || !scale || (reinterpret_cast<uintptr_t>(tiled) & 31)) return -1;
+  const int n_mtiles = (N + kBlockM - 1) / kBlockM, n_kslabs = (K + kBlockK8 - 1) / kBlockK8;
+  retile_f4_kernel<<<dim3(n_kslabs, n_mtiles), 256>>>(static_cast<const uint8_t*>(rowmajor_nibbles), static_cast<uint8_t*>(tiled), N, K, n_kslabs);
+  if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+  if (make_map_u4(&w->map8, tiled, static_cast<long long>(n_mtiles) * n_kslabs * kBlockM)) return -1;
+  w->scale = scale;
+  w->N = N;
+  w->K = K;
+  w->f8 = true;
+  w->f4 = true;
   w->ready = true;
   return 0;
 }
@@ -1038,7 +1094,7 @@ static int launch_f8(const TcWeight& w, const TcActivation8& a, int box, int T, 
   cfg.numAttrs = 1;
   const long long stride = split_stride;
   cudaError_t err = cudaLaunchKernelEx(&cfg, tc_gemm_f8_kernel<TN_MAX>, w.map8, a.map[box], T, w.N, kb_total, kb_per, a.rows, w.scale,
-                                       static_cast<const float*>(a.scale), out, stride, error, epi);
+                                       static_cast<const float*>(a.scale), out, stride, error, epi, w.f4 ? 1 : 0);
   return err == cudaSuccess ? 1 : -1;
 }
 

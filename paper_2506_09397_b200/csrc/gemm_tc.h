@@ -19,6 +19,10 @@ struct TcWeight {       // [N][K] bf16 weights, stored as 128 x 64 tiles of 16 K
   CUtensorMap map8;
   const float* scale = nullptr;
   bool f8 = false;
+  // 4-bit weights (tc_weight_init_f4): e2m1 nibbles, two per byte, as 128 x 128 tiles of 8 KB behind map8 (whose
+  // element type makes the copy spread every 8 bytes of nibbles over 16 bytes of shared memory, the form the fp8
+  // kind of MMA reads 4-bit operands in); f8 is set as well: everything but the weight operand is the 8-bit path
+  bool f4 = false;
 };
 
 struct TcActivation8 {  // an activation tensor as two e4m3 parts per element and one fp32 scale per token (see
@@ -57,6 +61,11 @@ int tc_weight_init(TcWeight* w, const void* rowmajor, void* tiled, int N, int K)
 // 0x7f / 0xff (NaN in e4m3) must not occur.
 size_t tc_weight_f8_tiled_bytes(int N, int K);
 int tc_weight_init_f8(TcWeight* w, const void* rowmajor_bytes, void* tiled, const float* scale, int N, int K);
+// The same for e2m1 nibbles [N][K / 2] bytes (row-major, device; element k of a row in byte k / 2, even k in the low
+// half; K a multiple of 16): W[n][k] = scale[n] * e2m1(nibble).  `tiled` (32-byte aligned) holds
+// tc_weight_f4_tiled_bytes(N, K) bytes.
+size_t tc_weight_f4_tiled_bytes(int N, int K);
+int tc_weight_init_f4(TcWeight* w, const void* rowmajor_nibbles, void* tiled, const float* scale, int N, int K);
 // `data`: 2 * rows * K bytes, `scale`: rows floats (device, zero-initialised by the caller); rows a multiple of 128
 int tc_activation8_init(TcActivation8* a, void* data, float* scale, int rows, int K);
 // a[T][K] bf16 (device) -> the two e4m3 parts and the token scales of `dst`; returns kernels launched or < 0

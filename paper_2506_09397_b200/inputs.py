@@ -125,22 +125,48 @@ def from_e4m3_rows(q: torch.Tensor, scale: torch.Tensor) -> torch.Tensor:
     return q.view(torch.float8_e4m3fn).to(torch.float32) * scale[:, None]
 
 
-def quantize_linear_weights(w: dict, dequantised: bool = True):
-    """(weights for the 8-bit path, the same model with its linear layers as fp32 matrices - or None when
-    `dequantised` is off).  The first holds e4m3 bytes and `<name>_scale` for the linear layers and the LM head,
-    everything else as in `w`; the second is what those bytes mean, for whoever wants to compute with them in
-    another way."""
+E2M1_VALUES = (0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0)   # magnitudes of the 4-bit float (1 sign, 2 exponent, 1 mantissa bit)
+
+
+def to_e2m1_rows(w: torch.Tensor):
+    """Storage format of the 4-bit weight path: every row divided by its scale = max|row| / 6 and rounded to the
+    nearest e2m1 value (codes 0..7 = E2M1_VALUES, bit 3 = sign), two codes per byte, the even column in the low half.
+    Returns (bytes uint8 [N, K / 2], scale fp32 [N]); K must be even."""
+    w32 = w.to(torch.float32)
+    assert w32.shape[1] % 2 == 0
+    scale = w32.abs().amax(dim=1) / 6.0
+    scale = torch.where(scale > 0, scale, torch.ones_like(scale))
+    x = w32 / scale[:, None]
+    grid = torch.tensor(E2M1_VALUES, device=w32.device)
+    code = torch.bucketize(x.abs(), (grid[1:] + grid[:-1]) / 2).to(torch.uint8)      # nearest magnitude
+    code = code | ((x < 0) & (code > 0)).to(torch.uint8) * 8
+    return (code[:, 0::2] | (code[:, 1::2] << 4)).contiguous(), scale.contiguous()
+
+
+def from_e2m1_rows(q: torch.Tensor, scale: torch.Tensor) -> torch.Tensor:
+    """The matrix those nibbles and scales stand for, in fp32."""
+    table = torch.tensor(E2M1_VALUES + tuple(-v for v in E2M1_VALUES), device=q.device)
+    codes = torch.stack([q & 15, q >> 4], dim=2).reshape(q.shape[0], -1).long()
+    return table[codes] * scale[:, None]
+
+
+def quantize_linear_weights(w: dict, dequantised: bool = True, bits: int = 8):
+    """(weights for the 8-bit - or, bits = 4, the 4-bit - path, the same model with its linear layers as fp32
+    matrices - or None when `dequantised` is off).  The first holds e4m3 bytes (e2m1 nibbles) and `<name>_scale` for
+    the linear layers and the LM head, everything else as in `w`; the second is what those bytes mean, for whoever
+    wants to compute with them in another way."""
+    to_rows, from_rows = (to_e4m3_rows, from_e4m3_rows) if bits == 8 else (to_e2m1_rows, from_e2m1_rows)
     q, deq = dict(w), (dict(w) if dequantised else None)
-    b, sc = to_e4m3_rows(w["lm_head"])
+    b, sc = to_rows(w["lm_head"])
     q["lm_head"], q["lm_head_scale"] = b, sc
     if dequantised:
-        deq["lm_head"] = from_e4m3_rows(b, sc)
+        deq["lm_head"] = from_rows(b, sc)
     for name in LINEAR_NAMES:
-        pairs = [to_e4m3_rows(t) for t in w[name]]
+        pairs = [to_rows(t) for t in w[name]]
         q[name] = [p[0] for p in pairs]
         q[name + "_scale"] = [p[1] for p in pairs]
         if dequantised:
-            deq[name] = [from_e4m3_rows(*p) for p in pairs]
+            deq[name] = [from_rows(*p) for p in pairs]
     return q, deq
 
 

@@ -24,7 +24,7 @@ def _full_step(shape, batch, ks, ctx, seed, check, greedy=False, gpu_vs_rounded=
         each flip is a full rounding step, so ahead of the next rounding the two differ by 1e-4, which flips one in
         forty there, and after three or four rounding points the two round independently;
       * decisions bit-exact on the GPU's own logits.
-    weight_bits = 8: the engine gets the linear layers as e4m3 bytes with row scales, the oracle the fp32 matrices
+    weight_bits = 8 (4): the engine gets the linear layers as e4m3 bytes (e2m1 nibbles) with row scales, the oracle the fp32 matrices
     those bytes stand for; the device then hands its activations to fp8 MMAs as two e4m3 parts per element, whose
     eight significant bits are compared with the oracle's bf16-rounding mode in the same way."""
     if gpu_vs_rounded is None:
@@ -34,9 +34,9 @@ def _full_step(shape, batch, ks, ctx, seed, check, greedy=False, gpu_vs_rounded=
     T = sum(k + 1 for k in ks)
     n_pages = sum((c + k + 1 + 15) // 16 for c, k in zip(ctx, ks)) + 8
     w_orc, shape_orc = w, shape
-    if weight_bits == 8:
+    if weight_bits in (8, 4):
         from dataclasses import replace
-        w, deq = I.quantize_linear_weights(w)
+        w, deq = I.quantize_linear_weights(w, bits=weight_bits)
         w_orc = {k: ([t.float() for t in v] if isinstance(v, list) else v.float()) for k, v in deq.items()}
         shape_orc = replace(shape, weight_dtype="fp32")
         del deq
@@ -137,6 +137,20 @@ def test_llama8b_shapes_two_layers_8bit_weights():
     ks = I.draw_k(16, list(range(2, 9)), 2)
     ctx = I.draw_context_lengths(16, 256, 2048, 2)
     _full_step(shape, 16, ks, ctx, 2, check=_pick(ks, ctx, 2), weight_bits=8, gpu_vs_exact=W8_VS_EXACT, gpu_vs_rounded=W8_VS_ROUNDED)
+
+
+def test_llama8b_shapes_two_layers_4bit_weights():
+    # the same shapes with the linear layers as e2m1 nibbles: the weight tiles reach shared memory through the copy
+    # that spreads 8 bytes of nibbles over 16, everything else is the 8-bit path
+    from dataclasses import replace
+    shape = replace(I.LLAMA_8B, n_layers=2)
+    ks = I.draw_k(16, [3, 5, 8], 0)
+    ctx = I.draw_context_lengths(16, 512, 4096, 0)
+    _full_step(shape, 16, ks, ctx, 0, check=_pick(ks, ctx) | {0}, weight_bits=4, gpu_vs_exact=W8_VS_EXACT, gpu_vs_rounded=W8_VS_ROUNDED)
+    _full_step(shape, 1, [5], [3000], 4, check={0}, weight_bits=4, gpu_vs_exact=W8_VS_EXACT, gpu_vs_rounded=W8_VS_ROUNDED)
+    ks = I.draw_k(64, [3, 5, 8], 1)
+    ctx = I.draw_context_lengths(64, 512, 4096, 1)
+    _full_step(shape, 64, ks, ctx, 1, check=_pick(ks, ctx, 2), weight_bits=4, gpu_vs_exact=W8_VS_EXACT, gpu_vs_rounded=W8_VS_ROUNDED)
 
 
 def test_llama8b_step_batch16():

@@ -212,3 +212,26 @@ def test_e4m3_storage_format_round_trip():
     table = I.from_e4m3_rows(torch.arange(256, dtype=torch.uint8)[:, None], torch.ones(256))[:, 0]
     assert float(table[0x01]) == 2.0 ** -9 and float(table[0x08]) == 2.0 ** -6 and float(table[0x38]) == 1.0
     assert float(table[0x7e]) == 448.0 and float(table[0xb8]) == -1.0
+
+
+def test_e2m1_storage_format_round_trip():
+    # what inputs.to_e2m1_rows stores: the nearest of the sixteen e2m1 values to the row-scaled entry (neighbouring
+    # values are at most 2 apart, so within 1 of it), the row's largest entry on +-6, the even column in the low half
+    # of a byte; the code table is the 4-bit float's definition (exponent bias 1, one mantissa bit, subnormal 0.5)
+    import torch
+    from paper_2506_09397_b200 import inputs as I
+    w = torch.randn(64, 256, generator=torch.Generator().manual_seed(2)) * 0.02
+    b, sc = I.to_e2m1_rows(w)
+    back = I.from_e2m1_rows(b, sc)
+    assert b.dtype == torch.uint8 and tuple(b.shape) == (64, 128)
+    assert torch.all((back - w).abs() <= sc[:, None] * 1.0 + 1e-9)
+    assert torch.allclose(back.abs().amax(dim=1), w.abs().amax(dim=1))
+    small = (w.abs() <= sc[:, None] * 2.0)                      # up to 2 the values are half a unit apart
+    assert torch.all((back - w).abs()[small] <= (sc[:, None] * 0.25 + 1e-9).expand_as(w)[small])
+    table = I.from_e2m1_rows(torch.arange(16, dtype=torch.uint8)[:, None], torch.ones(16))
+    for code in range(16):
+        e, m, sign = (code >> 1) & 3, code & 1, -1.0 if code & 8 else 1.0
+        want = sign * (0.5 * m if e == 0 else (1 + 0.5 * m) * 2.0 ** (e - 1))
+        assert float(table[code, 0]) == want and float(table[code, 1]) == 0.0     # high half empty
+    one = I.from_e2m1_rows(torch.tensor([[0x2f]], dtype=torch.uint8), torch.ones(1))
+    assert one.tolist() == [[-6.0, 1.0]]                       # low half first
