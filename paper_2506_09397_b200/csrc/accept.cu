@@ -136,6 +136,15 @@ __device__ __forceinline__ void fixed_exp_pair(float z0, float z1, const Exp2Con
   e1 = __float2ull_rz(s1);
 }
 
+// 16-byte load with an L2 eviction policy (createpolicy): rows that will be read again are kept, rows and draft
+// rows on their last reading make room first
+__device__ __forceinline__ float4 ld4_policy(const float* p, uint64_t policy) {
+  float4 v;
+  asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(policy));
+  return v;
+}
+
 __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -229,6 +238,10 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
   // the draft rows are the caller's memory: any 4-byte aligned address is legal, 16-byte loads need more
   const bool q_vec = vec && ((reinterpret_cast<uintptr_t>(qbase) & (q16 ? 7 : 15)) == 0);   // four entries per load
   int xphase = 0;   // parity of the sum exchange slots
+  uint64_t pol_keep, pol_last;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_last));
+  if (kCache) pol_keep = pol_last;   // a row is read from memory once
 
   for (int j = 0; j <= k; ++j) {
     const float* z = a.logits + static_cast<int64_t>(row0 + j) * V;
@@ -261,10 +274,10 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
       };
       int v = w_lo + lane * kVec;
       for (; v + 3 * kStep < w_hi; v += 4 * kStep) {
-        const float4 x0 = *reinterpret_cast<const float4*>(z + v);
-        const float4 x1 = *reinterpret_cast<const float4*>(z + v + kStep);
-        const float4 x2 = *reinterpret_cast<const float4*>(z + v + 2 * kStep);
-        const float4 x3 = *reinterpret_cast<const float4*>(z + v + 3 * kStep);
+        const float4 x0 = ld4_policy(z + v, pol_keep);
+        const float4 x1 = ld4_policy(z + v + kStep, pol_keep);
+        const float4 x2 = ld4_policy(z + v + 2 * kStep, pol_keep);
+        const float4 x3 = ld4_policy(z + v + 3 * kStep, pol_keep);
         look(x0); look(x1); look(x2); look(x3);
         if constexpr (kCache) {
           *reinterpret_cast<float4*>(zc + (v - b_lo)) = x0;
@@ -274,7 +287,7 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
         }
       }
       for (; v < w_hi; v += kStep) {
-        const float4 x0 = *reinterpret_cast<const float4*>(z + v);
+        const float4 x0 = ld4_policy(z + v, pol_keep);
         look(x0);
         if constexpr (kCache) *reinterpret_cast<float4*>(zc + (v - b_lo)) = x0;
       }
@@ -432,11 +445,11 @@ __global__ void __launch_bounds__(kThreads, kThreads == 512 ? 3 : 1) accept_kern
     auto fetch = [&](int v0, float (&zs)[kVec], float (&qs)[kVec]) {
       if (vec) {   // V % 4 == 0: a lane's four entries are inside the row together
         if constexpr (!kCache) {
-          const float4 z4 = *reinterpret_cast<const float4*>(z + v0);
+          const float4 z4 = ld4_policy(z + v0, pol_last);
           zs[0] = z4.x; zs[1] = z4.y; zs[2] = z4.z; zs[3] = z4.w;
         }
         if (use_q && q_vec && !q16) {
-          const float4 q4 = *reinterpret_cast<const float4*>(static_cast<const float*>(qbase) + q_off + v0);
+          const float4 q4 = ld4_policy(static_cast<const float*>(qbase) + q_off + v0, pol_last);
           qs[0] = q4.x; qs[1] = q4.y; qs[2] = q4.z; qs[3] = q4.w;
         } else if (use_q && q_vec) {
           const uint2 q4 = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(qbase) + q_off + v0);
