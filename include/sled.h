@@ -171,7 +171,9 @@ typedef struct sled_stats {
 
 /* ---- the three calls of the verification service ---------------------------------- */
 
-/* Creates an engine: checks cfg, allocates weights, KV pool and workspaces on
+/* Creates an engine around the one target model that all devices share (Section 3.2: the
+ * server holds a single large model; Section 3.4: it verifies the drafts of many devices
+ * together): checks cfg, allocates weights, KV pool and workspaces on
  * cfg->device_index, copies the weights.  Errors: SLED_ERR_ARG, SLED_ERR_NO_DEVICE,
  * SLED_ERR_DEVICE (allocation failed: nothing is left allocated). */
 int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out);
@@ -188,7 +190,10 @@ int sled_init(const sled_weights* w, const sled_config* cfg, sled_engine** out);
 int sled_verify_batch(sled_engine* e, const sled_request* reqs, int32_t n_reqs, uint64_t seed,
                       sled_result* results);
 
-/* Closes a context: its pages return to the pool. */
+/* Closes a context - a device's conversation has ended, or the device has left (Section 3.2:
+ * each device is served on its own sequence) - and returns its pages to the pool.  The paper
+ * leaves cache management to future work (Section 5); this call is what frees it here.
+ * Errors: SLED_ERR_UNKNOWN_CTX. */
 int sled_release(sled_engine* e, uint64_t ctx_id);
 
 /* ---- what makes the three usable --------------------------------------------------- */

@@ -593,7 +593,7 @@ static int launch_accept_t(const AcceptArgs& a, int C, cudaStream_t s) {
 
 // Whether the cached form applies with C blocks per request: sampling, 16-byte aligned rows, and a block's share of
 // a row within kCacheBytes.  (More blocks per request than occupancy asks for, only to make a row fit, measured slower
-// on 512 requests: a row then costs six exchanges between eight blocks, and those, not the arithmetic, set the pace.)
+// on 512 requests: a row then costs three exchanges between eight blocks, and those, not the arithmetic, set the pace.)
 template <int kThreads>
 static bool cached_form_fits(const AcceptArgs& a, int C) {
   if (a.greedy || (a.V & 3) || (reinterpret_cast<uintptr_t>(a.logits) & 15)) return false;
