@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <queue>
 #include <vector>
 
 #include "../../include/sled.h"
@@ -354,20 +355,59 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
       per_item *= 1.5;   // fewer, longer chunks until the partial results fit
     }
   } else {
-    int64_t chunk = 256;
-    for (;;) {
+    // Many requests: every request is cut into equal parts of about the same cost, and that cost is the one whose
+    // items, handed out longest first to the resident blocks as these retire, end soonest by a small model: an
+    // item costs its key tiles (weighted as above) plus a fixed part worth about six tiles when its request is
+    // split (set-up, partial results, their merge) and three when it is not - the figures that make the model
+    // follow the measured launch times at 64 and 128 requests (2048 against 4096 keys: 0.47 against 0.57 ms).
+    auto parts_for = [&](double per_item, std::vector<int64_t>& out) {   // parts of about per_item cost each
       int64_t items = 0;
       for (int i = 0; i < B; ++i) {
-        chunk_of[i] = chunk;
-        items += (n_keys[i] + chunk - 1) / chunk * Hkv;
+        const int64_t tiles = (n_keys[i] + 63) / 64;
+        const int64_t nc = std::max<int64_t>(1, std::min<int64_t>(static_cast<int64_t>(std::ceil(cost[i] / per_item)),
+                                                                  std::max<int64_t>(1, tiles / 2)));
+        out[i] = (tiles + nc - 1) / nc * 64;
+        items += (n_keys[i] + out[i] - 1) / out[i] * Hkv;
       }
+      return items;
+    };
+    auto end_time = [&](const std::vector<int64_t>& chunks) {
+      std::vector<std::pair<bool, double>> c;   // (heavy, cost)
+      for (int i = 0; i < B; ++i) {
+        const int64_t nc = (n_keys[i] + chunks[i] - 1) / chunks[i];
+        for (int64_t j = 0; j < nc; ++j) {
+          const int64_t cnt = std::min<int64_t>(chunks[i], n_keys[i] - j * chunks[i]);
+          const double w = cost[i] * cnt / static_cast<double>(n_keys[i]) + (nc > 1 ? 6.0 : 3.0);
+          c.emplace_back(heavy(i), w);   // stands for the Hkv equal items of this part: they start side by side
+        }
+      }
+      std::sort(c.begin(), c.end(), [](const auto& x, const auto& y) { return x.first != y.first ? x.first : x.second > y.second; });
+      std::priority_queue<double, std::vector<double>, std::greater<double>> free_at;
+      for (int64_t k = 0; k < std::max<int64_t>(1, slots / Hkv); ++k) free_at.push(0.0);
+      double end = 0.0;
+      for (const auto& it : c) {
+        const double t = free_at.top() + it.second;
+        free_at.pop();
+        free_at.push(t);
+        end = std::max(end, t);
+      }
+      return end;
+    };
+    std::vector<int64_t> trial(B);
+    double best = -1.0;
+    double max_cost = 1.0;
+    for (int i = 0; i < B; ++i) max_cost = std::max(max_cost, cost[i]);
+    for (double per_item = 4.0;; per_item *= 2.0) {   // from 256 keys on (a finer grid measured no better)
+      const bool whole = per_item >= max_cost;           // nobody is split any more: the last candidate
+      const int64_t items = parts_for(whole ? max_cost : per_item, trial);
+      std::swap(trial, chunk_of);
       const bool fits = part_rows_of() <= e->part_rows_cap;
-      if ((items <= 2 * slots && fits) || chunk >= (1 << 30)) break;
-      // doubling would still leave enough items, or we must shrink the partial rows
-      int64_t items2 = 0;
-      for (int i = 0; i < B; ++i) items2 += ((n_keys[i] + 2 * chunk - 1) / (2 * chunk)) * Hkv;
-      if (!fits || items2 >= slots) chunk *= 2;
-      else break;
+      std::swap(trial, chunk_of);
+      if (fits && (items <= 4 * slots || whole)) {
+        const double end = end_time(trial);
+        if (best < 0.0 || end < best) { best = end; chunk_of = trial; }
+      }
+      if (whole) break;
     }
   }
   struct It { int req, kvh, start, count; double cost; bool heavy; };
