@@ -299,11 +299,11 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
     std::memcpy(h_pt + h_ptoff[i], c->pages.data(), sizeof(int32_t) * np);
   }
 
-  // Attention work items: (request, KV head, chunk of keys).  The chunk length is chosen per request.
-  // Few requests (every item can be resident at once, two blocks per SM): a request gets chunks in proportion to
-  // its cost - key tiles, weighted up when it has more than 32 query rows, whose tiles take the tensor pipes
-  // longer - so that all blocks end together.  Many requests: one common chunk length, doubled until the item
-  // count is near the machine size; the hardware hands items out as blocks retire.
+  // Attention work items: (request, KV head, chunk of keys).  The chunk length is chosen per request: every request
+  // is cut into equal parts.  Candidates are the one-wave plan (few requests: every item resident at once, two blocks
+  // per SM, parts in proportion to a request's cost - key tiles, weighted up when it has more than 32 query rows,
+  // whose tiles take the tensor pipes longer - so that all blocks end together) and plans of several waves, which
+  // the hardware hands out as blocks retire; a small model of that picks among them (below).
   const int group = e->cfg.n_q_heads / Hkv;
   int max_rows = 0;
   for (int i = 0; i < B; ++i) max_rows = std::max(max_rows, plan[i].n * group);
@@ -326,40 +326,11 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
     }
     return rows;
   };
-  if (static_cast<int64_t>(B) * Hkv <= slots) {
-    // smallest cost per item for which the items still fit the slots (bisection on a monotone count)
-    auto chunks_at = [&](int i, double per_item) {
-      const int64_t tiles = (n_keys[i] + 63) / 64;
-      const int64_t want = static_cast<int64_t>(std::ceil(cost[i] / per_item));
-      return std::max<int64_t>(1, std::min(want, std::max<int64_t>(1, tiles / 2)));   // chunks of at least 2 tiles
-    };
-    auto items_at = [&](double per_item) {
-      int64_t n = 0;
-      for (int i = 0; i < B; ++i) n += chunks_at(i, per_item) * Hkv;
-      return n;
-    };
-    double lo = 1.0, hi = 1.0;
-    for (int i = 0; i < B; ++i) hi = std::max(hi, cost[i]);
-    for (int it = 0; it < 30 && items_at(lo) > slots; ++it) {
-      const double mid = 0.5 * (lo + hi);
-      if (items_at(mid) > slots) lo = mid; else hi = mid;
-    }
-    double per_item = items_at(lo) <= slots ? lo : hi;
-    for (;;) {
-      for (int i = 0; i < B; ++i) {
-        const int64_t tiles = (n_keys[i] + 63) / 64;
-        const int64_t nc = chunks_at(i, per_item);
-        chunk_of[i] = (tiles + nc - 1) / nc * 64;
-      }
-      if (part_rows_of() <= e->part_rows_cap) break;
-      per_item *= 1.5;   // fewer, longer chunks until the partial results fit
-    }
-  } else {
-    // Many requests: every request is cut into equal parts of about the same cost, and that cost is the one whose
-    // items, handed out longest first to the resident blocks as these retire, end soonest by a small model: an
-    // item costs its key tiles (weighted as above) plus a fixed part worth about six tiles when its request is
-    // split (set-up, partial results, their merge) and three when it is not - the figures that make the model
-    // follow the measured launch times at 64 and 128 requests (2048 against 4096 keys: 0.47 against 0.57 ms).
+  // How the items of a plan end on the resident blocks, by a small model: they are handed out longest first as blocks
+  // retire; an item costs its key tiles (weighted as above) plus a fixed part worth about six tiles when its request
+  // is cut (set-up, partial results, their merge) and three when it is not - the figures that make the model follow
+  // the measured launch times at 64 and 128 requests (2048 against 4096 keys: 0.47 against 0.57 ms).
+  {
     auto parts_for = [&](double per_item, std::vector<int64_t>& out) {   // parts of about per_item cost each
       int64_t items = 0;
       for (int i = 0; i < B; ++i) {
@@ -393,8 +364,41 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
       }
       return end;
     };
-    std::vector<int64_t> trial(B);
     double best = -1.0;
+    if (static_cast<int64_t>(B) * Hkv <= slots) {
+      // one wave: the smallest cost per item for which the items still fit the slots (bisection on a monotone count)
+      auto chunks_at = [&](int i, double per_item) {
+        const int64_t tiles = (n_keys[i] + 63) / 64;
+        const int64_t want = static_cast<int64_t>(std::ceil(cost[i] / per_item));
+        return std::max<int64_t>(1, std::min(want, std::max<int64_t>(1, tiles / 2)));   // chunks of at least 2 tiles
+      };
+      auto items_at = [&](double per_item) {
+        int64_t n = 0;
+        for (int i = 0; i < B; ++i) n += chunks_at(i, per_item) * Hkv;
+        return n;
+      };
+      double lo = 1.0, hi = 1.0;
+      for (int i = 0; i < B; ++i) hi = std::max(hi, cost[i]);
+      for (int it = 0; it < 30 && items_at(lo) > slots; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (items_at(mid) > slots) lo = mid; else hi = mid;
+      }
+      double per_item = items_at(lo) <= slots ? lo : hi;
+      for (;;) {
+        for (int i = 0; i < B; ++i) {
+          const int64_t tiles = (n_keys[i] + 63) / 64;
+          const int64_t nc = chunks_at(i, per_item);
+          chunk_of[i] = (tiles + nc - 1) / nc * 64;
+        }
+        if (part_rows_of() <= e->part_rows_cap) break;
+        per_item *= 1.5;   // fewer, longer chunks until the partial results fit
+      }
+      best = end_time(chunk_of);
+    }
+    // several waves: every request in equal parts of about one cost; the candidate that ends soonest wins (with few
+    // requests that is the one-wave plan up to about 24 of them; at 32 - 36 the uncut requests of one wave differ too
+    // much in length: 0.33 -> 0.29 and 0.47 -> 0.31 ms of attention in a 4-layer step)
+    std::vector<int64_t> trial(B);
     double max_cost = 1.0;
     for (int i = 0; i < B; ++i) max_cost = std::max(max_cost, cost[i]);
     for (double per_item = 4.0;; per_item *= 2.0) {   // from 256 keys on (a finer grid measured no better)
