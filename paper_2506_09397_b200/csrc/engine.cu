@@ -316,7 +316,11 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
   auto heavy = [&](int i) { return !pk->use_tc && plan[i].n * group > 32; };
   for (int i = 0; i < B; ++i) {
     const double passes = pk->use_tc ? 1.0 : (plan[i].n * group + 63) / 64;
-    cost[i] = static_cast<double>((n_keys[i] + 63) / 64) * passes * (heavy(i) ? 1.75 : 1.0);
+    // time per key tile by query rows, from per-block timestamps inside a B=16 step: 1.0 us with up to 16 rows (memory
+    // paces those blocks), 1.15 with up to 32, 1.93 with more (each warp then takes all 64 keys of a tile)
+    const int rows = plan[i].n * group;
+    const double per_tile = pk->use_tc ? 1.0 : rows > 32 ? 1.93 : rows > 16 ? 1.15 : 1.0;
+    cost[i] = static_cast<double>((n_keys[i] + 63) / 64) * passes * per_tile;
   }
   auto part_rows_of = [&]() {
     int64_t rows = 0;
