@@ -118,6 +118,11 @@ def test_llama8b_shapes_two_layers():
     ks = I.draw_k(64, [3, 5, 8], 1)
     ctx = I.draw_context_lengths(64, 512, 4096, 1)
     _full_step(shape, 64, ks, ctx, 1, check=_pick(ks, ctx))
+    # 36 requests: every (request, KV head) item could be resident at once, but the attention items are planned in
+    # several waves (the longest contexts cut, the short ones whole)
+    ks = I.draw_k(36, [3, 5, 8], 3)
+    ctx = I.draw_context_lengths(36, 512, 4096, 3)
+    _full_step(shape, 36, ks, ctx, 3, check=_pick(ks, ctx))
 
 
 def test_llama8b_shapes_two_layers_8bit_weights():
