@@ -12,7 +12,8 @@ pinned host memory (copied in and results copied out inside the timed region).  
 distributions correlated with the target's own logits (`--drafts independent`: from distributions
 that ignore the target).  `roofline` is for the tensor-core linear-layer kernel, the dominant one;
 `kernel_ms` splits an untouched step by kind of kernel from per-launch device timestamps,
-`kernel_ms_serialised` is the same with events between the kernels.  `sweep` repeats the step at
+`kernel_ms_serialised` is the same with events between the kernels.  `independent_drafts` / `greedy` time the same
+step with drafts that ignore the target / with greedy verification.  `sweep` repeats the step at
 other batch sizes (fewer steps, no end-to-end leg), `weights_8bit` / `weights_4bit` with the linear layers'
 weights as e4m3 bytes / e2m1 nibbles (`--weight-bits 8` / `4` runs everything that way).  `--impl reference` times the CPU oracle.
 Under torchrun every rank runs its own replica on its own requests (no data-path collective).
@@ -588,6 +589,12 @@ def run_sled(args):
         s_i = pt.summary(c_i, ms_i, max(5, args.steps // 2), Bn, peaks)
         line["independent_drafts"] = {k: s_i[k] for k in ("ms_per_step", "tokens_per_s", "acceptance_rate", "frac_of_hbm_peak")}
         del d2, q2, r2
+        # greedy verification of the headline's drafts (argmax comparison: the draft rows are not read)
+        pt.eng.set_sampling(1.0, True)
+        c_g, ms_g, _ = pt.timed(reqs_dev, max(5, args.steps // 2), 3)
+        s_g = pt.summary(c_g, ms_g, max(5, args.steps // 2), 0, peaks)
+        line["greedy"] = {k: s_g[k] for k in ("ms_per_step", "tokens_per_s", "acceptance_rate", "frac_of_hbm_peak")}
+        pt.eng.set_sampling(1.0, False)
     if e2e and not args.greedy and not args.no_sweep:
         # the same end-to-end step with the draft rows sent as bf16 (half the bytes; decisions then use the rounded
         # rows); it replaces the point's engine, so it comes last
