@@ -240,6 +240,15 @@ int sled_planner_push(sled_planner* p, uint64_t ticket, uint64_t ctx_id, int32_t
 int32_t sled_planner_next_batch(sled_planner* p, int32_t flush, uint64_t* tickets_out, int32_t cap);
 int32_t sled_planner_queued(sled_planner* p);
 
+/* Host only: how a step's requests are cut into attention work items (request, KV head, chunk of keys) - the paper's
+ * batched verification (Section 3.4) leaves the scheduling of the batch on the GPU open.  n_keys[i]: keys request i
+ * attends to (cached prefix + its k_i + 1 new tokens), q_tokens[i] = k_i + 1, group: query heads per KV head,
+ * resident_blocks: blocks of the attention kernel the GPU holds at once (two per SM), part_rows_cap: most rows of
+ * partial results.  chunk_keys_out[i] (caller-allocated, n_reqs entries): keys per item of request i, a multiple of 64;
+ * a request is cut into ceil(n_keys / chunk) equal parts.  Returns SLED_ERR_ARG on null pointers or non-positive sizes. */
+int sled_debug_plan_attention(const int64_t* n_keys, const int32_t* q_tokens, int32_t n_reqs, int32_t n_kv_heads,
+                              int32_t group, int32_t resident_blocks, int64_t part_rows_cap, int64_t* chunk_keys_out);
+
 /* ---- stand-alone pieces of the step (device-resident operands) ---------------------- */
 
 /* Acceptance only (Eq. 1 + residual / bonus draw) on logits already in device memory.

@@ -51,3 +51,26 @@ class PlannerModel:
         out = [self.queue[p][0] for p in chosen]
         self.queue = [r for p, r in enumerate(self.queue) if p not in set(chosen)]
         return out
+
+
+def attention_plan_end_time(n_keys, q_tokens, chunk_keys, n_kv_heads: int, group: int, resident_blocks: int) -> float:
+    """How long the attention items of a cut take by the planner's model, in key-tile times: a request of n keys and
+    q tokens costs ceil(n / 64) tiles, weighted 1.15 with more than 16 query rows (q * group) and 1.93 with more than
+    32, once per 64 query rows; an item carries its share of that plus 6 when its request is cut and 3 when it is
+    not; the items of one part (one per KV head) start side by side, costly-row requests first, then longest first,
+    each on the group of blocks that is free earliest."""
+    items = []
+    for n, q, c in zip(n_keys, q_tokens, chunk_keys):
+        rows = q * group
+        weight = 1.93 if rows > 32 else 1.15 if rows > 16 else 1.0
+        cost = -(-n // 64) * ((rows + 63) // 64) * weight
+        parts = -(-n // c)
+        for j in range(parts):
+            count = min(c, n - j * c)
+            items.append((rows > 32, cost * count / n + (6.0 if parts > 1 else 3.0)))
+    items.sort(key=lambda it: (not it[0], -it[1]))
+    free_at = [0.0] * max(1, resident_blocks // n_kv_heads)
+    for _, w in items:
+        k = free_at.index(min(free_at))
+        free_at[k] += w
+    return max(free_at)

@@ -33,6 +33,7 @@ EXPORTS = (
     "sled_kvm_commit_tokens", "sled_kvm_history",
     "sled_server_config", "sled_submit", "sled_step", "sled_poll", "sled_queued",
     "sled_planner_create", "sled_planner_destroy", "sled_planner_push", "sled_planner_next_batch", "sled_planner_queued",
+    "sled_debug_plan_attention",
 )
 
 
@@ -135,6 +136,7 @@ def lib():
             "sled_planner_push": (C.c_int, [P, U64, U64, I32]),
             "sled_planner_next_batch": (I32, [P, I32, P, I32]),
             "sled_planner_queued": (I32, [P]),
+            "sled_debug_plan_attention": (C.c_int, [P, P, I32, I32, I32, I32, C.c_int64, P]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -490,3 +492,13 @@ class Planner:
                 self.h = None
         except Exception:
             pass
+
+
+def plan_attention(n_keys, q_tokens, n_kv_heads: int, group: int, resident_blocks: int, part_rows_cap: int):
+    """Keys per attention work item of every request (sled_debug_plan_attention: host only, needs no device)."""
+    nk = np.ascontiguousarray(n_keys, dtype=np.int64)
+    qt = np.ascontiguousarray(q_tokens, dtype=np.int32)
+    out = np.zeros(len(nk), dtype=np.int64)
+    _check(lib().sled_debug_plan_attention(nk.ctypes.data, qt.ctypes.data, len(nk), n_kv_heads, group, resident_blocks,
+                                           part_rows_cap, out.ctypes.data), "sled_debug_plan_attention")
+    return [int(c) for c in out]

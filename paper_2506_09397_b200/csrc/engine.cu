@@ -312,112 +312,11 @@ int pack_step(sled_engine* e, const std::vector<PlanReq>& plan, bool already_cac
   const int64_t slots = (pk->use_tc ? 1LL : 2LL) * e->n_sm;
   std::vector<int64_t> chunk_of(B, 256);
   std::vector<double> cost(B);
-  // the warp-level kernel's tiles take the tensor pipes longer when a request has more than 32 query rows
+  std::vector<int32_t> q_tokens(B);
+  for (int i = 0; i < B; ++i) q_tokens[i] = plan[i].n;
+  plan_attention_chunks(n_keys.data(), q_tokens.data(), B, Hkv, group, slots, pk->use_tc, e->part_rows_cap, chunk_of.data(),
+                        cost.data());
   auto heavy = [&](int i) { return !pk->use_tc && plan[i].n * group > 32; };
-  for (int i = 0; i < B; ++i) {
-    const double passes = pk->use_tc ? 1.0 : (plan[i].n * group + 63) / 64;
-    // time per key tile by query rows, from per-block timestamps inside a B=16 step: 1.0 us with up to 16 rows (memory
-    // paces those blocks), 1.15 with up to 32, 1.93 with more (each warp then takes all 64 keys of a tile)
-    const int rows = plan[i].n * group;
-    const double per_tile = pk->use_tc ? 1.0 : rows > 32 ? 1.93 : rows > 16 ? 1.15 : 1.0;
-    cost[i] = static_cast<double>((n_keys[i] + 63) / 64) * passes * per_tile;
-  }
-  auto part_rows_of = [&]() {
-    int64_t rows = 0;
-    for (int i = 0; i < B; ++i) {
-      const int64_t nc = (n_keys[i] + chunk_of[i] - 1) / chunk_of[i];
-      if (nc > 1) rows += nc * plan[i].n;
-    }
-    return rows;
-  };
-  // How the items of a plan end on the resident blocks, by a small model: they are handed out longest first as blocks
-  // retire; an item costs its key tiles (weighted as above) plus a fixed part worth about six tiles when its request
-  // is cut (set-up, partial results, their merge) and three when it is not - the figures that make the model follow
-  // the measured launch times at 64 and 128 requests (2048 against 4096 keys: 0.47 against 0.57 ms).
-  {
-    auto parts_for = [&](double per_item, std::vector<int64_t>& out) {   // parts of about per_item cost each
-      int64_t items = 0;
-      for (int i = 0; i < B; ++i) {
-        const int64_t tiles = (n_keys[i] + 63) / 64;
-        const int64_t nc = std::max<int64_t>(1, std::min<int64_t>(static_cast<int64_t>(std::ceil(cost[i] / per_item)),
-                                                                  std::max<int64_t>(1, tiles / 2)));
-        out[i] = (tiles + nc - 1) / nc * 64;
-        items += (n_keys[i] + out[i] - 1) / out[i] * Hkv;
-      }
-      return items;
-    };
-    auto end_time = [&](const std::vector<int64_t>& chunks) {
-      std::vector<std::pair<bool, double>> c;   // (heavy, cost)
-      for (int i = 0; i < B; ++i) {
-        const int64_t nc = (n_keys[i] + chunks[i] - 1) / chunks[i];
-        for (int64_t j = 0; j < nc; ++j) {
-          const int64_t cnt = std::min<int64_t>(chunks[i], n_keys[i] - j * chunks[i]);
-          const double w = cost[i] * cnt / static_cast<double>(n_keys[i]) + (nc > 1 ? 6.0 : 3.0);
-          c.emplace_back(heavy(i), w);   // stands for the Hkv equal items of this part: they start side by side
-        }
-      }
-      std::sort(c.begin(), c.end(), [](const auto& x, const auto& y) { return x.first != y.first ? x.first : x.second > y.second; });
-      std::priority_queue<double, std::vector<double>, std::greater<double>> free_at;
-      for (int64_t k = 0; k < std::max<int64_t>(1, slots / Hkv); ++k) free_at.push(0.0);
-      double end = 0.0;
-      for (const auto& it : c) {
-        const double t = free_at.top() + it.second;
-        free_at.pop();
-        free_at.push(t);
-        end = std::max(end, t);
-      }
-      return end;
-    };
-    double best = -1.0;
-    if (static_cast<int64_t>(B) * Hkv <= slots) {
-      // one wave: the smallest cost per item for which the items still fit the slots (bisection on a monotone count)
-      auto chunks_at = [&](int i, double per_item) {
-        const int64_t tiles = (n_keys[i] + 63) / 64;
-        const int64_t want = static_cast<int64_t>(std::ceil(cost[i] / per_item));
-        return std::max<int64_t>(1, std::min(want, std::max<int64_t>(1, tiles / 2)));   // chunks of at least 2 tiles
-      };
-      auto items_at = [&](double per_item) {
-        int64_t n = 0;
-        for (int i = 0; i < B; ++i) n += chunks_at(i, per_item) * Hkv;
-        return n;
-      };
-      double lo = 1.0, hi = 1.0;
-      for (int i = 0; i < B; ++i) hi = std::max(hi, cost[i]);
-      for (int it = 0; it < 30 && items_at(lo) > slots; ++it) {
-        const double mid = 0.5 * (lo + hi);
-        if (items_at(mid) > slots) lo = mid; else hi = mid;
-      }
-      double per_item = items_at(lo) <= slots ? lo : hi;
-      for (;;) {
-        for (int i = 0; i < B; ++i) {
-          const int64_t tiles = (n_keys[i] + 63) / 64;
-          const int64_t nc = chunks_at(i, per_item);
-          chunk_of[i] = (tiles + nc - 1) / nc * 64;
-        }
-        if (part_rows_of() <= e->part_rows_cap) break;
-        per_item *= 1.5;   // fewer, longer chunks until the partial results fit
-      }
-      best = end_time(chunk_of);
-    }
-    // several waves: every request in equal parts of about one cost; the candidate that ends soonest wins (with few
-    // requests that is the one-wave plan up to about 24 of them; at 32 - 36 the uncut requests of one wave differ too
-    // much in length: 0.33 -> 0.29 and 0.47 -> 0.31 ms of attention in a 4-layer step)
-    std::vector<int64_t> trial(B);
-    double max_cost = 1.0;
-    for (int i = 0; i < B; ++i) max_cost = std::max(max_cost, cost[i]);
-    for (double per_item = 4.0;; per_item *= 2.0) {   // from 256 keys on (a finer grid measured no better)
-      const bool whole = per_item >= max_cost;           // nobody is split any more: the last candidate
-      const int64_t items = parts_for(whole ? max_cost : per_item, trial);
-      std::swap(trial, chunk_of);
-      const bool fits = part_rows_of() <= e->part_rows_cap;
-      std::swap(trial, chunk_of);
-      if (fits && (items <= 4 * slots || whole)) {
-        const double end = end_time(trial);
-        if (best < 0.0 || end < best) { best = end; chunk_of = trial; }
-      }
-      if (whole) break;
-    }
-  }
   struct It { int req, kvh, start, count; double cost; bool heavy; };
   std::vector<It> its;
   int part_rows = 0;

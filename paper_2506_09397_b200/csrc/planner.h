@@ -44,4 +44,13 @@ class Planner {
   std::deque<QueuedRequest> q_;
 };
 
+// The cut of a step's requests into attention work items: chunk_out[i] = keys per item of request i (a multiple of
+// 64; the request has ceil(n_keys[i] / chunk_out[i]) items per KV head).  n_keys[i]: keys request i attends to,
+// q_tokens[i]: its query tokens (k + 1), group: query heads per KV head, slots: blocks resident at once,
+// uniform_tiles: every key tile costs the same whatever the number of query rows (the tcgen05 kernel),
+// part_rows_cap: most rows of partial results (one per chunk and query token of every request that is cut).
+// cost_out (may be null): the cost the plan assigns to each whole request, in key tiles.
+void plan_attention_chunks(const int64_t* n_keys, const int32_t* q_tokens, int B, int Hkv, int group, int64_t slots,
+                           bool uniform_tiles, int64_t part_rows_cap, int64_t* chunk_out, double* cost_out);
+
 }  // namespace sled

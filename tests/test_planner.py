@@ -90,3 +90,88 @@ def test_planner_refuses_bad_configurations():
                  (B.SLED_BATCH_CONTINUOUS, 0, 0, 10), (B.SLED_BATCH_CONTINUOUS, 0, 4, 0)):
         with pytest.raises(B.SledError):
             B.Planner(*args)
+
+
+# ---- the cut of a step's requests into attention work items (host only) ----------------------------------------
+def _bench_like(b, seed=0):
+    from paper_2506_09397_b200 import inputs as I
+    ks = I.draw_k(b, [3, 5, 8], seed)
+    ctx = I.draw_context_lengths(b, 512, 4096, seed)
+    return [c + k + 1 for c, k in zip(ctx, ks)], [k + 1 for k in ks]
+
+
+@pytest.mark.parametrize("b", [1, 3, 16, 36, 64, 128])
+def test_attention_plan_is_a_valid_cut(b):
+    # every request in equal parts of whole 64-key tiles, at least two tiles a part when it is cut, the partial
+    # results within the room that there is
+    n_keys, q_tok = _bench_like(b, seed=b)
+    for cap in (1 << 20, 400, 0):
+        chunks = B.plan_attention(n_keys, q_tok, 8, 4, 296, cap)
+        part_rows = 0
+        for n, q, c in zip(n_keys, q_tok, chunks):
+            parts = -(-n // c)
+            assert c % 64 == 0 and c > 0
+            assert (parts - 1) * c < n <= parts * c
+            if parts > 1:
+                assert c >= 128
+                assert c - 64 < -(-n // parts) + 63           # equal parts: no part a whole tile longer than need be
+                part_rows += parts * q
+        assert part_rows <= cap
+        if cap == 0:
+            assert all(c >= n for n, c in zip(n_keys, chunks))
+
+
+def test_attention_plan_follows_what_was_measured():
+    # the configurations that were timed with forced chunk lengths (8B shape, contexts 512..4096, 296 resident blocks):
+    # one wave of items for 16 requests; at 36 and 64 requests the long contexts are cut and the short ones are not;
+    # at 128 requests nothing is cut
+    n_keys, q_tok = _bench_like(16)
+    chunks = B.plan_attention(n_keys, q_tok, 8, 4, 296, 1 << 20)
+    assert sum(-(-n // c) for n, c in zip(n_keys, chunks)) * 8 <= 296
+    for b in (36, 64):
+        n_keys, q_tok = _bench_like(b)
+        chunks = B.plan_attention(n_keys, q_tok, 8, 4, 296, 1 << 20)
+        cut = [n for n, c in zip(n_keys, chunks) if c < n]
+        whole = [n for n, c in zip(n_keys, chunks) if c >= n]
+        assert cut and whole and sum(cut) / len(cut) > 1.3 * sum(whole) / len(whole)
+        assert 296 < sum(-(-n // c) for n, c in zip(n_keys, chunks)) * 8 <= 4 * 296
+    n_keys, q_tok = _bench_like(128)
+    chunks = B.plan_attention(n_keys, q_tok, 8, 4, 296, 1 << 20)
+    assert all(c >= n for n, c in zip(n_keys, chunks))
+
+
+@pytest.mark.parametrize("b,seed", [(8, 1), (24, 2), (40, 3), (64, 4), (100, 5)])
+def test_attention_plan_ends_no_later_than_its_candidates(b, seed):
+    # by the planner's own model (restated with plain lists), the chosen cut ends no later than any cut of its
+    # candidate family: every request in equal parts of about one cost, that cost doubling from 4 key tiles up to
+    # "nobody is cut" (candidates of more than four items per resident block are not considered)
+    n_keys, q_tok = _bench_like(b, seed)
+    chosen = B.plan_attention(n_keys, q_tok, 8, 4, 296, 1 << 20)
+    t_chosen = PM.attention_plan_end_time(n_keys, q_tok, chosen, 8, 4, 296)
+    costs = []
+    for n, q in zip(n_keys, q_tok):
+        rows = q * 4
+        costs.append(-(-n // 64) * ((rows + 63) // 64) * (1.93 if rows > 32 else 1.15 if rows > 16 else 1.0))
+    per_item, seen = 4.0, 0
+    while True:
+        whole = per_item >= max(costs)
+        alt = []
+        for n, c in zip(n_keys, costs):
+            tiles = -(-n // 64)
+            parts = 1 if whole else max(1, min(int(np.ceil(c / per_item)), max(1, tiles // 2)))
+            alt.append(-(-tiles // parts) * 64)
+        n_items = sum(-(-n // c) for n, c in zip(n_keys, alt)) * 8
+        if whole or n_items <= 4 * 296:
+            seen += 1
+            assert t_chosen <= PM.attention_plan_end_time(n_keys, q_tok, alt, 8, 4, 296) * (1 + 1e-9), per_item
+        if whole:
+            break
+        per_item *= 2.0
+    assert seen >= 2
+
+
+def test_attention_plan_refuses_bad_arguments():
+    with pytest.raises(B.SledError):
+        B.plan_attention([100, 0], [2, 2], 8, 4, 296, 100)
+    with pytest.raises(B.SledError):
+        B.plan_attention([100], [2], 0, 4, 296, 100)
